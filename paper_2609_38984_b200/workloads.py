@@ -1,0 +1,274 @@
+"""Seeded synthetic workloads shaped like the five benchmark configurations.
+
+This module serves both the CUDA path and the CPU oracle and therefore holds
+none of the method's arithmetic: it only describes shapes and integer budgets
+and draws Q/K/V tensors.  The tensors stand in for the activations of a
+world-action model (which are not available offline); their structure follows
+what the paper observes about action-to-future attention (Sec. 3.2): each
+future frame is attended by its own contiguous group of action queries, the
+attended region is a spatial hotspot that differs between frames, and the
+hotspot barely moves between consecutive denoising steps.
+
+Sequence order is [observed | future frame 0 .. F-1 | action]; tensors are
+[B, L, N_h, D], token-major.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+from concurrent.futures import ThreadPoolExecutor
+from typing import Dict, List, Optional, Tuple
+
+import numpy as np
+
+F32 = 0
+BF16 = 1
+
+
+def budgets_from_keep(keep: float, n_spatial: int) -> Tuple[int, int]:
+    """Integer per-frame budgets (K_c, K_s) for a keep ratio.
+
+    The paper only gives integer budgets (Table 5: 80 core + 104 anchors of 360)
+    and defines the pruning ratio as r = 1 - K/N_s (Sec. 5.4).  The rule used for
+    the benchmark shapes is K = round-half-up(keep * N_s) and a 10:13 split
+    (80:104) between core tokens and shared anchors.
+    """
+    k = int(math.floor(keep * n_spatial + 0.5))
+    k = max(0, min(k, n_spatial))
+    k_core = int(math.floor(k * 10.0 / 23.0 + 0.5))
+    return k_core, k - k_core
+
+
+@dataclasses.dataclass(frozen=True)
+class Workload:
+    name: str
+    batch: int
+    n_obs: int
+    n_frames: int
+    views: int
+    grid_h: int
+    grid_w: int
+    n_action: int
+    n_heads: int
+    head_dim: int
+    dtype: int
+    keep: float
+    steps: int
+    refresh: int
+    seed: int
+    blobs: int = 0          # hotspots per (view, frame); 0 = plain i.i.d. N(0,1)
+    rho: float = 0.8        # AR(1) coefficient of future/action tensors across steps
+    blob_logit: float = 4.0  # logit added at a hotspot centre
+    blob_sigma: float = 3.0  # hotspot width in patches
+    k_core: Optional[int] = None
+    k_anchor: Optional[int] = None
+
+    @property
+    def n_spatial(self) -> int:
+        return self.views * self.grid_h * self.grid_w
+
+    @property
+    def budgets(self) -> Tuple[int, int]:
+        if self.k_core is not None and self.k_anchor is not None:
+            return self.k_core, self.k_anchor
+        return budgets_from_keep(self.keep, self.n_spatial)
+
+    @property
+    def k_keep(self) -> int:
+        return sum(self.budgets)
+
+    @property
+    def seq_len(self) -> int:
+        return self.n_obs + self.n_frames * self.n_spatial + self.n_action
+
+    @property
+    def packed_len(self) -> int:
+        return self.n_obs + self.n_frames * self.k_keep + self.n_action
+
+    @property
+    def group(self) -> int:
+        return self.n_action // self.n_frames
+
+    @property
+    def row_elems(self) -> int:
+        return self.n_heads * self.head_dim
+
+    @property
+    def elem_bytes(self) -> int:
+        return 4 if self.dtype == F32 else 2
+
+    def with_(self, **kw) -> "Workload":
+        return dataclasses.replace(self, **kw)
+
+
+WORKLOADS: Dict[str, Workload] = {
+    # batch 1; 2 x 8x8 future tokens, 16 observed, 8 action; 2 heads x 32; fp32; i.i.d. N(0,1)
+    "tiny": Workload("tiny", 1, 16, 2, 1, 8, 8, 8, 2, 32, F32, 0.5, 3, 2, 0, blobs=0),
+    # 4 x 24x24 future, 576 observed, 32 action; 24 x 64; bf16
+    "single_view": Workload("single_view", 1, 576, 4, 1, 24, 24, 32, 24, 64, BF16, 0.25, 10, 2, 1, blobs=1),
+    # 8 x 32x32 future, 1024 observed, 64 action; 32 x 128; bf16; two hotspots per frame
+    "larger_imagination": Workload("larger_imagination", 1, 1024, 8, 1, 32, 32, 64, 32, 128, BF16, 0.3, 10, 2, 2, blobs=2),
+    # batch 8, 3 views x 4 x 24x24 future, 1728 observed, 32 action; 24 x 64; bf16
+    "multi_view": Workload("multi_view", 8, 1728, 4, 3, 24, 24, 32, 24, 64, BF16, 0.25, 10, 2, 3, blobs=1),
+}
+
+SWEEP_KEEPS = (0.1, 0.2, 0.3, 0.5, 1.0)
+SWEEP_REFRESH = (1, 2, 4)
+
+
+def sweep_workload(keep: float, refresh: int) -> Workload:
+    """The keep-ratio x refresh-interval sweep runs at the larger-imagination shape with seed 4."""
+    base = WORKLOADS["larger_imagination"]
+    return base.with_(name=f"sweep_keep{keep:g}_r{refresh}", keep=keep, refresh=refresh, seed=4)
+
+
+def refresh_schedule(steps: int, refresh: int) -> List[bool]:
+    """True where a denoising step is a full (refresh) step: every `refresh`-th step from step 0."""
+    return [(t % refresh) == 0 for t in range(steps)]
+
+
+# ----------------------------------------------------------------------------
+# bf16 helpers (storage only)
+# ----------------------------------------------------------------------------
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round float32 to bfloat16 (round to nearest even); returns uint16 bit patterns."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    rounded = u + (np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1)))
+    return (rounded >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+# ----------------------------------------------------------------------------
+# generator
+# ----------------------------------------------------------------------------
+_TENSOR_ID = {"q": 0, "k": 1, "v": 2}
+_CHUNK_ROWS = 512
+
+
+def _normal_rows(seed: int, step: int, tensor: int, b: int, n_rows: int, row_elems: int, stream: int) -> np.ndarray:
+    """[n_rows, row_elems] float32 N(0,1), reproducible per (seed, step, tensor, sample, stream), drawn in
+    parallel chunks with one counter-based generator key per chunk."""
+    out = np.empty((n_rows, row_elems), dtype=np.float32)
+    n_chunks = (n_rows + _CHUNK_ROWS - 1) // _CHUNK_ROWS
+
+    def fill(c: int) -> None:
+        lo = c * _CHUNK_ROWS
+        hi = min(n_rows, lo + _CHUNK_ROWS)
+        key = [(seed << 40) | (step << 20) | (tensor << 8) | stream, (b << 32) | c]
+        g = np.random.Generator(np.random.Philox(key=key))
+        out[lo:hi] = g.standard_normal((hi - lo, row_elems), dtype=np.float32)
+
+    if n_chunks == 1:
+        fill(0)
+    else:
+        with ThreadPoolExecutor(max_workers=8) as ex:
+            list(ex.map(fill, range(n_chunks)))
+    return out
+
+
+class Generator:
+    """Draws the Q/K/V tensors of one workload step by step.
+
+    Observed-token rows are fixed across steps.  Future and action rows follow
+    x_t = rho * x_{t-1} + sqrt(1 - rho^2) * n_t (tiny: rho = 0, fresh noise each
+    step).  When the workload has hotspots, each (sample, view, frame) carries
+    `blobs` Gaussian bumps whose centres start uniform on the patch grid and move
+    by at most one patch per axis per step; along a seeded unit direction
+    u[f, h] the future keys of frame f get amplitude a * bump(j) and the action
+    queries of the frame's query group get amplitude a, with a^2 / sqrt(D) =
+    blob_logit, so a hotspot centre raises the aligned logit by `blob_logit`.
+    """
+
+    def __init__(self, wl: Workload):
+        self.wl = wl
+        self._t = -1
+        self._base: Dict[str, np.ndarray] = {}
+        rng = np.random.Generator(np.random.Philox(key=[wl.seed, 0xB10B]))
+        if wl.blobs > 0:
+            self._centres = rng.uniform(
+                0.0, 1.0, size=(wl.batch, wl.views, wl.n_frames, wl.blobs, 2)
+            ) * np.array([wl.grid_h - 1, wl.grid_w - 1], dtype=np.float64)
+            u = rng.standard_normal((wl.n_frames, wl.n_heads, wl.head_dim))
+            self._u = (u / np.linalg.norm(u, axis=-1, keepdims=True)).astype(np.float32)
+        else:
+            self._centres = None
+            self._u = None
+        self._drift_rng = np.random.Generator(np.random.Philox(key=[wl.seed, 0xD21F7]))
+
+    # -- hotspot geometry -------------------------------------------------
+    def centres(self) -> Optional[np.ndarray]:
+        return None if self._centres is None else self._centres.copy()
+
+    def _bump(self) -> np.ndarray:
+        """[B, F, N_s] float32: sum of Gaussian bumps, within-frame order view-major."""
+        wl = self.wl
+        yy, xx = np.meshgrid(np.arange(wl.grid_h), np.arange(wl.grid_w), indexing="ij")
+        pos = np.stack([yy.reshape(-1), xx.reshape(-1)], axis=-1).astype(np.float64)  # [hw, 2]
+        c = self._centres  # [B, views, F, blobs, 2]
+        d2 = ((pos[None, None, None, None, :, :] - c[:, :, :, :, None, :]) ** 2).sum(-1)  # [B,views,F,blobs,hw]
+        g = np.exp(-d2 / (2.0 * wl.blob_sigma ** 2)).sum(axis=3)  # [B, views, F, hw]
+        g = np.transpose(g, (0, 2, 1, 3)).reshape(wl.batch, wl.n_frames, wl.n_spatial)
+        return g.astype(np.float32)
+
+    # -- stepping ---------------------------------------------------------
+    def next_step(self) -> Dict[str, np.ndarray]:
+        """Advance one denoising step; returns float32 arrays q, k, v of shape [B, L, N_h, D] whose values
+        are already rounded to the workload's storage type (bf16 workloads: bf16-representable)."""
+        wl = self.wl
+        self._t += 1
+        t = self._t
+        rho = wl.rho if wl.blobs > 0 else 0.0
+        n_fut = wl.n_frames * wl.n_spatial
+        out: Dict[str, np.ndarray] = {}
+        if t > 0 and self._centres is not None:
+            drift = self._drift_rng.uniform(-1.0, 1.0, size=self._centres.shape)
+            hi = np.array([wl.grid_h - 1, wl.grid_w - 1], dtype=np.float64)
+            self._centres = np.clip(self._centres + drift, 0.0, hi)
+        bump = self._bump() if self._centres is not None else None
+        amp = math.sqrt(wl.blob_logit * math.sqrt(wl.head_dim))
+        for name, tid in _TENSOR_ID.items():
+            if t == 0:
+                base = np.empty((wl.batch, wl.seq_len, wl.row_elems), dtype=np.float32)
+                for b in range(wl.batch):
+                    base[b] = _normal_rows(wl.seed, 0, tid, b, wl.seq_len, wl.row_elems, 0)
+                self._base[name] = base
+            else:
+                base = self._base[name]
+                c1 = np.float32(math.sqrt(1.0 - rho * rho))
+                for b in range(wl.batch):
+                    noise = _normal_rows(wl.seed, t, tid, b, wl.seq_len - wl.n_obs, wl.row_elems, 1)
+                    dyn = base[b, wl.n_obs:]
+                    dyn *= np.float32(rho)
+                    noise *= c1
+                    dyn += noise
+            x = base.reshape(wl.batch, wl.seq_len, wl.n_heads, wl.head_dim).copy()
+            if bump is not None and name == "k":
+                fut = x[:, wl.n_obs:wl.n_obs + n_fut].reshape(
+                    wl.batch, wl.n_frames, wl.n_spatial, wl.n_heads, wl.head_dim)
+                fut += np.float32(amp) * bump[:, :, :, None, None] * self._u[None, :, None, :, :]
+            if bump is not None and name == "q":
+                act = x[:, wl.n_obs + n_fut:].reshape(
+                    wl.batch, wl.n_frames, wl.group, wl.n_heads, wl.head_dim)
+                act += np.float32(amp) * self._u[None, :, None, :, :]
+            if wl.dtype == BF16:
+                x = bf16_bits_to_f32(f32_to_bf16_bits(x)).reshape(x.shape)
+            out[name] = x
+        return out
+
+
+def generate_steps(wl: Workload, n_steps: Optional[int] = None) -> List[Dict[str, np.ndarray]]:
+    g = Generator(wl)
+    return [g.next_step() for _ in range(wl.steps if n_steps is None else n_steps)]
+
+
+def random_scores(seed: int, batch: int, n_frames: int, n_spatial: int, ties: bool = False) -> np.ndarray:
+    """[B, F, N_s] float32 positive score arrays for testing selection alone; `ties` quantises them so
+    that many exact ties occur."""
+    rng = np.random.Generator(np.random.Philox(key=[seed, 0x5C0]))
+    s = rng.gamma(0.7, 1.0, size=(batch, n_frames, n_spatial)).astype(np.float32) / np.float32(n_spatial)
+    if ties:
+        s = (np.floor(s * np.float32(n_spatial * 4)) / np.float32(n_spatial * 4)).astype(np.float32)
+    return s
