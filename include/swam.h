@@ -1,0 +1,143 @@
+/*
+ * swam - one action-guided sparse denoising step of a world-action model's
+ * joint attention (Sparse-WAM), for NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Every call returns an int status (0 = SWAM_OK), never throws, never
+ * allocates device memory and, unless stated otherwise, never synchronises: work
+ * is enqueued on the caller's stream (`stream` is a cudaStream_t passed as
+ * void*; NULL is the default stream).  The caller owns every tensor and the
+ * workspace; the context owns host memory only.
+ *
+ * Notation (the paper's): B batch, N_o observed tokens, F future latent frames,
+ * N_s tokens per future frame, H action tokens, N_h heads, D head dim,
+ * g = H/F queries per frame-aligned group, K = K_c + K_s retained tokens per
+ * frame, L = N_o + F*N_s + H, L' = N_o + F*K + H.
+ * Sequence order: [observed | future frame 0 .. F-1 | action].
+ * Tensor layout: [B, L, N_h, D] contiguous (token-major rows of N_h*D elements),
+ * element type given by swam_shape.dtype.  "dev" = device pointer, "host" =
+ * host pointer.  Device pointers must be 16-byte aligned.
+ */
+#ifndef SWAM_H_
+#define SWAM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct swam_ctx swam_ctx;
+
+enum {
+  SWAM_OK = 0,
+  SWAM_ERR_INVALID_ARG = 1,  /* NULL / misaligned pointer, inconsistent shape */
+  SWAM_ERR_UNSUPPORTED = 2,  /* valid request without a kernel (e.g. head_dim, group size) */
+  SWAM_ERR_WORKSPACE = 3,    /* workspace missing or too small */
+  SWAM_ERR_STATE = 4,        /* reuse requested before any refresh */
+  SWAM_ERR_CUDA = 5,         /* a CUDA runtime call failed; see swam_last_error */
+  SWAM_ERR_DEVICE_CHECK = 6, /* a kernel met an out-of-range map entry or an impossible count */
+  SWAM_ERR_TIMEOUT = 7       /* a bounded device-side wait ran out */
+};
+
+enum { SWAM_F32 = 0, SWAM_BF16 = 1 };
+
+/* swam_step modes */
+enum {
+  SWAM_REUSE = 0,         /* sparse step: pack -> packed attention -> scatter with the cached maps */
+  SWAM_REFRESH_FULL = 1,  /* full step: dense attention (fills the cache) -> score -> select */
+  SWAM_REFRESH_LIGHT = 2  /* score (normaliser computed here) -> select -> pack -> packed attention -> scatter */
+};
+
+typedef struct {
+  int32_t batch, n_obs, n_frames, n_spatial, n_action, n_heads, head_dim;
+  int32_t k_core, k_anchor;   /* K_c, K_s; K_c + K_s <= N_s (Sec. 4.1) */
+  int32_t dtype;              /* SWAM_F32 | SWAM_BF16 */
+  float softmax_scale;        /* 0 => 1/sqrt(head_dim) */
+  float cv_beta;              /* coefficient of the cross-frame variation penalty; the paper uses 1.0 */
+  const float* query_weights; /* host, [H/F], non-negative, sums to 1; NULL => central half 2x outer quarters */
+} swam_shape;
+
+/* Context: validates the shape (H divisible by F, Eq. 8; K_c + K_s <= N_s; head_dim in {32, 64, 128};
+ * NULL weights need H/F divisible by 4) and fixes the workspace layout.  The shape (and the weights) are
+ * copied.  The current CUDA device at creation is the device every later call must run on. */
+int swam_create(const swam_shape* shape, swam_ctx** out_ctx);
+int swam_destroy(swam_ctx* ctx);
+
+/* Device workspace, caller-allocated (256-byte aligned).  It holds the cross-step state (scores, action-row
+ * normalisers, selection, maps, status word) and the packed Q/K/V/O buffers that swam_step uses.  Binding
+ * zeroes the status word and clears the "has selection" state (synchronous, small). */
+int swam_workspace_bytes(const swam_ctx* ctx, size_t* bytes);
+int swam_bind_workspace(swam_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/* (1) Action-to-future scoring, Eq. 12 (extraction form of Eq. 1-2):
+ *   S[b,f,j] = 1/N_h * sum_{i in I_f} sum_h alpha_i * exp(scale * q_{i,h} . k_{(f,j),h} - lambda[b,h,i])
+ * q, k: dev, full tensors [B, L, N_h, D] (only the action rows of q and, when lambda is given, only the
+ * future rows of k are read).  lse_action: dev float [B, N_h, H], log-sum-exp of each action query over ALL
+ * L keys (Sec. 4.2 "reuses the original normalisers"); NULL => computed here over all L keys (uses workspace
+ * scratch).  scores: dev float [B, F, N_s].  quality: dev float [B, 3] = (R, E, Q) of Eq. 9, or NULL. */
+int swam_score(swam_ctx* ctx, const void* q, const void* k, const float* lse_action,
+               float* scores, float* quality, void* stream);
+
+/* (2) Selection and packing metadata, Eq. 4-6, 10-11 with one profiled layer (V = V_all = S):
+ * pool = top (N_s - K_s) of max_f S; core_f = top K_c of S[f] within the pool; anchors = top K_s of
+ * mu_j / (1 + beta * CV_j) over positions that are core in no frame (population std, fp64, mu_j = 0 => CV_j = 0).
+ * Equal keys go to the lower index.  scores: dev float [B, F, N_s] (finite).  sel_idx: dev int32 [B, F, K]
+ * ascending spatial indices; pack_map: dev int32 [B, L'] original row of each packed row (strictly increasing);
+ * inv_map: dev int32 [B, L] packed row of each original row, -1 if omitted.  Any output may be NULL. */
+int swam_select(swam_ctx* ctx, const float* scores, int32_t* sel_idx, int32_t* pack_map, int32_t* inv_map,
+                void* stream);
+
+/* (3) Packing (Sec. 4.2): xp[b, p, :] = x[b, pack_map[b, p], :] for x in {q, k, v}; xp: dev [B, L', N_h, D].
+ * Any of the three pairs may be NULL/NULL.  Out-of-range map entries are skipped and flagged in the status word. */
+int swam_pack(swam_ctx* ctx, const void* q, const void* k, const void* v, const int32_t* pack_map,
+              void* qp, void* kp, void* vp, void* stream);
+
+/* (4) Joint attention over a compact (or the full) sequence, plain softmax attention with full visibility:
+ * out[b,r,h,:] = sum_c softmax_c(scale * q[b,r,h,:] . k[b,c,h,:]) v[b,c,h,:], tensors [B, seq_len, N_h, D].
+ * lse: dev float [B, N_h, seq_len] natural-log normalisers, or NULL.  bf16: fp32 accumulation. */
+int swam_sparse_attn(swam_ctx* ctx, const void* qp, const void* kp, const void* vp, int32_t seq_len,
+                     void* out_p, float* lse, void* stream);
+
+/* (5) Scatter back, Eq. 7: out[b, pack_map[b,p], :] = out_p[b, p, :]; every omitted row takes cached's row.
+ * cached may equal out (in place: omitted rows are left untouched, which is Eq. 7 when out still holds the
+ * last full step's result).  inv_map is only read when cached != out. */
+int swam_scatter(swam_ctx* ctx, const void* out_p, const int32_t* pack_map, const int32_t* inv_map,
+                 const void* cached, void* out, void* stream);
+
+/* One denoising step (Sec. 4.2).  q, k, v, out: dev [B, L, N_h, D]; out persists across steps and holds the
+ * last full step's result on omitted rows.  mode: SWAM_REFRESH_FULL runs dense attention into out, scores the
+ * future tokens with the dense pass's action-row normalisers, selects and builds the maps; SWAM_REUSE packs by
+ * the cached maps, attends over L' tokens and scatters into out (SWAM_ERR_STATE before any refresh);
+ * SWAM_REFRESH_LIGHT recomputes normalisers, scores and selection from this step's q, k without a dense pass,
+ * then runs the sparse step with the new maps. */
+int swam_step(swam_ctx* ctx, const void* q, const void* k, const void* v, int32_t mode, void* out, void* stream);
+
+/* The same step for callers whose tensors live in (pinned) host memory: copies q, k, v into a device staging
+ * area, runs swam_step, copies out back; all on `stream`, no synchronisation.  The staging area (4 full
+ * tensors, caller-allocated, dev) is bound once; on SWAM_REUSE steps the staged out of the previous step is
+ * the cache, so staging must not be touched between steps. */
+int swam_host_io_bytes(const swam_ctx* ctx, size_t* bytes);
+int swam_bind_host_io(swam_ctx* ctx, void* dev_ptr, size_t bytes);
+int swam_step_host(swam_ctx* ctx, const void* q_host, const void* k_host, const void* v_host, int32_t mode,
+                   void* out_host, void* stream);
+
+/* Device pointers (inside the workspace) of the state swam_step keeps; any argument may be NULL. */
+int swam_get_selection(const swam_ctx* ctx, const int32_t** sel_idx, const int32_t** pack_map,
+                       const int32_t** inv_map);
+int swam_get_scores(const swam_ctx* ctx, const float** scores, const float** lse_action, const float** quality);
+
+/* Synchronises `stream`, reads and clears the device status word; returns SWAM_OK, SWAM_ERR_DEVICE_CHECK,
+ * SWAM_ERR_TIMEOUT or SWAM_ERR_CUDA. */
+int swam_check(swam_ctx* ctx, void* stream);
+
+/* Number of kernels this context has launched so far (host-side counter). */
+int swam_launch_count(const swam_ctx* ctx, int64_t* count);
+
+const char* swam_last_error(const swam_ctx* ctx);
+const char* swam_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SWAM_H_ */

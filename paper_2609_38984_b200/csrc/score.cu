@@ -1,0 +1,479 @@
+// Action-to-future scoring (Eq. 12) and the action-row normalisers it needs.
+//
+// The scorer is a stream over the future keys: every key row is read exactly once, multiplied against the
+// g = H/F action queries aligned with its frame (Eq. 8), and reduced over heads and queries into one float.
+// At g = 8 that is 8 FMAs per loaded bf16 element, more than the FP32 pipes sustain at HBM speed, so the
+// bf16 path feeds the (skinny) products to mma.sync m16n8k16 directly from 16-byte global loads: because a
+// dot product does not care about the order of its terms, each thread's 16-byte chunk of a key row is used
+// as four k-slots of two MMAs and the query fragment is the same 16-byte chunk of the query row.
+#include "swam_internal.cuh"
+
+namespace swam {
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p));
+  return r;
+}
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+struct ScoreParams {
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k;
+  const float* lse;  // [B, N_h, H]
+  float* scores;     // [B, F, N_s]
+  int n_obs, F, N_s, H, N_h, L, g;
+  float scale_log2, inv_nh;
+  Alpha alpha;
+};
+
+constexpr int kScoreThreads = 256;
+constexpr int kScoreKeys = 32;  // keys per CTA: 2 m-tiles of 16
+constexpr int kHeadGroups = 4;
+
+// smem: query fragments [N_h][D/32][NT][32] uint4, lambda*log2e [N_h][NT*8], partial sums [4][32]
+template <int D, int NT>
+__global__ void __launch_bounds__(kScoreThreads, 2) score_bf16_kernel(const ScoreParams p) {
+  constexpr int KB = D / 32;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint4* q_frag = reinterpret_cast<uint4*>(smem_raw);
+  float* lam2 = reinterpret_cast<float*>(q_frag + (size_t)p.N_h * KB * NT * 32);
+  float* red = lam2 + p.N_h * NT * 8;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int f = blockIdx.y, b = blockIdx.z;
+  const int key0 = blockIdx.x * kScoreKeys;
+  const int64_t act0 = (int64_t)p.n_obs + (int64_t)p.F * p.N_s;
+  const int64_t tok = (int64_t)p.N_h * D;
+
+  // stage this frame's query group as MMA B fragments (zero beyond the group)
+  const int n_frag = p.N_h * KB * NT * 32;
+  for (int i = tid; i < n_frag; i += kScoreThreads) {
+    const int ln = i & 31;
+    const int nt = (i >> 5) % NT;
+    const int kb = ((i >> 5) / NT) % KB;
+    const int h = (i >> 5) / (NT * KB);
+    const int n = nt * 8 + (ln >> 2), t = ln & 3;
+    uint4 val = make_uint4(0, 0, 0, 0);
+    if (n < p.g) {
+      const __nv_bfloat16* src = p.q + ((int64_t)b * p.L + act0 + (int64_t)f * p.g + n) * tok + (int64_t)h * D +
+                                 kb * 32 + t * 8;
+      val = *reinterpret_cast<const uint4*>(src);
+    }
+    q_frag[i] = val;
+  }
+  for (int i = tid; i < p.N_h * NT * 8; i += kScoreThreads) {
+    const int n = i % (NT * 8), h = i / (NT * 8);
+    lam2[i] = (n < p.g) ? p.lse[((int64_t)b * p.N_h + h) * p.H + f * p.g + n] * kLog2e : 0.f;
+  }
+  __syncthreads();
+
+  const int mt = warp & 1, hg = warp >> 1;
+  const int gq = lane >> 2, t = lane & 3;
+  const int r0 = key0 + mt * 16 + gq, r1 = r0 + 8;
+  const bool v0 = r0 < p.N_s, v1 = r1 < p.N_s;
+  const __nv_bfloat16* kbase = p.k + ((int64_t)b * p.L + p.n_obs + (int64_t)f * p.N_s) * tok + t * 8;
+  const __nv_bfloat16* k0 = kbase + (int64_t)(v0 ? r0 : 0) * tok;
+  const __nv_bfloat16* k1 = kbase + (int64_t)(v1 ? r1 : 0) * tok;
+
+  float w[NT][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    w[nt][0] = p.alpha.w[nt * 8 + 2 * t];
+    w[nt][1] = p.alpha.w[nt * 8 + 2 * t + 1];
+  }
+
+  float sum0 = 0.f, sum1 = 0.f;
+  uint4 a0[2][KB], a1[2][KB];
+  const uint4 zero = make_uint4(0, 0, 0, 0);
+  auto load = [&](int h, int buf) {
+#pragma unroll
+    for (int kb = 0; kb < KB; ++kb) {
+      a0[buf][kb] = v0 ? ldg_stream(k0 + (int64_t)h * D + kb * 32) : zero;
+      a1[buf][kb] = v1 ? ldg_stream(k1 + (int64_t)h * D + kb * 32) : zero;
+    }
+  };
+  auto compute = [&](int h, int buf) {
+    float c[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+#pragma unroll
+    for (int kb = 0; kb < KB; ++kb) {
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const uint4 bq = q_frag[((h * KB + kb) * NT + nt) * 32 + lane];
+        mma_bf16_16816(c[nt], a0[buf][kb].x, a1[buf][kb].x, a0[buf][kb].y, a1[buf][kb].y, bq.x, bq.y);
+        mma_bf16_16816(c[nt], a0[buf][kb].z, a1[buf][kb].z, a0[buf][kb].w, a1[buf][kb].w, bq.z, bq.w);
+      }
+    }
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const float l0 = lam2[h * NT * 8 + nt * 8 + 2 * t], l1 = lam2[h * NT * 8 + nt * 8 + 2 * t + 1];
+      sum0 += w[nt][0] * exp2f(c[nt][0] * p.scale_log2 - l0) + w[nt][1] * exp2f(c[nt][1] * p.scale_log2 - l1);
+      sum1 += w[nt][0] * exp2f(c[nt][2] * p.scale_log2 - l0) + w[nt][1] * exp2f(c[nt][3] * p.scale_log2 - l1);
+    }
+  };
+
+  // heads hg, hg+4, ... with the next head's keys in flight while this head's products run
+  int h = hg;
+  if (h < p.N_h) load(h, 0);
+  for (; h < p.N_h; h += 2 * kHeadGroups) {
+    const int h1 = h + kHeadGroups, h2 = h + 2 * kHeadGroups;
+    if (h1 < p.N_h) load(h1, 1);
+    compute(h, 0);
+    if (h1 < p.N_h) {
+      if (h2 < p.N_h) load(h2, 0);
+      compute(h1, 1);
+    }
+  }
+
+  sum0 += __shfl_xor_sync(0xffffffffu, sum0, 1);
+  sum0 += __shfl_xor_sync(0xffffffffu, sum0, 2);
+  sum1 += __shfl_xor_sync(0xffffffffu, sum1, 1);
+  sum1 += __shfl_xor_sync(0xffffffffu, sum1, 2);
+  if (t == 0) {
+    red[hg * kScoreKeys + mt * 16 + gq] = sum0;
+    red[hg * kScoreKeys + mt * 16 + gq + 8] = sum1;
+  }
+  __syncthreads();
+  if (tid < kScoreKeys && key0 + tid < p.N_s) {
+    const float s = (red[tid] + red[kScoreKeys + tid]) + (red[2 * kScoreKeys + tid] + red[3 * kScoreKeys + tid]);
+    p.scores[((int64_t)b * p.F + f) * p.N_s + key0 + tid] = s * p.inv_nh;
+  }
+}
+
+// fp32 inputs: one warp per key, lanes across the head dimension
+struct ScoreParamsF32 {
+  const float* q;
+  const float* k;
+  const float* lse;
+  float* scores;
+  int n_obs, F, N_s, H, N_h, D, L, g;
+  float scale, inv_nh;
+  Alpha alpha;
+};
+
+__global__ void __launch_bounds__(256) score_f32_kernel(const ScoreParamsF32 p) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int f = blockIdx.y, b = blockIdx.z;
+  const int j = blockIdx.x * 8 + warp;
+  if (j >= p.N_s) return;
+  const int64_t tok = (int64_t)p.N_h * p.D;
+  const int64_t act0 = (int64_t)p.n_obs + (int64_t)p.F * p.N_s;
+  const float* kt = p.k + ((int64_t)b * p.L + p.n_obs + (int64_t)f * p.N_s + j) * tok;
+  float acc = 0.f;
+  for (int a = 0; a < p.g; ++a) {
+    const int i = f * p.g + a;
+    const float* qt = p.q + ((int64_t)b * p.L + act0 + i) * tok;
+    for (int h = 0; h < p.N_h; ++h) {
+      float dot = 0.f;
+      for (int d = lane; d < p.D; d += 32) dot = fmaf(qt[h * p.D + d], kt[h * p.D + d], dot);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      acc += p.alpha.w[a] * expf(p.scale * dot - p.lse[((int64_t)b * p.N_h + h) * p.H + i]);
+    }
+  }
+  if (lane == 0) p.scores[((int64_t)b * p.F + f) * p.N_s + j] = acc * p.inv_nh;
+}
+
+// ---- layer quality (Eq. 9): R = sum S / F, E = mean normalised spatial entropy, Q = R (1 - E) ----------
+__device__ double block_sum(double v, double* sh) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if (lane == 0) sh[warp] = v;
+  __syncthreads();
+  double tot = 0.0;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += sh[w];
+  return tot;
+}
+
+__global__ void __launch_bounds__(256) quality_kernel(const float* scores, float* quality, int F, int N_s) {
+  __shared__ double sh[8];
+  const int b = blockIdx.x;
+  const float* s = scores + (int64_t)b * F * N_s;
+  double total = 0.0, ent = 0.0;
+  for (int f = 0; f < F; ++f) {
+    double part = 0.0;
+    for (int j = threadIdx.x; j < N_s; j += blockDim.x) part += (double)s[f * N_s + j];
+    const double fs = block_sum(part, sh);
+    total += fs;
+    double e = 0.0;
+    if (fs > 0.0) {
+      for (int j = threadIdx.x; j < N_s; j += blockDim.x) {
+        const double pj = (double)s[f * N_s + j] / fs;
+        if (pj > 0.0) e -= pj * log(pj);
+      }
+    }
+    ent += block_sum(e, sh);
+  }
+  if (threadIdx.x == 0) {
+    const double R = total / (double)F;
+    const double E = ent / ((double)F * log((double)N_s));
+    quality[b * 3 + 0] = (float)R;
+    quality[b * 3 + 1] = (float)E;
+    quality[b * 3 + 2] = (float)(R * (1.0 - E));
+  }
+}
+
+// ---- action-row normalisers over all L keys -----------------------------------------------------------
+// bf16: each CTA takes 128 keys (8 warps x 16), loops over heads, multiplies against all H action queries
+// (NT = H/8 column tiles) and keeps a running (max, sum) per query in the log2 domain; the per-CTA partials
+// go to scratch [B, chunks, N_h, H] and a second kernel merges them.
+constexpr int kLseKeys = 128;
+constexpr int kLseThreads = 256;
+
+struct LseParams {
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k;
+  float2* partial;
+  int H, N_h, L, n_chunks, NT;
+  float scale_log2;
+};
+
+__device__ __forceinline__ void merge_ms(float& m, float& s, float m2, float s2) {
+  const float mn = fmaxf(m, m2);
+  if (mn == -INFINITY) { m = mn; s = 0.f; return; }
+  s = s * exp2f(m - mn) + s2 * exp2f(m2 - mn);
+  m = mn;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kLseThreads) lse_partial_bf16_kernel(const LseParams p) {
+  constexpr int KB = D / 32;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint4* q_frag = reinterpret_cast<uint4*>(smem_raw);                        // [KB][NT][32]
+  float2* wpart = reinterpret_cast<float2*>(q_frag + (size_t)KB * p.NT * 32);  // [8 warps][NT*8]
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int chunk = blockIdx.x, b = blockIdx.y;
+  const int64_t tok = (int64_t)p.N_h * D;
+  const int gq = lane >> 2, t = lane & 3;
+  const int r0 = chunk * kLseKeys + warp * 16 + gq, r1 = r0 + 8;
+  const bool v0 = r0 < p.L, v1 = r1 < p.L;
+  const __nv_bfloat16* k0 = p.k + ((int64_t)b * p.L + (v0 ? r0 : 0)) * tok + t * 8;
+  const __nv_bfloat16* k1 = p.k + ((int64_t)b * p.L + (v1 ? r1 : 0)) * tok + t * 8;
+  const int64_t act0 = (int64_t)p.L - p.H;
+  const int n_frag = KB * p.NT * 32;
+  const uint4 zero = make_uint4(0, 0, 0, 0);
+
+  for (int h = 0; h < p.N_h; ++h) {
+    __syncthreads();  // previous head's fragments and partials are no longer read
+    for (int i = tid; i < n_frag; i += kLseThreads) {
+      const int ln = i & 31;
+      const int nt = (i >> 5) % p.NT;
+      const int kb = (i >> 5) / p.NT;
+      const int n = nt * 8 + (ln >> 2);
+      uint4 val = zero;
+      if (n < p.H)
+        val = *reinterpret_cast<const uint4*>(p.q + ((int64_t)b * p.L + act0 + n) * tok + (int64_t)h * D + kb * 32 +
+                                              (ln & 3) * 8);
+      q_frag[i] = val;
+    }
+    uint4 a0[KB], a1[KB];
+#pragma unroll
+    for (int kb = 0; kb < KB; ++kb) {
+      a0[kb] = v0 ? ldg_stream(k0 + (int64_t)h * D + kb * 32) : zero;
+      a1[kb] = v1 ? ldg_stream(k1 + (int64_t)h * D + kb * 32) : zero;
+    }
+    __syncthreads();
+    for (int nt = 0; nt < p.NT; ++nt) {
+      float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int kb = 0; kb < KB; ++kb) {
+        const uint4 bq = q_frag[(kb * p.NT + nt) * 32 + lane];
+        mma_bf16_16816(c, a0[kb].x, a1[kb].x, a0[kb].y, a1[kb].y, bq.x, bq.y);
+        mma_bf16_16816(c, a0[kb].z, a1[kb].z, a0[kb].w, a1[kb].w, bq.z, bq.w);
+      }
+      // columns 2t, 2t+1; rows gq (c0, c1) and gq+8 (c2, c3)
+      float x00 = v0 ? c[0] * p.scale_log2 : -INFINITY, x01 = v0 ? c[1] * p.scale_log2 : -INFINITY;
+      float x10 = v1 ? c[2] * p.scale_log2 : -INFINITY, x11 = v1 ? c[3] * p.scale_log2 : -INFINITY;
+      float m0 = x00, s0 = (x00 == -INFINITY) ? 0.f : 1.f;
+      float m1 = x01, s1 = (x01 == -INFINITY) ? 0.f : 1.f;
+      merge_ms(m0, s0, x10, (x10 == -INFINITY) ? 0.f : 1.f);
+      merge_ms(m1, s1, x11, (x11 == -INFINITY) ? 0.f : 1.f);
+#pragma unroll
+      for (int o = 4; o < 32; o <<= 1) {
+        const float om0 = __shfl_xor_sync(0xffffffffu, m0, o), os0 = __shfl_xor_sync(0xffffffffu, s0, o);
+        const float om1 = __shfl_xor_sync(0xffffffffu, m1, o), os1 = __shfl_xor_sync(0xffffffffu, s1, o);
+        merge_ms(m0, s0, om0, os0);
+        merge_ms(m1, s1, om1, os1);
+      }
+      if (gq == 0) {
+        wpart[warp * p.NT * 8 + nt * 8 + 2 * t] = make_float2(m0, s0);
+        wpart[warp * p.NT * 8 + nt * 8 + 2 * t + 1] = make_float2(m1, s1);
+      }
+    }
+    __syncthreads();
+    for (int n = tid; n < p.H; n += kLseThreads) {
+      float m = -INFINITY, s = 0.f;
+      for (int w = 0; w < 8; ++w) {
+        const float2 ws = wpart[w * p.NT * 8 + n];
+        merge_ms(m, s, ws.x, ws.y);
+      }
+      p.partial[(((int64_t)b * p.n_chunks + chunk) * p.N_h + h) * p.H + n] = make_float2(m, s);
+    }
+  }
+}
+
+// merges the per-chunk partials: lambda = ln2 * (m + log2 s)
+__global__ void lse_merge_kernel(const float2* partial, float* lse, int n_chunks, int N_h, int H) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  const int b = blockIdx.y;
+  if (i >= N_h * H) return;
+  float m = -INFINITY, s = 0.f;
+  for (int c = 0; c < n_chunks; ++c) {
+    const float2 ms = partial[((int64_t)b * n_chunks + c) * N_h * H + i];
+    merge_ms(m, s, ms.x, ms.y);
+  }
+  lse[(int64_t)b * N_h * H + i] = (m + log2f(s)) * 0.6931471805599453f;
+}
+
+// fp32: one CTA per (b, h, i); threads stride over keys with a running (max, sum) in natural-log units
+__global__ void __launch_bounds__(128) lse_f32_kernel(const float* q, const float* k, float* lse, int L, int H,
+                                                      int N_h, int D, float scale) {
+  __shared__ float sm[4], ss[4];
+  const int i = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int64_t tok = (int64_t)N_h * D;
+  const float* qt = q + ((int64_t)b * L + (L - H) + i) * tok + (int64_t)h * D;
+  float m = -INFINITY, s = 0.f;
+  for (int c = threadIdx.x; c < L; c += blockDim.x) {
+    const float* kt = k + ((int64_t)b * L + c) * tok + (int64_t)h * D;
+    float dot = 0.f;
+    for (int d = 0; d < D; ++d) dot = fmaf(qt[d], kt[d], dot);
+    const float x = dot * scale;
+    const float mn = fmaxf(m, x);
+    s = s * expf(m - mn) + expf(x - mn);
+    m = mn;
+  }
+  auto merge = [](float& m, float& s, float m2, float s2) {
+    const float mn = fmaxf(m, m2);
+    if (mn == -INFINITY) { s = 0.f; m = mn; return; }
+    s = s * expf(m - mn) + s2 * expf(m2 - mn);
+    m = mn;
+  };
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
+    merge(m, s, om, os);
+  }
+  if ((threadIdx.x & 31) == 0) { sm[threadIdx.x >> 5] = m; ss[threadIdx.x >> 5] = s; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) merge(m, s, sm[w], ss[w]);
+    lse[((int64_t)b * N_h + h) * H + i] = m + logf(s);
+  }
+}
+
+template <int D, int NT>
+cudaError_t launch_score_bf16(const Dims& d, const ScoreParams& p, cudaStream_t st) {
+  const size_t smem = (size_t)d.N_h * (D / 32) * NT * 32 * sizeof(uint4) + (size_t)d.N_h * NT * 8 * sizeof(float) +
+                      kHeadGroups * kScoreKeys * sizeof(float);
+  if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
+  cudaError_t e = cudaFuncSetAttribute(score_bf16_kernel<D, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid((d.N_s + kScoreKeys - 1) / kScoreKeys, d.F, d.B);
+  score_bf16_kernel<D, NT><<<grid, kScoreThreads, smem, st>>>(p);
+  return cudaGetLastError();
+}
+
+template <int D>
+cudaError_t launch_score_bf16_d(const Dims& d, const ScoreParams& p, cudaStream_t st) {
+  const int nt = (d.g + 7) / 8;
+  switch (nt) {
+    case 1: return launch_score_bf16<D, 1>(d, p, st);
+    case 2: return launch_score_bf16<D, 2>(d, p, st);
+    case 3: case 4: return launch_score_bf16<D, 4>(d, p, st);
+    default: return cudaErrorInvalidConfiguration;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_score(const Dims& d, const Alpha& alpha, const void* q, const void* k, const float* lse,
+                         float* scores, cudaStream_t st, int* launches) {
+  ++*launches;
+  if (d.dtype == 0) {
+    ScoreParamsF32 p{(const float*)q, (const float*)k, lse, scores, d.n_obs, d.F, d.N_s, d.H,
+                     d.N_h, d.D, d.L, d.g, d.scale, 1.0f / (float)d.N_h, alpha};
+    dim3 grid((d.N_s + 7) / 8, d.F, d.B);
+    score_f32_kernel<<<grid, 256, 0, st>>>(p);
+    return cudaGetLastError();
+  }
+  ScoreParams p{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, lse, scores, d.n_obs, d.F, d.N_s, d.H,
+                d.N_h, d.L, d.g, d.scale * kLog2e, 1.0f / (float)d.N_h, alpha};
+  switch (d.D) {
+    case 32: return launch_score_bf16_d<32>(d, p, st);
+    case 64: return launch_score_bf16_d<64>(d, p, st);
+    case 128: return launch_score_bf16_d<128>(d, p, st);
+    default: return cudaErrorInvalidConfiguration;
+  }
+}
+
+cudaError_t launch_quality(const Dims& d, const float* scores, float* quality, cudaStream_t st, int* launches) {
+  ++*launches;
+  quality_kernel<<<d.B, 256, 0, st>>>(scores, quality, d.F, d.N_s);
+  return cudaGetLastError();
+}
+
+size_t lse_scratch_bytes(const Dims& d) {
+  if (d.dtype == 0) return 0;
+  const size_t chunks = (d.L + kLseKeys - 1) / kLseKeys;
+  return (size_t)d.B * chunks * d.N_h * d.H * sizeof(float2);
+}
+
+cudaError_t launch_action_lse(const Dims& d, const void* q, const void* k, float* lse, void* scratch,
+                              cudaStream_t st, int* launches) {
+  if (d.dtype == 0) {
+    ++*launches;
+    dim3 grid(d.H, d.N_h, d.B);
+    lse_f32_kernel<<<grid, 128, 0, st>>>((const float*)q, (const float*)k, lse, d.L, d.H, d.N_h, d.D, d.scale);
+    return cudaGetLastError();
+  }
+  const int n_chunks = (d.L + kLseKeys - 1) / kLseKeys;
+  const int NT = (d.H + 7) / 8;
+  LseParams p{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (float2*)scratch, d.H, d.N_h, d.L, n_chunks, NT,
+              d.scale * kLog2e};
+  const size_t smem = (size_t)(d.D / 32) * NT * 32 * sizeof(uint4) + (size_t)8 * NT * 8 * sizeof(float2);
+  if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
+  dim3 grid(n_chunks, d.B);
+  cudaError_t e = cudaSuccess;
+  *launches += 2;
+  switch (d.D) {
+    case 32:
+      e = cudaFuncSetAttribute(lse_partial_bf16_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e == cudaSuccess) lse_partial_bf16_kernel<32><<<grid, kLseThreads, smem, st>>>(p);
+      break;
+    case 64:
+      e = cudaFuncSetAttribute(lse_partial_bf16_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e == cudaSuccess) lse_partial_bf16_kernel<64><<<grid, kLseThreads, smem, st>>>(p);
+      break;
+    case 128:
+      e = cudaFuncSetAttribute(lse_partial_bf16_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e == cudaSuccess) lse_partial_bf16_kernel<128><<<grid, kLseThreads, smem, st>>>(p);
+      break;
+    default: return cudaErrorInvalidConfiguration;
+  }
+  if (e != cudaSuccess) return e;
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  dim3 g2((d.N_h * d.H + 127) / 128, d.B);
+  lse_merge_kernel<<<g2, 128, 0, st>>>((const float2*)scratch, lse, n_chunks, d.N_h, d.H);
+  return cudaGetLastError();
+}
+
+}  // namespace swam

@@ -1,0 +1,361 @@
+// C-ABI layer of libswam: context, validation, workspace layout, and the step state machine.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "../../include/swam.h"
+#include "swam_internal.cuh"
+
+using namespace swam;
+
+struct swam_ctx {
+  Dims d;
+  Alpha alpha;
+  int device;
+  // workspace (device)
+  unsigned char* ws;
+  size_t ws_bytes;
+  size_t off_status, off_scores, off_quality, off_lse, off_sel, off_pack, off_inv, off_scratch, off_qp, off_kp,
+      off_vp, off_op, ws_need;
+  bool has_selection;
+  // host-io staging (device)
+  unsigned char* io;
+  size_t io_need;
+  int launches_i;
+  int64_t launches;
+  char err[256];
+};
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int fail(swam_ctx* c, int code, const char* msg) {
+  if (c) snprintf(c->err, sizeof(c->err), "%s", msg);
+  return code;
+}
+int fail_cuda(swam_ctx* c, cudaError_t e, const char* where) {
+  if (c) snprintf(c->err, sizeof(c->err), "%s: %s", where, cudaGetErrorString(e));
+  return SWAM_ERR_CUDA;
+}
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+size_t elem_bytes(const Dims& d) { return d.dtype == SWAM_F32 ? 4 : 2; }
+size_t full_bytes(const Dims& d) { return (size_t)d.B * d.L * d.N_h * d.D * elem_bytes(d); }
+size_t packed_bytes(const Dims& d) { return (size_t)d.B * d.Lp * d.N_h * d.D * elem_bytes(d); }
+
+void count(swam_ctx* c) {
+  c->launches += c->launches_i;
+  c->launches_i = 0;
+}
+
+int run_attention(swam_ctx* c, const void* q, const void* k, const void* v, int n, void* out, float* lse, int lse_row0,
+                  int lse_rows, cudaStream_t st) {
+  AttnArgs a{q, k, v, out, lse, lse_row0, lse_rows, c->d.B, n, c->d.N_h, c->d.D, c->d.scale};
+  cudaError_t e = (c->d.dtype == SWAM_F32) ? launch_attn_f32(a, st, &c->launches_i)
+                                           : launch_attn_bf16_mma(a, st, &c->launches_i);
+  count(c);
+  if (e != cudaSuccess) return fail_cuda(c, e, "attention launch");
+  return SWAM_OK;
+}
+
+int need_ws(swam_ctx* c) {
+  if (!c->ws) return fail(c, SWAM_ERR_WORKSPACE, "no workspace bound");
+  return SWAM_OK;
+}
+
+int check_device(swam_ctx* c) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail_cuda(c, e, "cudaGetDevice");
+  if (dev != c->device) return fail(c, SWAM_ERR_INVALID_ARG, "current device differs from the context's device");
+  return SWAM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* swam_version(void) { return "swam 0.1 (sm_100a)"; }
+
+const char* swam_last_error(const swam_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+int swam_create(const swam_shape* s, swam_ctx** out_ctx) {
+  if (!s || !out_ctx) return SWAM_ERR_INVALID_ARG;
+  *out_ctx = nullptr;
+  if (s->batch <= 0 || s->n_obs < 0 || s->n_frames <= 0 || s->n_spatial <= 0 || s->n_action <= 0 || s->n_heads <= 0 ||
+      s->k_core < 0 || s->k_anchor < 0)
+    return SWAM_ERR_INVALID_ARG;
+  if (s->n_action % s->n_frames != 0) return SWAM_ERR_INVALID_ARG;          // Eq. 8 needs H divisible by F
+  if (s->k_core + s->k_anchor > s->n_spatial) return SWAM_ERR_INVALID_ARG;   // K_c + K_s <= N_s
+  if (s->dtype != SWAM_F32 && s->dtype != SWAM_BF16) return SWAM_ERR_INVALID_ARG;
+  if (!(s->softmax_scale >= 0.f) || !(s->cv_beta >= 0.f)) return SWAM_ERR_INVALID_ARG;
+  if (s->head_dim != 32 && s->head_dim != 64 && s->head_dim != 128) return SWAM_ERR_UNSUPPORTED;
+  const int g = s->n_action / s->n_frames;
+  if (g > kMaxGroup) return SWAM_ERR_UNSUPPORTED;
+  if (!s->query_weights && (g % 4) != 0) return SWAM_ERR_INVALID_ARG;
+  const long long L = (long long)s->n_obs + (long long)s->n_frames * s->n_spatial + s->n_action;
+  if (L > (1 << 24) || (long long)s->batch * L > (1ll << 30)) return SWAM_ERR_UNSUPPORTED;
+
+  swam_ctx* c = new (std::nothrow) swam_ctx();
+  if (!c) return SWAM_ERR_INVALID_ARG;
+  memset(c, 0, sizeof(*c));
+  Dims& d = c->d;
+  d.B = s->batch; d.n_obs = s->n_obs; d.F = s->n_frames; d.N_s = s->n_spatial; d.H = s->n_action;
+  d.N_h = s->n_heads; d.D = s->head_dim; d.Kc = s->k_core; d.Ks = s->k_anchor; d.K = d.Kc + d.Ks;
+  d.L = (int)L; d.Lp = d.n_obs + d.F * d.K + d.H; d.g = g; d.dtype = s->dtype;
+  d.scale = s->softmax_scale > 0.f ? s->softmax_scale : 1.0f / sqrtf((float)d.D);
+  d.beta = s->cv_beta;
+  if (s->query_weights) {
+    double sum = 0.0;
+    for (int i = 0; i < g; ++i) {
+      if (!(s->query_weights[i] >= 0.f)) { delete c; return SWAM_ERR_INVALID_ARG; }
+      c->alpha.w[i] = s->query_weights[i];
+      sum += s->query_weights[i];
+    }
+    if (fabs(sum - 1.0) > 1e-4) { delete c; return SWAM_ERR_INVALID_ARG; }
+  } else {
+    // central half of the group weighs twice the outer quarters; normalised: 2/(3g) outside, 4/(3g) inside
+    for (int i = 0; i < g; ++i)
+      c->alpha.w[i] = (float)(((i >= g / 4 && i < g - g / 4) ? 4.0 : 2.0) / (3.0 * g));
+  }
+  if (select_smem_bytes(d) > 227 * 1024) { delete c; return SWAM_ERR_UNSUPPORTED; }
+  if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return SWAM_ERR_CUDA; }
+
+  // workspace layout, every block 256-byte aligned
+  size_t off = 0;
+  auto put = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  c->off_status = put(256);
+  c->off_scores = put((size_t)d.B * d.F * d.N_s * 4);
+  c->off_quality = put((size_t)d.B * 3 * 4);
+  c->off_lse = put((size_t)d.B * d.N_h * d.H * 4);
+  c->off_sel = put((size_t)d.B * d.F * d.K * 4);
+  c->off_pack = put((size_t)d.B * d.Lp * 4);
+  c->off_inv = put((size_t)d.B * d.L * 4);
+  c->off_scratch = put(lse_scratch_bytes(d));
+  c->off_qp = put(packed_bytes(d));
+  c->off_kp = put(packed_bytes(d));
+  c->off_vp = put(packed_bytes(d));
+  c->off_op = put(packed_bytes(d));
+  c->ws_need = off;
+  c->io_need = 4 * align_up(full_bytes(d), 256);
+  *out_ctx = c;
+  return SWAM_OK;
+}
+
+int swam_destroy(swam_ctx* ctx) {
+  delete ctx;
+  return SWAM_OK;
+}
+
+int swam_workspace_bytes(const swam_ctx* ctx, size_t* bytes) {
+  if (!ctx || !bytes) return SWAM_ERR_INVALID_ARG;
+  *bytes = ctx->ws_need;
+  return SWAM_OK;
+}
+
+int swam_bind_workspace(swam_ctx* c, void* dev_ptr, size_t bytes) {
+  if (!c || !dev_ptr) return SWAM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(dev_ptr) & 255u) != 0) return fail(c, SWAM_ERR_INVALID_ARG, "workspace not 256-byte aligned");
+  if (bytes < c->ws_need) return fail(c, SWAM_ERR_WORKSPACE, "workspace too small");
+  if (int r = check_device(c)) return r;
+  cudaError_t e = select_prepare(c->d);
+  if (e != cudaSuccess) return fail_cuda(c, e, "select_prepare");
+  e = cudaMemset(dev_ptr, 0, 256);
+  if (e != cudaSuccess) return fail_cuda(c, e, "cudaMemset(status)");
+  c->ws = (unsigned char*)dev_ptr;
+  c->ws_bytes = bytes;
+  c->has_selection = false;
+  return SWAM_OK;
+}
+
+int swam_host_io_bytes(const swam_ctx* ctx, size_t* bytes) {
+  if (!ctx || !bytes) return SWAM_ERR_INVALID_ARG;
+  *bytes = ctx->io_need;
+  return SWAM_OK;
+}
+
+int swam_bind_host_io(swam_ctx* c, void* dev_ptr, size_t bytes) {
+  if (!c || !dev_ptr) return SWAM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(dev_ptr) & 255u) != 0) return fail(c, SWAM_ERR_INVALID_ARG, "staging not 256-byte aligned");
+  if (bytes < c->io_need) return fail(c, SWAM_ERR_WORKSPACE, "staging area too small");
+  c->io = (unsigned char*)dev_ptr;
+  return SWAM_OK;
+}
+
+int swam_score(swam_ctx* c, const void* q, const void* k, const float* lse_action, float* scores, float* quality,
+               void* stream) {
+  if (!c || !q || !k || !scores) return fail(c, SWAM_ERR_INVALID_ARG, "swam_score: null argument");
+  if (!aligned16(q) || !aligned16(k) || !aligned16(scores)) return fail(c, SWAM_ERR_INVALID_ARG, "swam_score: misaligned pointer");
+  cudaStream_t st = (cudaStream_t)stream;
+  const float* lse = lse_action;
+  if (!lse) {
+    if (int r = need_ws(c)) return r;
+    float* own = (float*)(c->ws + c->off_lse);
+    cudaError_t e = launch_action_lse(c->d, q, k, own, c->ws + c->off_scratch, st, &c->launches_i);
+    count(c);
+    if (e != cudaSuccess) return fail_cuda(c, e, "action lse launch");
+    lse = own;
+  }
+  cudaError_t e = launch_score(c->d, c->alpha, q, k, lse, scores, st, &c->launches_i);
+  count(c);
+  if (e != cudaSuccess) return fail_cuda(c, e, "score launch");
+  if (quality) {
+    e = launch_quality(c->d, scores, quality, st, &c->launches_i);
+    count(c);
+    if (e != cudaSuccess) return fail_cuda(c, e, "quality launch");
+  }
+  return SWAM_OK;
+}
+
+int swam_select(swam_ctx* c, const float* scores, int32_t* sel_idx, int32_t* pack_map, int32_t* inv_map, void* stream) {
+  if (!c || !scores) return fail(c, SWAM_ERR_INVALID_ARG, "swam_select: null argument");
+  if (int r = need_ws(c)) return r;
+  cudaError_t e = launch_select(c->d, scores, sel_idx, pack_map, inv_map, (int*)(c->ws + c->off_status),
+                                (cudaStream_t)stream, &c->launches_i);
+  count(c);
+  if (e != cudaSuccess) return fail_cuda(c, e, "select launch");
+  return SWAM_OK;
+}
+
+int swam_pack(swam_ctx* c, const void* q, const void* k, const void* v, const int32_t* pack_map, void* qp, void* kp,
+              void* vp, void* stream) {
+  if (!c || !pack_map) return fail(c, SWAM_ERR_INVALID_ARG, "swam_pack: null argument");
+  if ((!q) != (!qp) || (!k) != (!kp) || (!v) != (!vp)) return fail(c, SWAM_ERR_INVALID_ARG, "swam_pack: unpaired tensor");
+  const void* ptrs[6] = {q, k, v, qp, kp, vp};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return fail(c, SWAM_ERR_INVALID_ARG, "swam_pack: misaligned pointer");
+  if (int r = need_ws(c)) return r;
+  const void* src[3] = {q, k, v};
+  void* dst[3] = {qp, kp, vp};
+  cudaError_t e = launch_pack(c->d, src, dst, pack_map, (int*)(c->ws + c->off_status), (cudaStream_t)stream, &c->launches_i);
+  count(c);
+  if (e != cudaSuccess) return fail_cuda(c, e, "pack launch");
+  return SWAM_OK;
+}
+
+int swam_sparse_attn(swam_ctx* c, const void* qp, const void* kp, const void* vp, int32_t seq_len, void* out_p, float* lse,
+                     void* stream) {
+  if (!c || !qp || !kp || !vp || !out_p) return fail(c, SWAM_ERR_INVALID_ARG, "swam_sparse_attn: null argument");
+  if (seq_len <= 0 || seq_len > c->d.L) return fail(c, SWAM_ERR_INVALID_ARG, "swam_sparse_attn: seq_len out of range");
+  if (!aligned16(qp) || !aligned16(kp) || !aligned16(vp) || !aligned16(out_p))
+    return fail(c, SWAM_ERR_INVALID_ARG, "swam_sparse_attn: misaligned pointer");
+  return run_attention(c, qp, kp, vp, seq_len, out_p, lse, 0, seq_len, (cudaStream_t)stream);
+}
+
+int swam_scatter(swam_ctx* c, const void* out_p, const int32_t* pack_map, const int32_t* inv_map, const void* cached,
+                 void* out, void* stream) {
+  if (!c || !out_p || !pack_map || !out || !cached) return fail(c, SWAM_ERR_INVALID_ARG, "swam_scatter: null argument");
+  if (cached != out && !inv_map) return fail(c, SWAM_ERR_INVALID_ARG, "swam_scatter: inv_map needed when cached != out");
+  if (!aligned16(out_p) || !aligned16(cached) || !aligned16(out)) return fail(c, SWAM_ERR_INVALID_ARG, "swam_scatter: misaligned pointer");
+  if (int r = need_ws(c)) return r;
+  cudaError_t e = launch_scatter(c->d, out_p, pack_map, inv_map, cached, out, (int*)(c->ws + c->off_status),
+                                 (cudaStream_t)stream, &c->launches_i);
+  count(c);
+  if (e != cudaSuccess) return fail_cuda(c, e, "scatter launch");
+  return SWAM_OK;
+}
+
+int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t mode, void* out, void* stream) {
+  if (!c || !q || !k || !v || !out) return fail(c, SWAM_ERR_INVALID_ARG, "swam_step: null argument");
+  if (mode != SWAM_REUSE && mode != SWAM_REFRESH_FULL && mode != SWAM_REFRESH_LIGHT)
+    return fail(c, SWAM_ERR_INVALID_ARG, "swam_step: unknown mode");
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
+    return fail(c, SWAM_ERR_INVALID_ARG, "swam_step: misaligned pointer");
+  if (int r = need_ws(c)) return r;
+  if (mode == SWAM_REUSE && !c->has_selection)
+    return fail(c, SWAM_ERR_STATE, "swam_step: reuse requested before any refresh");
+  cudaStream_t st = (cudaStream_t)stream;
+  const Dims& d = c->d;
+  float* scores = (float*)(c->ws + c->off_scores);
+  float* quality = (float*)(c->ws + c->off_quality);
+  float* lse = (float*)(c->ws + c->off_lse);
+  int32_t* sel = (int32_t*)(c->ws + c->off_sel);
+  int32_t* pm = (int32_t*)(c->ws + c->off_pack);
+  int32_t* im = (int32_t*)(c->ws + c->off_inv);
+
+  if (mode == SWAM_REFRESH_FULL) {
+    // dense joint attention fills the cache and yields the action-row normalisers over all L keys
+    if (int r = run_attention(c, q, k, v, d.L, out, lse, d.L - d.H, d.H, st)) return r;
+  }
+  if (mode != SWAM_REUSE) {
+    const float* lse_in = (mode == SWAM_REFRESH_FULL) ? lse : nullptr;
+    if (int r = swam_score(c, q, k, lse_in, scores, quality, stream)) return r;
+    if (int r = swam_select(c, scores, sel, pm, im, stream)) return r;
+    c->has_selection = true;
+  }
+  if (mode != SWAM_REFRESH_FULL) {
+    void* qp = c->ws + c->off_qp;
+    void* kp = c->ws + c->off_kp;
+    void* vp = c->ws + c->off_vp;
+    void* op = c->ws + c->off_op;
+    if (int r = swam_pack(c, q, k, v, pm, qp, kp, vp, stream)) return r;
+    if (int r = run_attention(c, qp, kp, vp, d.Lp, op, nullptr, 0, 0, st)) return r;
+    if (int r = swam_scatter(c, op, pm, im, out, out, stream)) return r;
+  }
+  return SWAM_OK;
+}
+
+int swam_step_host(swam_ctx* c, const void* q_host, const void* k_host, const void* v_host, int32_t mode, void* out_host,
+                   void* stream) {
+  if (!c || !q_host || !k_host || !v_host || !out_host) return fail(c, SWAM_ERR_INVALID_ARG, "swam_step_host: null argument");
+  if (!c->io) return fail(c, SWAM_ERR_WORKSPACE, "swam_step_host: no staging area bound");
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t fb = full_bytes(c->d), stride = align_up(fb, 256);
+  void* dq = c->io;
+  void* dk = c->io + stride;
+  void* dv = c->io + 2 * stride;
+  void* dout = c->io + 3 * stride;
+  cudaError_t e = cudaMemcpyAsync(dq, q_host, fb, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dk, k_host, fb, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v_host, fb, cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return fail_cuda(c, e, "host to device copy");
+  if (int r = swam_step(c, dq, dk, dv, mode, dout, stream)) return r;
+  e = cudaMemcpyAsync(out_host, dout, fb, cudaMemcpyDeviceToHost, st);
+  if (e != cudaSuccess) return fail_cuda(c, e, "device to host copy");
+  return SWAM_OK;
+}
+
+int swam_get_selection(const swam_ctx* c, const int32_t** sel_idx, const int32_t** pack_map, const int32_t** inv_map) {
+  if (!c || !c->ws) return SWAM_ERR_WORKSPACE;
+  if (sel_idx) *sel_idx = (const int32_t*)(c->ws + c->off_sel);
+  if (pack_map) *pack_map = (const int32_t*)(c->ws + c->off_pack);
+  if (inv_map) *inv_map = (const int32_t*)(c->ws + c->off_inv);
+  return SWAM_OK;
+}
+
+int swam_get_scores(const swam_ctx* c, const float** scores, const float** lse_action, const float** quality) {
+  if (!c || !c->ws) return SWAM_ERR_WORKSPACE;
+  if (scores) *scores = (const float*)(c->ws + c->off_scores);
+  if (lse_action) *lse_action = (const float*)(c->ws + c->off_lse);
+  if (quality) *quality = (const float*)(c->ws + c->off_quality);
+  return SWAM_OK;
+}
+
+int swam_check(swam_ctx* c, void* stream) {
+  if (!c) return SWAM_ERR_INVALID_ARG;
+  if (int r = need_ws(c)) return r;
+  cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) return fail_cuda(c, e, "cudaStreamSynchronize");
+  int word = 0;
+  e = cudaMemcpy(&word, c->ws + c->off_status, sizeof(int), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return fail_cuda(c, e, "status read");
+  if (word != 0) {
+    e = cudaMemset(c->ws + c->off_status, 0, sizeof(int));
+    if (e != cudaSuccess) return fail_cuda(c, e, "status clear");
+    snprintf(c->err, sizeof(c->err), "device status word 0x%x%s%s%s", word, (word & ST_BAD_MAP) ? " [map entry out of range]" : "",
+             (word & ST_BAD_COUNT) ? " [selection count mismatch]" : "", (word & ST_TIMEOUT) ? " [bounded wait ran out]" : "");
+    return (word & ST_TIMEOUT) ? SWAM_ERR_TIMEOUT : SWAM_ERR_DEVICE_CHECK;
+  }
+  return SWAM_OK;
+}
+
+int swam_launch_count(const swam_ctx* c, int64_t* n) {
+  if (!c || !n) return SWAM_ERR_INVALID_ARG;
+  *n = c->launches;
+  return SWAM_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,64 @@
+// Internal declarations shared by the kernels and the C-ABI layer of libswam.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace swam {
+
+// bits of the device status word
+enum : int { ST_BAD_MAP = 1, ST_BAD_COUNT = 2, ST_TIMEOUT = 4 };
+
+constexpr int kMaxGroup = 32;  // largest frame-aligned query group the tensor-core scorer handles
+
+struct Dims {
+  int B, n_obs, F, N_s, H, N_h, D, Kc, Ks, K, L, Lp, g, dtype;
+  float scale, beta;
+};
+
+struct Alpha {
+  float w[kMaxGroup];
+};
+
+// ---- score.cu -------------------------------------------------------------
+// S[b,f,j] (Eq. 12) from the action rows of q, the future rows of k and lambda [B,N_h,H].
+cudaError_t launch_score(const Dims& d, const Alpha& alpha, const void* q, const void* k, const float* lse,
+                         float* scores, cudaStream_t st, int* launches);
+// (R, E, Q) of Eq. 9 per sample from stored scores.
+cudaError_t launch_quality(const Dims& d, const float* scores, float* quality, cudaStream_t st, int* launches);
+// lambda[b,h,i] = log sum over all L keys of exp(scale q_i.k_c); partial: scratch of lse_scratch_bytes().
+size_t lse_scratch_bytes(const Dims& d);
+cudaError_t launch_action_lse(const Dims& d, const void* q, const void* k, float* lse, void* scratch,
+                              cudaStream_t st, int* launches);
+
+// ---- select.cu ------------------------------------------------------------
+size_t select_smem_bytes(const Dims& d);
+cudaError_t select_prepare(const Dims& d);  // opt in to the dynamic shared memory the kernel needs
+cudaError_t launch_select(const Dims& d, const float* scores, int32_t* sel_idx, int32_t* pack_map,
+                          int32_t* inv_map, int* status, cudaStream_t st, int* launches);
+
+// ---- pack_scatter.cu ------------------------------------------------------
+// dst[b, p] = src[b, map[b,p]] for up to three tensor pairs (row_bytes per row).
+cudaError_t launch_pack(const Dims& d, const void* const src[3], void* const dst[3], const int32_t* pack_map,
+                        int* status, cudaStream_t st, int* launches);
+// in place: out[b, map[b,p]] = out_p[b,p];  blend: out[b,t] = inv[b,t] >= 0 ? out_p[b,inv[b,t]] : cached[b,t]
+cudaError_t launch_scatter(const Dims& d, const void* out_p, const int32_t* pack_map, const int32_t* inv_map,
+                           const void* cached, void* out, int* status, cudaStream_t st, int* launches);
+
+// ---- attn_*.cu ------------------------------------------------------------
+struct AttnArgs {
+  const void* q;
+  const void* k;
+  const void* v;
+  void* out;
+  float* lse;        // [B, N_h, lse_rows] or nullptr
+  int lse_row0;      // first query row whose normaliser is written
+  int lse_rows;      // number of rows written from lse_row0
+  int B, n, N_h, D;  // n = sequence length of this call
+  float scale;
+};
+cudaError_t attn_prepare(int D, int dtype);
+cudaError_t launch_attn_f32(const AttnArgs& a, cudaStream_t st, int* launches);
+cudaError_t launch_attn_bf16_mma(const AttnArgs& a, cudaStream_t st, int* launches);
+
+}  // namespace swam

@@ -1,0 +1,351 @@
+"""Parity of the CUDA path (through the C-ABI) against the CPU oracle, stage by stage and end to end.
+
+Bars: selected indices, pack maps and inverse maps bit-exact; packed/scattered tensors bit-exact; scores within
+1e-4 max-abs and 2e-5 relative; attention outputs within 1e-4 max-abs (fp32) or 2e-2 max-abs with relative
+L2 <= 1e-2 (bf16).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import reference as ora
+from paper_2609_38984_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+SCORE_REL = 2e-5
+
+
+def _swam():
+    from paper_2609_38984_b200 import swam
+    return swam
+
+
+def small(name="single_view", **kw):
+    base = dict(n_obs=70, grid_h=10, grid_w=9, n_heads=3, steps=3)
+    base.update(kw)
+    return W.WORKLOADS[name].with_(**base)
+
+
+def dev(x, wl):
+    return _swam().to_device(x, wl.dtype)
+
+
+def f64(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def check_float(got, want, dtype):
+    err = np.abs(got - want)
+    if dtype == W.F32:
+        assert err.max() <= 1e-4, err.max()
+    else:
+        assert err.max() <= 2e-2, err.max()
+        rel = np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-30)
+        assert rel <= 1e-2, rel
+
+
+# ------------------------------------------------------------------ select
+SELECT_SHAPES = [
+    # (B, F, N_s, K_c, K_s, n_obs, H)
+    (1, 2, 64, 14, 18, 16, 8),            # tiny
+    (3, 4, 90, 10, 13, 7, 32),            # ragged N_s
+    (2, 8, 360, 80, 104, 33, 32),         # the paper's 360-token frames with 80 + 104
+    (1, 2, 98, 19, 12, 5, 32),            # the paper's 98-token frames with 19 + 12
+    (1, 8, 1024, 133, 174, 1024, 64),     # larger-imagination shape
+    (8, 4, 1728, 188, 244, 1728, 32),     # multi-view shape
+    (1, 3, 50, 7, 0, 0, 3),               # no anchors, F not a power of two, no observed tokens
+    (1, 3, 50, 0, 9, 4, 3),               # no core tokens
+    (2, 5, 40, 15, 25, 4, 5),             # keep everything
+    (1, 1, 33, 4, 5, 2, 4),               # a single frame
+]
+
+
+@pytest.mark.parametrize("shape", SELECT_SHAPES)
+@pytest.mark.parametrize("ties", [False, True])
+def test_select_bit_exact(shape, ties):
+    swam = _swam()
+    B, F, N, kc, ks, n_obs, H = shape
+    s = W.random_scores(17 + N, B, F, N, ties=ties)
+    ctx = swam.Swam(B, n_obs, F, N, H, 2, 32, kc, ks, dtype=swam.F32, query_weights=[1.0 / (H // F)] * (H // F))
+    sel, pack, inv = ctx.select(torch.from_numpy(s).cuda())
+    ctx.check()
+    want = ora.select(s, kc, ks)
+    wp, wi = ora.maps(want["sel_idx"], n_obs, N, H)
+    assert np.array_equal(sel.cpu().numpy(), want["sel_idx"])
+    assert np.array_equal(pack.cpu().numpy(), wp)
+    assert np.array_equal(inv.cpu().numpy(), wi)
+
+
+def test_select_all_equal_and_zero_scores():
+    swam = _swam()
+    for val in (0.0, 0.25):
+        s = np.full((2, 4, 70), val, np.float32)
+        ctx = swam.Swam(2, 3, 4, 70, 8, 2, 32, 9, 11, dtype=swam.F32, query_weights=[0.5, 0.5])
+        sel, pack, inv = ctx.select(torch.from_numpy(s).cuda())
+        ctx.check()
+        want = ora.select(s, 9, 11)
+        assert np.array_equal(sel.cpu().numpy(), want["sel_idx"])
+        assert sel.cpu().numpy()[0, 0].tolist() == list(range(20))
+
+
+def test_select_is_deterministic():
+    swam = _swam()
+    s = torch.from_numpy(W.random_scores(3, 4, 8, 512, ties=True)).cuda()
+    ctx = swam.Swam(4, 10, 8, 512, 64, 2, 32, 60, 80, dtype=swam.F32)
+    first = [t.clone() for t in ctx.select(s)]
+    for _ in range(20):
+        again = ctx.select(s)
+        for a, b in zip(first, again):
+            assert torch.equal(a, b)
+
+
+# ------------------------------------------------------------------ score
+@pytest.mark.parametrize("wl", [
+    W.WORKLOADS["tiny"],
+    small(),                                              # bf16, D = 64, g = 8, ragged frame size
+    small("larger_imagination", n_obs=40, grid_h=7, grid_w=9, n_heads=5),   # bf16, D = 128
+    small(n_frames=2, n_action=32, head_dim=32),          # g = 16 (two query tiles), D = 32
+    small(n_frames=8, n_action=32),                       # g = 4 (padded query tile)
+], ids=["tiny_f32", "d64", "d128", "g16_d32", "g4"])
+@pytest.mark.parametrize("given_lse", [True, False])
+def test_score_matches_oracle(wl, given_lse):
+    swam = _swam()
+    x = W.generate_steps(wl, 1)[0]
+    ctx = swam.Swam.from_workload(wl)
+    q, k = dev(x["q"], wl), dev(x["k"], wl)
+    lse64 = ora.action_lse(x["q"], x["k"], wl.n_action)
+    lse_t = torch.from_numpy(lse64.astype(np.float32)).cuda() if given_lse else None
+    s, qual = ctx.score(q, k, lse_t, quality=True)
+    ctx.check()
+    want = ora.score(x["q"], x["k"], wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, lse=lse64)
+    got = s.cpu().numpy().astype(np.float64)
+    assert np.abs(got - want).max() <= 1e-4
+    rel = np.abs(got - want) / np.maximum(want, 1e-30)
+    assert rel.max() <= SCORE_REL, rel.max()
+    wq = ora.quality(want.astype(np.float32))
+    assert np.allclose(qual.cpu().numpy(), wq, rtol=1e-4, atol=1e-6)
+    if not given_lse:
+        _, lse_dev, _ = ctx.cached_scores()
+        assert np.abs(lse_dev.cpu().numpy() - lse64).max() <= 1e-4
+
+
+def test_score_custom_weights():
+    swam = _swam()
+    wl = small(n_frames=4, n_action=12)                   # g = 3: only valid with explicit weights
+    x = W.generate_steps(wl, 1)[0]
+    alpha = [0.2, 0.5, 0.3]
+    kc, ks = wl.budgets
+    with pytest.raises(swam.SwamError):
+        swam.Swam.from_workload(wl)
+    ctx = swam.Swam(wl.batch, wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, wl.n_heads, wl.head_dim, kc, ks,
+                    dtype=wl.dtype, query_weights=alpha)
+    s = ctx.score(dev(x["q"], wl), dev(x["k"], wl))
+    want = ora.score(x["q"], x["k"], wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, alpha=np.array(alpha))
+    rel = np.abs(s.cpu().numpy() - want) / want
+    assert rel.max() <= SCORE_REL
+
+
+# ------------------------------------------------------------------ pack / scatter
+@pytest.mark.parametrize("wl", [W.WORKLOADS["tiny"], small(batch=2)], ids=["f32", "bf16"])
+def test_pack_and_scatter_exact(wl):
+    swam = _swam()
+    x = W.generate_steps(wl, 1)[0]
+    ctx = swam.Swam.from_workload(wl)
+    kc, ks = wl.budgets
+    sc = W.random_scores(5, wl.batch, wl.n_frames, wl.n_spatial)
+    sel = ora.select(sc, kc, ks)["sel_idx"]
+    pm, im = ora.maps(sel, wl.n_obs, wl.n_spatial, wl.n_action)
+    pm_t, im_t = torch.from_numpy(pm).cuda(), torch.from_numpy(im).cuda()
+    q, k, v = (dev(x[n], wl) for n in "qkv")
+    qp, kp, vp = ctx.pack(q, k, v, pm_t)
+    for src, got in ((x["q"], qp), (x["k"], kp), (x["v"], vp)):
+        assert np.array_equal(got.float().cpu().numpy(), ora.pack(src, pm))
+    only_k = ctx.pack(None, k, None, pm_t)
+    assert only_k[0] is None and torch.equal(only_k[1], kp)
+    # in place: retained rows replaced, omitted rows untouched
+    cached = dev(x["v"], wl)
+    before = cached.clone()
+    ctx.scatter(qp, pm_t, im_t, cached)
+    want = ora.scatter(ora.pack(x["q"], pm), pm, x["v"])
+    assert np.array_equal(cached.float().cpu().numpy(), want)
+    # blend into a fresh buffer
+    out = torch.zeros_like(before)
+    ctx.scatter(qp, pm_t, im_t, before, out)
+    assert np.array_equal(out.float().cpu().numpy(), want)
+    ctx.check()
+
+
+def test_corrupt_map_is_reported_not_followed():
+    swam = _swam()
+    wl = small()
+    ctx = swam.Swam.from_workload(wl)
+    x = W.generate_steps(wl, 1)[0]
+    pm = torch.arange(wl.packed_len, dtype=torch.int32).repeat(wl.batch, 1).cuda()
+    pm[0, 5] = wl.seq_len + 3
+    pm[0, 6] = -2
+    q = dev(x["q"], wl)
+    qp = ctx.pack(q, None, None, pm)[0]
+    with pytest.raises(swam.SwamError) as e:
+        ctx.check()
+    assert e.value.code == swam.ERR_DEVICE_CHECK
+    ctx.check()     # the status word was cleared
+    assert torch.equal(qp[0, 7], q[0, 7])
+
+
+# ------------------------------------------------------------------ attention
+ATTN_CASES = [
+    ("tiny", dict()),
+    ("tiny", dict(n_obs=3, head_dim=64)),
+    ("single_view", dict(n_obs=70, grid_h=10, grid_w=9, n_heads=3)),                 # D = 64, L = 462
+    ("single_view", dict(n_obs=1, grid_h=4, grid_w=4, n_heads=2, n_action=16, head_dim=32)),
+    ("larger_imagination", dict(n_obs=40, grid_h=7, grid_w=9, n_heads=2, batch=2)),    # D = 128, L = 608
+    ("larger_imagination", dict(n_obs=0, grid_h=2, grid_w=2, n_heads=1, n_action=32)),  # L = 64: one tile
+    ("larger_imagination", dict(n_obs=1, grid_h=2, grid_w=2, n_heads=1, n_action=32)),  # L = 65
+]
+
+
+@pytest.mark.parametrize("name,kw", ATTN_CASES)
+def test_attention_matches_oracle(name, kw):
+    swam = _swam()
+    wl = W.WORKLOADS[name].with_(**kw)
+    x = W.generate_steps(wl, 1)[0]
+    ctx = swam.Swam.from_workload(wl)
+    q, k, v = (dev(x[n], wl) for n in "qkv")
+    out, lse = ctx.sparse_attn(q, k, v, want_lse=True)
+    ctx.check()
+    want, wlse = ora.attention(x["q"], x["k"], x["v"])
+    check_float(f64(out), want, wl.dtype)
+    assert np.abs(lse.cpu().numpy() - wlse).max() <= (1e-4 if wl.dtype == W.F32 else 2e-3)
+
+
+def test_attention_short_sequences():
+    """seq_len below the full length, down to one token."""
+    swam = _swam()
+    wl = small()
+    x = W.generate_steps(wl, 1)[0]
+    ctx = swam.Swam.from_workload(wl)
+    for n in (1, 2, 63, 64, 65, 127, 129, 200):
+        q, k, v = (dev(np.ascontiguousarray(x[m][:, :n]), wl) for m in "qkv")
+        out = ctx.sparse_attn(q, k, v)
+        want, _ = ora.attention(x["q"][:, :n], x["k"][:, :n], x["v"][:, :n])
+        check_float(f64(out), want, wl.dtype)
+
+
+# ------------------------------------------------------------------ whole steps
+def run_schedule(ctx, wl, steps, refresh):
+    swam = _swam()
+    out = ctx.empty_full().zero_()
+    log = []
+    for t, x in enumerate(steps):
+        mode = swam.REFRESH_FULL if t % refresh == 0 else swam.REUSE
+        ctx.step(dev(x["q"], wl), dev(x["k"], wl), dev(x["v"], wl), mode, out)
+        ctx.check()
+        sel, pm, im = ctx.selection()
+        sc, _, _ = ctx.cached_scores()
+        log.append(dict(out=f64(out), sel=sel.cpu().numpy().copy(), pm=pm.cpu().numpy().copy(),
+                        im=im.cpu().numpy().copy(), scores=sc.cpu().numpy().copy()))
+    return log
+
+
+def compare_schedule(wl, steps, refresh, log):
+    """Oracle run that follows the paper's step loop; index equality is required unless a TopK cut is closer
+    than the score error can resolve, in which case the case is reported by the assertion message."""
+    kc, ks = wl.budgets
+    want = ora.run_steps(steps, refresh, wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, kc, ks)
+    for t, (g, w) in enumerate(zip(log, want)):
+        rel = np.abs(g["scores"] - w["scores"].astype(np.float64)) / np.maximum(w["scores"], 1e-30)
+        assert rel.max() <= SCORE_REL, (t, rel.max())
+        # stage-isolated exactness: the GPU selection equals the oracle's selection of the GPU's own scores
+        iso = ora.select(g["scores"], kc, ks)
+        ipm, iim = ora.maps(iso["sel_idx"], wl.n_obs, wl.n_spatial, wl.n_action)
+        assert np.array_equal(g["sel"], iso["sel_idx"]) and np.array_equal(g["pm"], ipm) and np.array_equal(g["im"], iim)
+        # end to end
+        assert np.array_equal(g["sel"], w["sel_idx"]), (t, "cut margins", w["margins"], "score rel err", rel.max())
+        assert np.array_equal(g["pm"], w["pack_map"]) and np.array_equal(g["im"], w["inv_map"])
+        check_float(g["out"], w["out"], wl.dtype)
+
+
+def test_tiny_schedule_matches_oracle():
+    swam = _swam()
+    wl = W.WORKLOADS["tiny"]
+    steps = W.generate_steps(wl)
+    ctx = swam.Swam.from_workload(wl)
+    compare_schedule(wl, steps, wl.refresh, run_schedule(ctx, wl, steps, wl.refresh))
+
+
+@pytest.mark.parametrize("wl", [
+    small(batch=2),
+    small("larger_imagination", n_obs=40, grid_h=7, grid_w=9, n_heads=2, steps=3),
+    small("multi_view", batch=2, n_obs=33, grid_h=5, grid_w=4, n_heads=2, steps=4),
+], ids=["d64", "d128", "multiview"])
+def test_bf16_schedule_matches_oracle(wl):
+    swam = _swam()
+    steps = W.generate_steps(wl)
+    ctx = swam.Swam.from_workload(wl)
+    compare_schedule(wl, steps, wl.refresh, run_schedule(ctx, wl, steps, wl.refresh))
+
+
+def test_refresh_every_step_and_keep_all():
+    swam = _swam()
+    wl = small(steps=2)
+    steps = W.generate_steps(wl)
+    ctx = swam.Swam.from_workload(wl)
+    log = run_schedule(ctx, wl, steps, 1)
+    compare_schedule(wl, steps, 1, log)
+    # keep ratio 1.0: the sparse step runs over the identity map and reproduces dense attention
+    wl1 = wl.with_(keep=1.0)
+    ctx1 = swam.Swam.from_workload(wl1)
+    log1 = run_schedule(ctx1, wl1, steps, 2)
+    assert np.array_equal(log1[1]["pm"][0], np.arange(wl1.seq_len))
+    dense, _ = ora.attention(steps[1]["q"], steps[1]["k"], steps[1]["v"])
+    check_float(log1[1]["out"], dense, wl1.dtype)
+
+
+def test_light_refresh_step():
+    """score (normalisers computed on the device) -> select -> pack -> attention -> scatter in one call."""
+    swam = _swam()
+    wl = small()
+    steps = W.generate_steps(wl, 2)
+    ctx = swam.Swam.from_workload(wl)
+    kc, ks = wl.budgets
+    out = ctx.empty_full()
+    x0, x1 = steps
+    ctx.step(dev(x0["q"], wl), dev(x0["k"], wl), dev(x0["v"], wl), swam.REFRESH_FULL, out)
+    ctx.step(dev(x1["q"], wl), dev(x1["k"], wl), dev(x1["v"], wl), swam.REFRESH_LIGHT, out)
+    ctx.check()
+    st = ora.full_step(ora.StepState(), x0["q"], x0["k"], x0["v"], wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, kc, ks)
+    s1 = ora.score(x1["q"], x1["k"], wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action).astype(np.float32)
+    st.scores = s1
+    st.sel = ora.select(s1, kc, ks)
+    st.pack_map, st.inv_map = ora.maps(st.sel["sel_idx"], wl.n_obs, wl.n_spatial, wl.n_action)
+    ora.sparse_step(st, x1["q"], x1["k"], x1["v"])
+    sel, pm, _ = ctx.selection()
+    assert np.array_equal(sel.cpu().numpy(), st.sel["sel_idx"]), st.sel["margins"]
+    check_float(f64(out), st.out, wl.dtype)
+
+
+def test_reuse_before_refresh_is_a_state_error():
+    swam = _swam()
+    wl = W.WORKLOADS["tiny"]
+    ctx = swam.Swam.from_workload(wl)
+    t = ctx.empty_full().zero_()
+    with pytest.raises(swam.SwamError) as e:
+        ctx.step(t, t, t, swam.REUSE, ctx.empty_full())
+    assert e.value.code == swam.ERR_STATE
+
+
+def test_host_buffer_step_matches_device_step():
+    swam = _swam()
+    wl = small()
+    steps = W.generate_steps(wl, 2)
+    ctx_a, ctx_b = swam.Swam.from_workload(wl), swam.Swam.from_workload(wl)
+    out_dev = ctx_a.empty_full()
+    out_host = torch.empty(out_dev.shape, dtype=out_dev.dtype).pin_memory()
+    for t, x in enumerate(steps):
+        mode = swam.REFRESH_FULL if t == 0 else swam.REUSE
+        hq, hk, hv = (torch.from_numpy(x[n]).to(out_dev.dtype).pin_memory() for n in "qkv")
+        ctx_a.step(hq.cuda(), hk.cuda(), hv.cuda(), mode, out_dev)
+        ctx_b.step_host(hq, hk, hv, mode, out_host)
+        ctx_b.check()
+        assert torch.equal(out_dev.cpu(), out_host)
