@@ -131,6 +131,13 @@ int swam_get_scores(const swam_ctx* ctx, const float** scores, const float** lse
  * SWAM_ERR_TIMEOUT or SWAM_ERR_CUDA. */
 int swam_check(swam_ctx* ctx, void* stream);
 
+/* Options.  SWAM_OPT_ATTN_VARIANT selects the bf16 attention kernel: SWAM_ATTN_AUTO (default) runs the
+ * tcgen05/TMEM kernel for head_dim 64 and 128 and the warp-level mma.sync kernel for head_dim 32;
+ * SWAM_ATTN_WARP_MMA forces the mma.sync kernel (an independent on-device second opinion used by the tests). */
+enum { SWAM_OPT_ATTN_VARIANT = 1 };
+enum { SWAM_ATTN_AUTO = 0, SWAM_ATTN_WARP_MMA = 1 };
+int swam_set_option(swam_ctx* ctx, int32_t option, int32_t value);
+
 /* Number of kernels this context has launched so far (host-side counter). */
 int swam_launch_count(const swam_ctx* ctx, int64_t* count);
 

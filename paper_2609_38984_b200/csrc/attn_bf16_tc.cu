@@ -1,0 +1,474 @@
+// Joint softmax attention for bf16 tensors on the 5th-generation tensor cores (tcgen05 + TMEM), fed by TMA.
+//
+// One CTA owns two 128-row query tiles of one (sample, head) and walks over the keys in tiles of 128:
+//   warp 9      TMA producer: Q once, then K_j / V_j into a ring of shared-memory stages (128B-swizzled boxes)
+//   warp 8      one elected thread issues every tcgen05.mma: S_s = Q_s K_j^T (both operands K-major in shared
+//               memory) into TMEM, then O_s += P_s V_j with P_s read from TMEM and V_j as an MN-major operand
+//   warps 0-3   softmax of query tile 0: one thread per row reads its S row from TMEM, keeps the running max and
+//   warps 4-7   sum (exp2 domain), writes P as bf16 back over S; same for query tile 1
+// The two query tiles alternate on the tensor pipe, so one tile's exponentials overlap the other tile's MMAs.
+// O stays in TMEM for the whole key loop; it is rescaled only when a row's maximum has grown by more than 2^8
+// since the value its exponentials refer to (the result is exact either way: sums and outputs share the same
+// reference maximum).  Every wait on an mbarrier is bounded; when a wait runs out the kernel raises the timeout
+// bit of the status word, stops issuing work, and every role falls through to the common exit.
+#include <cuda.h>
+
+#include "swam_internal.cuh"
+
+namespace swam {
+namespace {
+
+constexpr int kTile = 128;          // query rows per tile and keys per tile
+constexpr int kThreadsTc = 320;     // 8 softmax warps + MMA warp + TMA warp
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kRescaleThreshold = 8.0f;
+constexpr unsigned long long kWaitCycles = 4000000000ull;  // about two seconds at 1.9 GHz
+
+// ---------------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// bounded wait: false when the limit ran out or another role already gave up
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = clock64();
+  while (true) {
+    if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if ((unsigned long long)(clock64() - t0) > kWaitCycles) { *abort_flag = 1; return false; }
+  }
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit_wait() {
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accum) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accum) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, tile rows of 128 bytes, 8-row groups 1024 bytes apart.
+// lbo: byte distance between 64-element blocks along the MN dimension (MN-major operands only).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;  // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;  // SWIZZLE_128B
+  return d;
+}
+
+struct TcParams {
+  float* lse;
+  int* status;
+  int lse_row0, lse_rows;
+  int n, N_h;
+  float scale_log2;
+};
+
+template <int D>
+struct TcCfg {
+  static constexpr int DB = D / 64;                 // 64-column (128-byte) blocks per row
+  static constexpr int kSubTile = kTile * 128;      // bytes of one [128 rows x 64 cols] block
+  static constexpr int kTileBytes = DB * kSubTile;  // one 128 x D tile
+  static constexpr int kStages = (D == 128) ? 2 : 4;
+  static constexpr int kSmemData = 2 * kTileBytes + 2 * kStages * kTileBytes;
+  static constexpr int kSmemBytes = kSmemData + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
+  static constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(D >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
+};
+
+template <int D>
+__global__ void __launch_bounds__(kThreadsTc, 1)
+attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                    const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o, const TcParams p) {
+  using C = TcCfg<D>;
+  constexpr int ST = C::kStages;
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = (smem_addr(smem_raw) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_raw + (base - smem_addr(smem_raw));
+  const uint32_t sQ = base;                                 // [2][tile]
+  const uint32_t sK = sQ + 2 * C::kTileBytes;               // [ST][tile]
+  const uint32_t sV = sK + ST * C::kTileBytes;              // [ST][tile]
+  const uint32_t bars = sV + ST * C::kTileBytes;
+  // barrier slots (8 bytes each)
+  const uint32_t bar_q = bars;
+  auto bar_k_full = [&](int s) { return bars + 8 * (1 + s); };
+  auto bar_k_empty = [&](int s) { return bars + 8 * (1 + ST + s); };
+  auto bar_v_full = [&](int s) { return bars + 8 * (1 + 2 * ST + s); };
+  auto bar_v_empty = [&](int s) { return bars + 8 * (1 + 3 * ST + s); };
+  auto bar_s_full = [&](int s) { return bars + 8 * (1 + 4 * ST + s); };
+  auto bar_p_full = [&](int s) { return bars + 8 * (3 + 4 * ST + s); };
+  const uint32_t bar_o_final = bars + 8 * (5 + 4 * ST);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + C::kSmemData + 8 * (6 + 4 * ST));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::kSmemData + 8 * (6 + 4 * ST) + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int row0 = blockIdx.x * 2 * kTile;
+  const int n_tiles = (p.n + kTile - 1) / kTile;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_q, 1);
+    for (int s = 0; s < ST; ++s) {
+      mbar_init(bar_k_full(s), 1);
+      mbar_init(bar_k_empty(s), 1);
+      mbar_init(bar_v_full(s), 1);
+      mbar_init(bar_v_empty(s), 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar_s_full(s), 1);
+      mbar_init(bar_p_full(s), kTile);
+    }
+    mbar_init(bar_o_final, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_addr(tmem_slot)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+D) O1 [256+D, 256+2D); P_s overlays the first 64 columns of S_s
+  auto tm_S = [&](int s) { return tmem + (uint32_t)(s * kTile); };
+  auto tm_O = [&](int s) { return tmem + (uint32_t)(2 * kTile + s * D); };
+
+  if (warp == 9) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      bool ok = true;
+      mbar_expect_tx(bar_q, 2 * C::kTileBytes);
+      for (int s = 0; s < 2; ++s)
+        for (int db = 0; db < C::DB; ++db)
+          tma_load_4d(sQ + s * C::kTileBytes + db * C::kSubTile, &map_q, bar_q, db * 64, row0 + s * kTile, h, b);
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int st = j % ST;
+        const uint32_t par = ((j / ST) & 1) ^ 1;  // first pass over the ring: slots start empty
+        ok = mbar_wait(bar_k_empty(st), par, abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(bar_k_full(st), C::kTileBytes);
+        for (int db = 0; db < C::DB; ++db)
+          tma_load_4d(sK + st * C::kTileBytes + db * C::kSubTile, &map_k, bar_k_full(st), db * 64, j * kTile, h, b);
+        ok = mbar_wait(bar_v_empty(st), par, abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(bar_v_full(st), C::kTileBytes);
+        for (int db = 0; db < C::DB; ++db)
+          tma_load_4d(sV + st * C::kTileBytes + db * C::kSubTile, &map_v, bar_v_full(st), db * 64, j * kTile, h, b);
+      }
+    }
+  } else if (warp == 8) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      bool ok = mbar_wait(bar_q, 0, abort_flag);
+      auto issue_qk = [&](int s, int st) {
+        // S_s = Q_s K^T : K dimension = D, 16 elements (32 bytes) per instruction inside the 128-byte swizzle row
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint32_t off = (ks >> 2) * C::kSubTile + (ks & 3) * 32;
+          mma_ss(tm_S(s), smem_desc(sQ + s * C::kTileBytes + off, 16, 1024), smem_desc(sK + st * C::kTileBytes + off, 16, 1024),
+                 C::kIdescQK, ks > 0);
+        }
+      };
+      auto issue_pv = [&](int s, int st, bool accum) {
+        // O_s += P_s V : K dimension = 128 keys, 16 keys (two 8-row groups) per instruction; V is MN-major
+#pragma unroll
+        for (int kk = 0; kk < kTile / 16; ++kk) {
+          mma_ts(tm_O(s), tm_S(s) + kk * 8, smem_desc(sV + st * C::kTileBytes + kk * 2048, C::kSubTile, 1024), C::kIdescPV,
+                 (accum || kk > 0) ? 1u : 0u);
+        }
+      };
+      if (ok) ok = mbar_wait(bar_k_full(0), 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+        issue_qk(0, 0);
+        tc_commit(bar_s_full(0));
+        issue_qk(1, 0);
+        tc_commit(bar_s_full(1));
+        tc_commit(bar_k_empty(0));
+      }
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int st = j % ST, st_next = (j + 1) % ST;
+        const uint32_t par_full = (j / ST) & 1, par_next = ((j + 1) / ST) & 1;
+        ok = mbar_wait(bar_v_full(st), par_full, abort_flag);
+        for (int s = 0; s < 2 && ok; ++s) {
+          ok = mbar_wait(bar_p_full(s), j & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          issue_pv(s, st, j > 0);
+          if (j + 1 < n_tiles) {
+            if (s == 0) ok = mbar_wait(bar_k_full(st_next), par_next, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            issue_qk(s, st_next);
+            tc_commit(bar_s_full(s));
+          }
+        }
+        if (!ok) break;
+        tc_commit(bar_v_empty(st));
+        if (j + 1 < n_tiles) tc_commit(bar_k_empty(st_next));
+      }
+      if (ok) tc_commit(bar_o_final);
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax warps: one thread per query row
+    const int s = warp >> 2;                 // query tile of this warpgroup
+    const int r = (warp & 3) * 32 + lane;    // row inside the tile == TMEM lane
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS = tm_S(s) + lane_off, tO = tm_O(s) + lane_off;
+    float m_used = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_tiles; ++j) {
+      ok = mbar_wait(bar_s_full(s), j & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      float sv[kTile];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<float(*)[32]>(&sv[c * 32]));
+      tmem_ld_wait();
+      const int valid = p.n - j * kTile;  // keys of this tile inside the sequence
+      if (valid < kTile) {
+#pragma unroll
+        for (int c = 0; c < kTile; ++c)
+          if (c >= valid) sv[c] = -INFINITY;
+      }
+      float mx = sv[0];
+#pragma unroll
+      for (int c = 1; c < kTile; ++c) mx = fmaxf(mx, sv[c]);
+      mx *= p.scale_log2;
+      // lazy rescale: only when some row of this warp outgrew its reference maximum by more than the threshold
+      const bool grow = mx > m_used + kRescaleThreshold;
+      if (j == 0) {
+        m_used = mx;
+      } else if (__any_sync(0xffffffffu, grow)) {
+        const float m_new = fmaxf(m_used, mx);
+        const float f = ex2(m_used - m_new);
+        l_run *= f;
+        m_used = m_new;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          float ov[32];
+          tmem_ld32(tO + c * 32, ov);
+          tmem_ld_wait();
+          uint32_t ou[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) ou[i] = __float_as_uint(ov[i] * f);
+          tmem_st32(tO + c * 32, ou);
+        }
+        tmem_st_wait();
+      }
+      float sum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const float p0 = ex2(fmaf(sv[c * 32 + 2 * i], p.scale_log2, -m_used));
+          const float p1 = ex2(fmaf(sv[c * 32 + 2 * i + 1], p.scale_log2, -m_used));
+          sum += p0 + p1;
+          pk[i] = pack_bf16x2(p0, p1);
+        }
+        tmem_st16(tS + c * 16, pk);
+      }
+      l_run += sum;
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(bar_p_full(s));
+    }
+    // epilogue: O / l -> bf16 -> swizzled staging in the (finished) Q tile -> TMA store; rows beyond n are clipped
+    if (ok) ok = mbar_wait(bar_o_final, 0, abort_flag);
+    if (ok) {
+      tc_fence_after();
+      const float inv = 1.f / l_run;
+      unsigned char* stage = base_ptr + s * C::kTileBytes;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        float ov[32];
+        tmem_ld32(tO + c * 32, ov);
+        tmem_ld_wait();
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          uint4 w;
+          w.x = pack_bf16x2(ov[q4 * 8 + 0] * inv, ov[q4 * 8 + 1] * inv);
+          w.y = pack_bf16x2(ov[q4 * 8 + 2] * inv, ov[q4 * 8 + 3] * inv);
+          w.z = pack_bf16x2(ov[q4 * 8 + 4] * inv, ov[q4 * 8 + 5] * inv);
+          w.w = pack_bf16x2(ov[q4 * 8 + 6] * inv, ov[q4 * 8 + 7] * inv);
+          const int col = c * 32 + q4 * 8;          // first of 8 output columns
+          const int db = col >> 6, chunk = (col & 63) >> 3;
+          *reinterpret_cast<uint4*>(stage + db * C::kSubTile + r * 128 + ((chunk ^ (r & 7)) << 4)) = w;
+        }
+      }
+      const int row = row0 + s * kTile + r;
+      if (p.lse && row < p.n && row >= p.lse_row0 && row < p.lse_row0 + p.lse_rows)
+        p.lse[((int64_t)b * p.N_h + h) * p.lse_rows + (row - p.lse_row0)] = (m_used + log2f(l_run)) * 0.6931471805599453f;
+      fence_proxy_async();
+    }
+    asm volatile("bar.sync %0, 128;" ::"r"(1 + s) : "memory");  // the four warps of this query tile
+    if (ok && (warp & 3) == 0 && lane == 0 && row0 + s * kTile < p.n) {
+      for (int db = 0; db < C::DB; ++db)
+        tma_store_4d(&map_o, sQ + s * C::kTileBytes + db * C::kSubTile, db * 64, row0 + s * kTile, h, b);
+      tma_store_commit_wait();
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, ST_TIMEOUT);
+  if (warp == 8) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)ptr;
+  }
+  return fn;
+}
+
+// [B, n, N_h, D] bf16 viewed as a 4-D tensor (d, row, head, sample); box = 64 columns x 128 rows, 128-byte swizzle
+bool make_map(CUtensorMap* map, const void* ptr, int B, int n, int N_h, int D) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)n, (cuuint64_t)N_h, (cuuint64_t)B};
+  const cuuint64_t strides[3] = {(cuuint64_t)N_h * D * 2, (cuuint64_t)D * 2, (cuuint64_t)n * N_h * D * 2};
+  const cuuint32_t box[4] = {64, (cuuint32_t)kTile, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D>
+cudaError_t launch_tc_d(const AttnArgs& a, int* status, cudaStream_t st) {
+  CUtensorMap mq, mk, mv, mo;
+  if (!make_map(&mq, a.q, a.B, a.n, a.N_h, D) || !make_map(&mk, a.k, a.B, a.n, a.N_h, D) ||
+      !make_map(&mv, a.v, a.B, a.n, a.N_h, D) || !make_map(&mo, a.out, a.B, a.n, a.N_h, D))
+    return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(attn_bf16_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<D>::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  TcParams p{a.lse, status, a.lse_row0, a.lse_rows, a.n, a.N_h, a.scale * kLog2e};
+  dim3 grid((a.n + 2 * kTile - 1) / (2 * kTile), a.N_h, a.B);
+  attn_bf16_tc_kernel<D><<<grid, kThreadsTc, TcCfg<D>::kSmemBytes, st>>>(mq, mk, mv, mo, p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, cudaStream_t st, int* launches) {
+  ++*launches;
+  switch (a.D) {
+    case 64: return launch_tc_d<64>(a, status, st);
+    case 128: return launch_tc_d<128>(a, status, st);
+    default: return cudaErrorInvalidConfiguration;
+  }
+}
+
+}  // namespace swam

@@ -20,6 +20,7 @@ struct swam_ctx {
   size_t off_status, off_scores, off_quality, off_lse, off_sel, off_pack, off_inv, off_scratch, off_qp, off_kp,
       off_vp, off_op, ws_need;
   bool has_selection;
+  int attn_variant;  // SWAM_ATTN_AUTO | SWAM_ATTN_WARP_MMA
   // host-io staging (device)
   unsigned char* io;
   size_t io_need;
@@ -54,8 +55,15 @@ void count(swam_ctx* c) {
 int run_attention(swam_ctx* c, const void* q, const void* k, const void* v, int n, void* out, float* lse, int lse_row0,
                   int lse_rows, cudaStream_t st) {
   AttnArgs a{q, k, v, out, lse, lse_row0, lse_rows, c->d.B, n, c->d.N_h, c->d.D, c->d.scale};
-  cudaError_t e = (c->d.dtype == SWAM_F32) ? launch_attn_f32(a, st, &c->launches_i)
-                                           : launch_attn_bf16_mma(a, st, &c->launches_i);
+  cudaError_t e;
+  if (c->d.dtype == SWAM_F32) {
+    e = launch_attn_f32(a, st, &c->launches_i);
+  } else if (c->d.D >= 64 && c->attn_variant == SWAM_ATTN_AUTO) {
+    if (!c->ws) return fail(c, SWAM_ERR_WORKSPACE, "no workspace bound");
+    e = launch_attn_bf16_tc(a, (int*)(c->ws + c->off_status), st, &c->launches_i);
+  } else {
+    e = launch_attn_bf16_mma(a, st, &c->launches_i);
+  }
   count(c);
   if (e != cudaSuccess) return fail_cuda(c, e, "attention launch");
   return SWAM_OK;
@@ -350,6 +358,15 @@ int swam_check(swam_ctx* c, void* stream) {
     return (word & ST_TIMEOUT) ? SWAM_ERR_TIMEOUT : SWAM_ERR_DEVICE_CHECK;
   }
   return SWAM_OK;
+}
+
+int swam_set_option(swam_ctx* c, int32_t option, int32_t value) {
+  if (!c) return SWAM_ERR_INVALID_ARG;
+  if (option == SWAM_OPT_ATTN_VARIANT && (value == SWAM_ATTN_AUTO || value == SWAM_ATTN_WARP_MMA)) {
+    c->attn_variant = value;
+    return SWAM_OK;
+  }
+  return fail(c, SWAM_ERR_INVALID_ARG, "swam_set_option: unknown option or value");
 }
 
 int swam_launch_count(const swam_ctx* c, int64_t* n) {

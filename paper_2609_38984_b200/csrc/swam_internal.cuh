@@ -60,5 +60,7 @@ struct AttnArgs {
 cudaError_t attn_prepare(int D, int dtype);
 cudaError_t launch_attn_f32(const AttnArgs& a, cudaStream_t st, int* launches);
 cudaError_t launch_attn_bf16_mma(const AttnArgs& a, cudaStream_t st, int* launches);
+// tcgen05 / TMEM / TMA kernel, head_dim 64 or 128; bounded waits report through the status word
+cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, cudaStream_t st, int* launches);
 
 }  // namespace swam

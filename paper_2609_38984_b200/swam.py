@@ -20,11 +20,13 @@ LIB_PATH = os.path.join(_HERE, "libswam.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_STATE, ERR_CUDA, ERR_DEVICE_CHECK, ERR_TIMEOUT = range(8)
 F32, BF16 = 0, 1
 REUSE, REFRESH_FULL, REFRESH_LIGHT = 0, 1, 2
+OPT_ATTN_VARIANT = 1
+ATTN_AUTO, ATTN_WARP_MMA = 0, 1
 
 EXPORTS = [
     "swam_create", "swam_destroy", "swam_workspace_bytes", "swam_bind_workspace", "swam_score", "swam_select",
     "swam_pack", "swam_sparse_attn", "swam_scatter", "swam_step", "swam_host_io_bytes", "swam_bind_host_io",
-    "swam_step_host", "swam_get_selection", "swam_get_scores", "swam_check", "swam_launch_count",
+    "swam_step_host", "swam_get_selection", "swam_get_scores", "swam_check", "swam_set_option", "swam_launch_count",
     "swam_last_error", "swam_version",
 ]
 
@@ -73,6 +75,7 @@ def load_library() -> ctypes.CDLL:
         lib.swam_get_selection.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
         lib.swam_get_scores.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
         lib.swam_check.argtypes = [vp, vp]
+        lib.swam_set_option.argtypes = [vp, i32, i32]
         lib.swam_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
         lib.swam_last_error.argtypes = [vp]
         lib.swam_last_error.restype = ctypes.c_char_p
@@ -246,6 +249,9 @@ class Swam:
 
     def check(self):
         self._chk(self.lib.swam_check(self.ctx, _stream()))
+
+    def set_option(self, option: int, value: int):
+        self._chk(self.lib.swam_set_option(self.ctx, option, value))
 
     def launch_count(self) -> int:
         n = ctypes.c_int64()
