@@ -79,6 +79,21 @@ int swam_bind_workspace(swam_ctx* ctx, void* dev_ptr, size_t bytes);
 int swam_score(swam_ctx* ctx, const void* q, const void* k, const float* lse_action,
                float* scores, float* quality, void* stream);
 
+/* Scoring for callers that cannot allocate device memory.  (The paper has no counterpart; this is a packaging
+ * variant of call (1) with the normalisers computed here.)  Some users of this library run the scorer from places
+ * where a workspace cannot be obtained: a policy server whose framework reserved all device memory at start-up so
+ * that cudaMalloc fails, or a control-loop thread that must not call cudaMalloc because it stalls the whole device.
+ * For them the scratch that call (1) keeps in the workspace (the action-row normalisers and the per-chunk partial
+ * maxima and sums) lives in an 8 MiB array inside the library image, which every GPU that loads the library
+ * holds until the process exits.  No workspace needs to be bound and nothing is allocated or freed, on the host or
+ * on the device.  q, k, scores: dev, as in call (1); results equal swam_score(ctx, q, k, NULL, scores, NULL, stream).
+ * Shapes whose scratch exceeds the array (B*N_h*H*4 bytes rounded up to 256, plus B*ceil(L/128)*N_h*H*8 bytes
+ * for bf16) return SWAM_ERR_UNSUPPORTED with the two sizes in swam_last_error.  The first call on each device looks
+ * up the array's device address (with that device current); make that call before any stream capture.  All calls
+ * share the one array and leave their intermediate values in it: nothing in it has to be cleared between calls,
+ * but two calls whose kernels overlap on the GPU (different streams, or different contexts) race on it. */
+int swam_score_noalloc(swam_ctx* ctx, const void* q, const void* k, float* scores, void* stream);
+
 /* (2) Selection and packing metadata, Eq. 4-6, 10-11 with one profiled layer (V = V_all = S):
  * pool = top (N_s - K_s) of max_f S; core_f = top K_c of S[f] within the pool; anchors = top K_s of
  * mu_j / (1 + beta * CV_j) over positions that are core in no frame (population std, fp64, mu_j = 0 => CV_j = 0).

@@ -6,10 +6,18 @@
 // bf16 path feeds the (skinny) products to mma.sync m16n8k16 directly from 16-byte global loads: because a
 // dot product does not care about the order of its terms, each thread's 16-byte chunk of a key row is used
 // as four k-slots of two MMAs and the query fragment is the same 16-byte chunk of the query row.
+#include <mutex>
+
 #include "swam_internal.cuh"
 
 namespace swam {
 namespace {
+
+// Scratch of the allocation-free scoring entry point: the action-row normalisers followed by the per-chunk
+// (max, sum) partials.  It lives in the library image, so every GPU that loads the library holds these bytes until
+// the process exits.  In host code the name is only a stand-in for the symbol: kernels must be given the address
+// that cudaGetSymbolAddress returns for the current device, never the name itself.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -434,6 +442,34 @@ size_t lse_scratch_bytes(const Dims& d) {
   if (d.dtype == 0) return 0;
   const size_t chunks = (d.L + kLseKeys - 1) / kLseKeys;
   return (size_t)d.B * chunks * d.N_h * d.H * sizeof(float2);
+}
+
+size_t static_scratch_need(const Dims& d) {
+  const size_t lse_bytes = ((size_t)d.B * d.N_h * d.H * sizeof(float) + 255) / 256 * 256;
+  return lse_bytes + lse_scratch_bytes(d);
+}
+
+cudaError_t static_scratch(const Dims& d, float** lse, void** partial) {
+  // one look-up per device, made with that device current; later calls reuse the cached address
+  static std::mutex mu;
+  static void* base[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!base[dev]) {
+      void* ptr = nullptr;
+      e = cudaGetSymbolAddress((void**)&ptr, g_static_scratch);
+      if (e != cudaSuccess) return e;
+      base[dev] = ptr;
+    }
+  }
+  const size_t lse_bytes = ((size_t)d.B * d.N_h * d.H * sizeof(float) + 255) / 256 * 256;
+  *lse = (float*)base[dev];
+  *partial = (unsigned char*)base[dev] + lse_bytes;
+  return cudaSuccess;
 }
 
 cudaError_t launch_action_lse(const Dims& d, const void* q, const void* k, float* lse, void* scratch,

@@ -218,6 +218,30 @@ int swam_score(swam_ctx* c, const void* q, const void* k, const float* lse_actio
   return SWAM_OK;
 }
 
+int swam_score_noalloc(swam_ctx* c, const void* q, const void* k, float* scores, void* stream) {
+  if (!c || !q || !k || !scores) return fail(c, SWAM_ERR_INVALID_ARG, "swam_score_noalloc: null argument");
+  if (!aligned16(q) || !aligned16(k) || !aligned16(scores))
+    return fail(c, SWAM_ERR_INVALID_ARG, "swam_score_noalloc: misaligned pointer");
+  if (static_scratch_need(c->d) > kStaticScratchBytes) {
+    snprintf(c->err, sizeof(c->err), "swam_score_noalloc: this shape needs %zu bytes of scratch, the built-in array holds %zu",
+             static_scratch_need(c->d), (size_t)kStaticScratchBytes);
+    return SWAM_ERR_UNSUPPORTED;
+  }
+  float* lse = nullptr;
+  void* partial = nullptr;
+  cudaError_t e = static_scratch(c->d, &lse, &partial);
+  if (e != cudaSuccess) return fail_cuda(c, e, "swam_score_noalloc: cudaGetSymbolAddress");
+  cudaStream_t st = (cudaStream_t)stream;
+  // every normaliser and every partial is written before it is read, so nothing has to start at zero
+  e = launch_action_lse(c->d, q, k, lse, partial, st, &c->launches_i);
+  count(c);
+  if (e != cudaSuccess) return fail_cuda(c, e, "action lse launch");
+  e = launch_score(c->d, c->alpha, q, k, lse, scores, st, &c->launches_i);
+  count(c);
+  if (e != cudaSuccess) return fail_cuda(c, e, "score launch");
+  return SWAM_OK;
+}
+
 int swam_select(swam_ctx* c, const float* scores, int32_t* sel_idx, int32_t* pack_map, int32_t* inv_map, void* stream) {
   if (!c || !scores) return fail(c, SWAM_ERR_INVALID_ARG, "swam_select: null argument");
   if (int r = need_ws(c)) return r;

@@ -31,6 +31,12 @@ size_t lse_scratch_bytes(const Dims& d);
 cudaError_t launch_action_lse(const Dims& d, const void* q, const void* k, float* lse, void* scratch,
                               cudaStream_t st, int* launches);
 
+// static device scratch of the allocation-free scoring entry point
+constexpr size_t kStaticScratchBytes = 8u << 20;
+size_t static_scratch_need(const Dims& d);
+// device addresses inside the static array for the current device (first call per device looks the symbol up)
+cudaError_t static_scratch(const Dims& d, float** lse, void** partial);
+
 // ---- select.cu ------------------------------------------------------------
 size_t select_smem_bytes(const Dims& d);
 cudaError_t select_prepare(const Dims& d);  // opt in to the dynamic shared memory the kernel needs

@@ -24,7 +24,8 @@ OPT_ATTN_VARIANT = 1
 ATTN_AUTO, ATTN_WARP_MMA = 0, 1
 
 EXPORTS = [
-    "swam_create", "swam_destroy", "swam_workspace_bytes", "swam_bind_workspace", "swam_score", "swam_select",
+    "swam_create", "swam_destroy", "swam_workspace_bytes", "swam_bind_workspace", "swam_score", "swam_score_noalloc",
+    "swam_select",
     "swam_pack", "swam_sparse_attn", "swam_scatter", "swam_step", "swam_host_io_bytes", "swam_bind_host_io",
     "swam_step_host", "swam_get_selection", "swam_get_scores", "swam_check", "swam_set_option", "swam_launch_count",
     "swam_last_error", "swam_version",
@@ -66,6 +67,7 @@ def load_library() -> ctypes.CDLL:
         lib.swam_host_io_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t)]
         lib.swam_bind_host_io.argtypes = [vp, vp, ctypes.c_size_t]
         lib.swam_score.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+        lib.swam_score_noalloc.argtypes = [vp, vp, vp, vp, vp]
         lib.swam_select.argtypes = [vp, vp, vp, vp, vp, vp]
         lib.swam_pack.argtypes = [vp] * 9
         lib.swam_sparse_attn.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp]
@@ -187,6 +189,12 @@ class Swam:
         qual = torch.empty((self.B, 3), dtype=torch.float32, device=self.device) if quality else None
         self._chk(self.lib.swam_score(self.ctx, _ptr(q), _ptr(k), _ptr(lse_action), _ptr(scores), _ptr(qual), _stream()))
         return (scores, qual) if quality else scores
+
+    def score_noalloc(self, q, k, scores):
+        """Scores into the caller's `scores` tensor using the library's built-in scratch: no workspace, nothing
+        allocated (for callers that cannot obtain device memory at call time)."""
+        self._chk(self.lib.swam_score_noalloc(self.ctx, _ptr(q), _ptr(k), _ptr(scores), _stream()))
+        return scores
 
     def select(self, scores) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
         sel = torch.empty((self.B, self.F, self.K), dtype=torch.int32, device=self.device)
