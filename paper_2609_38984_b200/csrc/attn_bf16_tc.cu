@@ -19,7 +19,7 @@ namespace swam {
 namespace {
 
 constexpr int kTile = 128;          // query rows per tile and keys per tile
-constexpr int kThreadsTc = 320;     // 8 softmax warps + MMA warp + TMA warp
+constexpr int kThreadsTc = 384;     // 8 softmax warps + MMA warp + TMA warp + 2 idle warps (three full warpgroups)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;
 constexpr unsigned long long kWaitCycles = 4000000000ull;  // about two seconds at 1.9 GHz
@@ -228,7 +228,15 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   auto tm_S = [&](int s) { return tmem + (uint32_t)(s * kTile); };
   auto tm_O = [&](int s) { return tmem + (uint32_t)(2 * kTile + s * D); };
 
-  if (warp == 9) {
+  // register budget: the softmax warpgroups hold a whole S row per thread, the third warpgroup (MMA issuer, TMA
+  // producer, two idle warps) needs almost nothing
+  // (setmaxnreg is a warpgroup-wide instruction: all four warps of a warpgroup execute the same one.  The kernel
+  // starts with 168 registers per thread (384 threads, one CTA per SM); lowering the third warpgroup to 64 releases
+  // 104 x 128 = 13312 registers, and raising the two softmax warpgroups to 216 takes 48 x 256 = 12288 of them.  An
+  // increase beyond what was released would wait forever.)
+  if (warp >= 8) {
+   asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+   if (warp == 9) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       bool ok = true;
@@ -251,7 +259,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           tma_load_4d(sV + st * C::kTileBytes + db * C::kSubTile, &map_v, bar_v_full(st), db * 64, j * kTile, h, b);
       }
     }
-  } else if (warp == 8) {
+   } else if (warp == 8) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       bool ok = mbar_wait(bar_q, 0, abort_flag);
@@ -304,7 +312,9 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       }
       if (ok) tc_commit(bar_o_final);
     }
+   }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     // ------------------------------------------------------------------ softmax warps: one thread per query row
     const int s = warp >> 2;                 // query tile of this warpgroup
     const int r = (warp & 3) * 32 + lane;    // row inside the tile == TMEM lane
