@@ -104,18 +104,39 @@ class ClockSampler:
 # ----------------------------------------------------------------------------------------------------------
 # the swam arm
 # ----------------------------------------------------------------------------------------------------------
-def median_us(fn, iters, flush):
-    """Median device time of fn() in microseconds, L2 flushed (a buffer larger than L2 is rewritten) before each run."""
-    times = []
-    for _ in range(iters):
-        flush.fill_(1)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
+N_ROT = 4  # rotating input sets for per-stage timing: their footprint exceeds L2 several times over
+
+
+def graph_of(fn):
+    """Capture fn() (which enqueues kernels on the current stream) into a CUDA graph."""
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        fn()   # warm-up outside capture (first-use attribute calls, tensor maps)
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
         fn()
-        b.record()
-        b.synchronize()
-        times.append(a.elapsed_time(b) * 1e3)
-    return float(np.median(times))
+    return g
+
+
+def per_launch_us(fns, reps):
+    """Average device time per launch: the callables (one per rotating input set, so consecutive launches read cold
+    data) are captured into one CUDA graph that is replayed `reps` times between two events."""
+    def all_sets():
+        for f in fns:
+            f()
+    g = graph_of(all_sets)
+    g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / (reps * len(fns))
 
 
 def bench_swam(args):
@@ -143,25 +164,29 @@ def bench_swam(args):
         for x, m in zip(dev_steps, modes):
             ctx.step(x["q"], x["k"], x["v"], m, out)
 
+    # the cycle has a fixed shape (fixed packed length), so it is captured once and replayed
+    l0 = ctx.launch_count()
+    cycle()
+    launches_per_cycle = ctx.launch_count() - l0
+    cycle_graph = graph_of(cycle)
     for _ in range(max(args.warmup, 3)):
-        cycle()
+        cycle_graph.replay()
     ctx.check()
 
     sampler = ClockSampler(local_rank)
     sd.barrier(device)
     torch.cuda.synchronize()
-    launches0 = ctx.launch_count()
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
-        cycle()
+        cycle_graph.replay()
     e1.record()
     torch.cuda.synchronize()
     clocks = sampler.stop()
     sd.barrier(device)
     ms_local = e0.elapsed_time(e1)
-    launches = ctx.launch_count() - launches0
+    launches = launches_per_cycle * args.steps
     ctx.check()
     ms_total = sd.max_over_ranks(ms_local, device)
     tokens_per_cycle = wl.batch * (wl.seq_len + (R - 1) * wl.packed_len)
@@ -194,37 +219,47 @@ def bench_swam(args):
 
     line = None
     if rank == 0:
-        # per-stage device times (L2 flushed before each run), through the individual C-ABI calls
-        flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)
+        # per-stage device times through the individual C-ABI calls; every launch of a stage reads one of N_ROT
+        # rotating input sets (together several times L2), launches are replayed back to back from a CUDA graph
+        lib, P, S = ctx.lib, swam._ptr, swam._stream
         x0, x1 = dev_steps[0], dev_steps[-1]
-        it = max(5, min(args.steps, 30))
+        rot = [{n: (x0[n] if i == 0 else x1[n] if i == 1 else x0[n].clone()) for n in "qkv"} for i in range(N_ROT)]
         _, lse_act, _ = ctx.cached_scores()
-        sel, pm, im = ctx.selection()
-        scores = ctx.score(x0["q"], x0["k"], lse_act)
-        qp, kp, vp = ctx.pack(x1["q"], x1["k"], x1["v"], pm)
-        op = ctx.sparse_attn(qp, kp, vp)
+        lse_act = lse_act.clone()
+        sel, pm, im = (t.clone() for t in ctx.selection())
+        scores = [ctx.score(r["q"], r["k"], lse_act) for r in rot]
+        packed = [ctx.pack(r["q"], r["k"], r["v"], pm) for r in rot]
+        outs_p = [ctx.sparse_attn(*pk) for pk in packed]
+        outs = [out] + [out.clone() for _ in range(N_ROT - 1)]
         eb = wl.elem_bytes
         row = wl.row_elems * eb
         B, L, Lp = wl.batch, wl.seq_len, wl.packed_len
         fut = wl.n_frames * wl.n_spatial
+        reps = max(3, min(args.steps, 20))
+
+        def stage(make):
+            return per_launch_us([make(i) for i in range(N_ROT)], reps)
+
         stage_us = {
-            "attn_dense": median_us(lambda: ctx.sparse_attn(x0["q"], x0["k"], x0["v"]), max(3, it // 3), flush),
-            "score": median_us(lambda: ctx.lib.swam_score(ctx.ctx, swam._ptr(x0["q"]), swam._ptr(x0["k"]), swam._ptr(lse_act),
-                                                          swam._ptr(scores), None, swam._stream()), it, flush),
-            "score_with_lse": median_us(lambda: ctx.lib.swam_score(ctx.ctx, swam._ptr(x0["q"]), swam._ptr(x0["k"]), None,
-                                                                   swam._ptr(scores), None, swam._stream()), it, flush),
-            "select": median_us(lambda: ctx.lib.swam_select(ctx.ctx, swam._ptr(scores), swam._ptr(sel), swam._ptr(pm),
-                                                            swam._ptr(im), swam._stream()), it, flush),
-            "pack": median_us(lambda: ctx.lib.swam_pack(ctx.ctx, swam._ptr(x1["q"]), swam._ptr(x1["k"]), swam._ptr(x1["v"]),
-                                                        swam._ptr(pm), swam._ptr(qp), swam._ptr(kp), swam._ptr(vp),
-                                                        swam._stream()), it, flush),
-            "attn_packed": median_us(lambda: ctx.lib.swam_sparse_attn(ctx.ctx, swam._ptr(qp), swam._ptr(kp), swam._ptr(vp), Lp,
-                                                                      swam._ptr(op), None, swam._stream()), it, flush),
-            "scatter": median_us(lambda: ctx.lib.swam_scatter(ctx.ctx, swam._ptr(op), swam._ptr(pm), swam._ptr(im),
-                                                              swam._ptr(out), swam._ptr(out), swam._stream()), it, flush),
-            "full_step": median_us(lambda: ctx.step(x0["q"], x0["k"], x0["v"], swam.REFRESH_FULL, out), max(3, it // 3), flush),
-            "sparse_step": median_us(lambda: ctx.step(x1["q"], x1["k"], x1["v"], swam.REUSE, out), it, flush),
-            "light_refresh_step": median_us(lambda: ctx.step(x1["q"], x1["k"], x1["v"], swam.REFRESH_LIGHT, out), it, flush),
+            "attn_dense": stage(lambda i: lambda: lib.swam_sparse_attn(ctx.ctx, P(rot[i]["q"]), P(rot[i]["k"]), P(rot[i]["v"]), L,
+                                                                       P(outs[i]), None, S())),
+            "score": stage(lambda i: lambda: lib.swam_score(ctx.ctx, P(rot[i]["q"]), P(rot[i]["k"]), P(lse_act), P(scores[i]),
+                                                            None, S())),
+            "score_with_lse": stage(lambda i: lambda: lib.swam_score(ctx.ctx, P(rot[i]["q"]), P(rot[i]["k"]), None,
+                                                                     P(scores[i]), None, S())),
+            "select": stage(lambda i: lambda: lib.swam_select(ctx.ctx, P(scores[i]), P(sel), P(pm), P(im), S())),
+            "pack": stage(lambda i: lambda: lib.swam_pack(ctx.ctx, P(rot[i]["q"]), P(rot[i]["k"]), P(rot[i]["v"]), P(pm),
+                                                          P(packed[i][0]), P(packed[i][1]), P(packed[i][2]), S())),
+            "attn_packed": stage(lambda i: lambda: lib.swam_sparse_attn(ctx.ctx, P(packed[i][0]), P(packed[i][1]),
+                                                                        P(packed[i][2]), Lp, P(outs_p[i]), None, S())),
+            "scatter": stage(lambda i: lambda: lib.swam_scatter(ctx.ctx, P(outs_p[i]), P(pm), P(im), P(outs[i]), P(outs[i]),
+                                                                S())),
+            "full_step": stage(lambda i: lambda: lib.swam_step(ctx.ctx, P(rot[i]["q"]), P(rot[i]["k"]), P(rot[i]["v"]),
+                                                               swam.REFRESH_FULL, P(outs[i]), S())),
+            "sparse_step": stage(lambda i: lambda: lib.swam_step(ctx.ctx, P(rot[i]["q"]), P(rot[i]["k"]), P(rot[i]["v"]),
+                                                                 swam.REUSE, P(outs[i]), S())),
+            "light_refresh_step": stage(lambda i: lambda: lib.swam_step(ctx.ctx, P(rot[i]["q"]), P(rot[i]["k"]),
+                                                                        P(rot[i]["v"]), swam.REFRESH_LIGHT, P(outs[i]), S())),
         }
         ctx.check()
         algo = {  # algorithmic bytes / flops per launch
@@ -266,10 +301,12 @@ def bench_swam(args):
             "config": {"workload": wl0.name, "batch_per_gpu": wl.batch, "seq_len": wl.seq_len, "packed_len": wl.packed_len,
                        "heads": wl.n_heads, "head_dim": wl.head_dim, "keep": wl.keep, "k_core": wl.budgets[0],
                        "k_anchor": wl.budgets[1], "refresh_interval": R,
-                       "step": f"one refresh cycle: 1 full step + {R - 1} sparse step(s)",
+                       "step": f"one refresh cycle: 1 full step + {R - 1} sparse step(s), replayed from a CUDA graph",
                        "tokens_per_step": tokens_per_cycle,
                        "l2": f"inputs exceed L2: {3 * R * full_bytes / 1e6:.0f} MB of q/k/v per step"
                              if 3 * R * full_bytes > (126 << 20) else "inputs smaller than L2, no flush in the step loop",
+                       "stage_timing": f"per stage: {N_ROT} rotating input sets (each launch reads cold data), launches "
+                                       "replayed back to back from a CUDA graph, CUDA events around the loop",
                        "parallelism": f"sample-sharded x{world}"},
             "sparse_step_us": stages["sparse_step"]["us"], "full_step_us": stages["full_step"]["us"],
             "roofline": roofline, "stages": stages, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),

@@ -1,15 +1,154 @@
 // Packing (Sec. 4.2) and scatter / cached-prediction blend (Eq. 7): row copies by index.
 //
-// Rows are N_h*D elements (256 B .. 8 KB), contiguous and 16-byte aligned, so both are pure HBM streams of
-// 16-byte chunks.  Each thread moves kUnroll chunks per iteration, all loads issued before the first store,
-// and the grid is a multiple of the SM count so that every SM holds the same number of resident CTAs.
+// Rows are N_h*D elements (256 B .. 16 KB), contiguous and 16-byte aligned, so pack and the in-place scatter are
+// pure HBM streams.  They run on the bulk-copy engine: one thread per warp moves row segments global -> shared ->
+// global with cp.async.bulk through a private ring of shared-memory buffers, so no data passes through registers
+// and each SM keeps 128 KB of copies in flight.  The 32 lanes of the warp fetch and validate the next 32 map
+// entries at once.  Waits on the load barriers are bounded; an out-of-range map entry is skipped and flagged.
+// The blend into a separate output buffer (out != cached) reads every row of the full sequence and uses plain
+// 16-byte loads and stores.
 #include "swam_internal.cuh"
 
 namespace swam {
 namespace {
 
-constexpr int kCopyThreads = 256;
-constexpr int kUnroll = 4;
+constexpr int kWarps = 8;
+constexpr int kStages = 4;
+constexpr int kSegMax = 4096;  // bytes per ring buffer
+constexpr unsigned long long kWaitCycles = 4000000000ull;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  const unsigned long long t0 = clock64();
+  while (true) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return true;
+    if ((unsigned long long)(clock64() - t0) > kWaitCycles) return false;
+  }
+}
+
+struct RowCopyParams {
+  const unsigned char* src[3];
+  unsigned char* dst[3];
+  const int32_t* src_idx;  // [B, n_rows] row of src for each listed row, or nullptr (identity)
+  const int32_t* dst_idx;  // [B, n_rows] row of dst for each listed row, or nullptr (identity)
+  int* status;
+  int n_tensors;
+  int n_rows;       // listed rows per sample
+  int src_rows;     // rows per sample in src
+  int dst_rows;     // rows per sample in dst
+  int row_bytes;
+  int seg_bytes;    // row_bytes / segs, <= kSegMax, multiple of 16
+  int segs;         // segments per row
+  long long units;  // n_tensors * B * n_rows * segs
+};
+
+// unit id -> (tensor, sample * n_rows + listed row, segment); units of one row are adjacent
+__global__ void __launch_bounds__(kWarps * 32, 1) row_copy_bulk_kernel(const RowCopyParams p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ __align__(8) unsigned long long bars[kWarps * kStages];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  unsigned char* ring = smem + (size_t)warp * kStages * kSegMax;
+  const uint32_t ring_a = smem_addr(ring);
+  const uint32_t bar0 = smem_addr(&bars[warp * kStages]);
+  if (lane == 0) {
+    for (int s = 0; s < kStages; ++s)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8 * s) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+
+  const long long n_warps = (long long)gridDim.x * kWarps;
+  const long long gw = (long long)blockIdx.x * kWarps + warp;
+  // this warp's units: gw, gw + n_warps, ...; processed in batches of 32 (one map look-up per lane)
+  const long long my_units = (p.units > gw) ? (p.units - gw + n_warps - 1) / n_warps : 0;
+  const long long rows_per_tensor = p.units / p.n_tensors / p.segs;
+
+  long long issued = 0, stored = 0;  // lane 0's counters over valid units
+  bool ok = true;
+  // lane 0 keeps up to kStages - 1 loads in flight; src/dst offsets of issued-but-not-stored units
+  long long pend_dst[kStages];
+  int pend_z[kStages];
+
+  auto retire_one = [&]() {  // wait for the oldest load, send it out, free one ring slot
+    const int st = (int)(stored % kStages);
+    if (!mbar_wait_bounded(bar0 + 8 * st, (uint32_t)((stored / kStages) & 1))) { ok = false; return; }
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(p.dst[pend_z[st]] + pend_dst[st]), "r"(ring_a + st * kSegMax), "r"(p.seg_bytes) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    ++stored;
+  };
+
+  for (long long b0 = 0; b0 < my_units && ok; b0 += 32) {
+    // every lane resolves one unit of the batch
+    const long long u = gw + (b0 + lane) * n_warps;
+    long long s_off = -1, d_off = -1;
+    int z = 0;
+    if (b0 + lane < my_units) {
+      const long long row_id = u / p.segs;            // tensor-major: z * rows_per_tensor + (b * n_rows + r)
+      const int seg = (int)(u - row_id * p.segs);
+      z = (int)(row_id / rows_per_tensor);
+      const long long br = row_id - (long long)z * rows_per_tensor;
+      const long long b = br / p.n_rows;
+      const long long lr = br - b * p.n_rows;
+      long long srow = lr, drow = lr;
+      bool valid = true;
+      if (p.src_idx) { srow = p.src_idx[br]; valid = srow >= 0 && srow < p.src_rows; }
+      if (p.dst_idx) { drow = p.dst_idx[br]; valid = valid && drow >= 0 && drow < p.dst_rows; }
+      if (valid) {
+        s_off = (b * p.src_rows + srow) * (long long)p.row_bytes + (long long)seg * p.seg_bytes;
+        d_off = (b * p.dst_rows + drow) * (long long)p.row_bytes + (long long)seg * p.seg_bytes;
+      } else if (seg == 0) {
+        atomicOr(p.status, ST_BAD_MAP);
+      }
+    }
+    const int in_batch = (int)((my_units - b0 < 32) ? (my_units - b0) : 32);
+    for (int i = 0; i < in_batch; ++i) {
+      const long long src_o = __shfl_sync(0xffffffffu, s_off, i);
+      const long long dst_o = __shfl_sync(0xffffffffu, d_off, i);
+      const int zz = __shfl_sync(0xffffffffu, z, i);
+      if (lane == 0 && ok && src_o >= 0) {
+        if (issued - stored == kStages - 1) retire_one();
+        if (ok) {
+          const int st = (int)(issued % kStages);
+          // the store that last read this slot (unit issued - kStages) must have finished reading it
+          asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+          const uint32_t bar = bar0 + 8 * st;
+          asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(p.seg_bytes) : "memory");
+          asm volatile(
+              "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+              ::"r"(ring_a + st * kSegMax), "l"(p.src[zz] + src_o), "r"(p.seg_bytes), "r"(bar) : "memory");
+          pend_dst[st] = dst_o;
+          pend_z[st] = zz;
+          ++issued;
+        }
+      }
+    }
+    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+  }
+  if (lane == 0) {
+    while (ok && stored < issued) retire_one();
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (!ok) atomicOr(p.status, ST_TIMEOUT);
+  }
+}
+
+// ---- blend into a separate buffer: out[b,t] = inv[b,t] >= 0 ? out_p[b, inv[b,t]] : cached[b,t] -----------------
+constexpr int kBlendThreads = 256;
+
+struct BlendParams {
+  const uint4* out_p;
+  const uint4* cached;
+  uint4* out;
+  const int32_t* inv_map;  // [B, L]
+  int* status;
+  int L, Lp, chunks;
+  long long rows;  // B * L
+};
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   uint4 r;
@@ -19,106 +158,61 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   return r;
 }
 
-struct RowCopyParams {
-  const uint4* src[3];
-  uint4* dst[3];
-  const int32_t* src_idx;  // [B, n_rows] row of src for each listed row, or nullptr (identity)
-  const int32_t* dst_idx;  // [B, n_rows] row of dst for each listed row, or nullptr (identity)
-  int* status;
-  int n_tensors;
-  int n_rows;       // listed rows per sample
-  int src_rows;     // rows per sample in src
-  int dst_rows;     // rows per sample in dst
-  int chunks;       // 16-byte chunks per row
-  long long total;  // n_tensors * B * n_rows * chunks
-};
-
-// chunk id -> (tensor, sample, listed row, chunk in row)
-__global__ void __launch_bounds__(kCopyThreads) row_copy_kernel(const RowCopyParams p) {
-  const long long stride = (long long)gridDim.x * kCopyThreads;
-  const long long per_tensor = p.total / p.n_tensors;
-  for (long long base = (long long)blockIdx.x * kCopyThreads + threadIdx.x; base < p.total; base += stride * kUnroll) {
-    uint4 val[kUnroll];
-    uint4* out[kUnroll];
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const long long id = base + (long long)u * stride;
-      out[u] = nullptr;
-      if (id < p.total) {
-        const int z = (int)(id / per_tensor);
-        const long long r = id - (long long)z * per_tensor;
-        const int c = (int)(r % p.chunks);
-        const long long row = r / p.chunks;          // b * n_rows + listed row
-        const long long b = row / p.n_rows;
-        const long long lr = row - b * p.n_rows;
-        long long srow = lr, drow = lr;
-        bool ok = true;
-        if (p.src_idx) { srow = p.src_idx[row]; ok = srow >= 0 && srow < p.src_rows; }
-        if (p.dst_idx) { drow = p.dst_idx[row]; ok = ok && drow >= 0 && drow < p.dst_rows; }
-        if (ok) {
-          val[u] = ld_stream(p.src[z] + (b * p.src_rows + srow) * p.chunks + c);
-          out[u] = p.dst[z] + (b * p.dst_rows + drow) * p.chunks + c;
-        } else if (c == 0) {
-          atomicOr(p.status, ST_BAD_MAP);
-        }
-      }
+// one warp per row, lanes stride over the row's 16-byte chunks, four chunks in flight per lane
+__global__ void __launch_bounds__(kBlendThreads) blend_kernel(const BlendParams p) {
+  const int lane = threadIdx.x & 31;
+  const long long warps = (long long)gridDim.x * (kBlendThreads / 32);
+  for (long long row = (long long)blockIdx.x * (kBlendThreads / 32) + (threadIdx.x >> 5); row < p.rows; row += warps) {
+    const long long b = row / p.L;
+    const int pr = p.inv_map[row];
+    if (pr >= p.Lp) {
+      if (lane == 0) atomicOr(p.status, ST_BAD_MAP);
+      continue;
     }
+    const uint4* src = (pr >= 0) ? p.out_p + (b * p.Lp + pr) * p.chunks : p.cached + row * p.chunks;
+    uint4* dst = p.out + row * p.chunks;
+    for (int c0 = lane; c0 < p.chunks; c0 += 128) {
+      uint4 v[4];
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u)
-      if (out[u]) *out[u] = val[u];
+      for (int u = 0; u < 4; ++u)
+        if (c0 + 32 * u < p.chunks) v[u] = ld_stream(src + c0 + 32 * u);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (c0 + 32 * u < p.chunks) dst[c0 + 32 * u] = v[u];
+    }
   }
 }
 
-struct BlendParams {
-  const uint4* out_p;
-  const uint4* cached;
-  uint4* out;
-  const int32_t* inv_map;  // [B, L]
-  int* status;
-  int L, Lp, chunks;
-  long long total;  // B * L * chunks
-};
-
-// out[b,t] = inv[b,t] >= 0 ? out_p[b, inv[b,t]] : cached[b,t]
-__global__ void __launch_bounds__(kCopyThreads) blend_kernel(const BlendParams p) {
-  const long long stride = (long long)gridDim.x * kCopyThreads;
-  for (long long base = (long long)blockIdx.x * kCopyThreads + threadIdx.x; base < p.total; base += stride * kUnroll) {
-    uint4 val[kUnroll];
-    bool live[kUnroll];
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const long long id = base + (long long)u * stride;
-      live[u] = id < p.total;
-      if (live[u]) {
-        const int c = (int)(id % p.chunks);
-        const long long row = id / p.chunks;  // b * L + t
-        const long long b = row / p.L;
-        const int pr = p.inv_map[row];
-        if (pr >= p.Lp) {
-          if (c == 0) atomicOr(p.status, ST_BAD_MAP);
-          live[u] = false;
-        } else if (pr >= 0) {
-          val[u] = ld_stream(p.out_p + (b * p.Lp + pr) * p.chunks + c);
-        } else {
-          val[u] = ld_stream(p.cached + id);
-        }
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u)
-      if (live[u]) p.out[base + (long long)u * stride] = val[u];
-  }
-}
-
-int copy_grid(long long total) {
+int sm_count() {
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const long long per_cta = (long long)kCopyThreads * kUnroll;
-  long long need = (total + per_cta - 1) / per_cta;
-  const long long cap = (long long)sms * 8;  // 8 resident CTAs of 256 threads per SM
-  if (need >= cap) return (int)cap;
-  return (int)(need < 1 ? 1 : need);
+  return sms;
+}
+
+cudaError_t launch_row_copy(RowCopyParams& p, int batch, cudaStream_t st) {
+  int segs = 1;
+  while (p.row_bytes / segs > kSegMax || (p.row_bytes % (segs * 16)) != 0) {
+    segs *= 2;
+    if (segs > 64) return cudaErrorInvalidConfiguration;
+  }
+  p.segs = segs;
+  p.seg_bytes = p.row_bytes / segs;
+  p.units = (long long)p.n_tensors * batch * p.n_rows * segs;
+  if (p.units == 0) return cudaSuccess;
+  const size_t smem = (size_t)kWarps * kStages * kSegMax;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(row_copy_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  long long ctas = (p.units + kWarps * 4 - 1) / (kWarps * 4);  // at least four units per warp
+  const int sms = sm_count();
+  if (ctas > sms) ctas = sms;
+  if (ctas < 1) ctas = 1;
+  row_copy_bulk_kernel<<<(int)ctas, kWarps * 32, smem, st>>>(p);
+  return cudaGetLastError();
 }
 
 }  // namespace
@@ -128,38 +222,34 @@ cudaError_t launch_pack(const Dims& d, const void* const src[3], void* const dst
   RowCopyParams p{};
   int n = 0;
   for (int i = 0; i < 3; ++i)
-    if (src[i] && dst[i]) { p.src[n] = (const uint4*)src[i]; p.dst[n] = (uint4*)dst[i]; ++n; }
-  if (n == 0) return cudaSuccess;
+    if (src[i] && dst[i]) { p.src[n] = (const unsigned char*)src[i]; p.dst[n] = (unsigned char*)dst[i]; ++n; }
+  if (n == 0 || d.Lp == 0) return cudaSuccess;
   p.src_idx = pack_map; p.dst_idx = nullptr; p.status = status;
   p.n_tensors = n; p.n_rows = d.Lp; p.src_rows = d.L; p.dst_rows = d.Lp;
-  p.chunks = d.N_h * d.D * (d.dtype == 0 ? 4 : 2) / 16;
-  p.total = (long long)n * d.B * d.Lp * p.chunks;
-  if (p.total == 0) return cudaSuccess;
+  p.row_bytes = d.N_h * d.D * (d.dtype == 0 ? 4 : 2);
   ++*launches;
-  row_copy_kernel<<<copy_grid(p.total), kCopyThreads, 0, st>>>(p);
-  return cudaGetLastError();
+  return launch_row_copy(p, d.B, st);
 }
 
 cudaError_t launch_scatter(const Dims& d, const void* out_p, const int32_t* pack_map, const int32_t* inv_map,
                            const void* cached, void* out, int* status, cudaStream_t st, int* launches) {
-  const int chunks = d.N_h * d.D * (d.dtype == 0 ? 4 : 2) / 16;
+  const int row_bytes = d.N_h * d.D * (d.dtype == 0 ? 4 : 2);
+  if (d.Lp == 0) return cudaSuccess;
   if (cached == out) {
     RowCopyParams p{};
-    p.src[0] = (const uint4*)out_p; p.dst[0] = (uint4*)out;
+    p.src[0] = (const unsigned char*)out_p; p.dst[0] = (unsigned char*)out;
     p.src_idx = nullptr; p.dst_idx = pack_map; p.status = status;
     p.n_tensors = 1; p.n_rows = d.Lp; p.src_rows = d.Lp; p.dst_rows = d.L;
-    p.chunks = chunks;
-    p.total = (long long)d.B * d.Lp * chunks;
-    if (p.total == 0) return cudaSuccess;
+    p.row_bytes = row_bytes;
     ++*launches;
-    row_copy_kernel<<<copy_grid(p.total), kCopyThreads, 0, st>>>(p);
-    return cudaGetLastError();
+    return launch_row_copy(p, d.B, st);
   }
-  BlendParams p{(const uint4*)out_p, (const uint4*)cached, (uint4*)out, inv_map, status, d.L, d.Lp, chunks,
-                (long long)d.B * d.L * chunks};
-  if (p.total == 0) return cudaSuccess;
+  BlendParams p{(const uint4*)out_p, (const uint4*)cached, (uint4*)out, inv_map, status, d.L, d.Lp, row_bytes / 16,
+                (long long)d.B * d.L};
   ++*launches;
-  blend_kernel<<<copy_grid(p.total), kCopyThreads, 0, st>>>(p);
+  const long long need = (p.rows + 7) / 8;
+  const long long cap = (long long)sm_count() * 8;
+  blend_kernel<<<(int)(need < cap ? need : cap), kBlendThreads, 0, st>>>(p);
   return cudaGetLastError();
 }
 

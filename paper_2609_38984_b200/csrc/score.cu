@@ -47,14 +47,13 @@ struct ScoreParams {
   Alpha alpha;
 };
 
-constexpr int kScoreThreads = 256;
 constexpr int kScoreKeys = 32;  // keys per CTA: 2 m-tiles of 16
-constexpr int kHeadGroups = 4;
 
 // smem: query fragments [N_h][D/32][NT][32] uint4, lambda*log2e [N_h][NT*8], partial sums [4][32]
-template <int D, int NT>
-__global__ void __launch_bounds__(kScoreThreads, 2) score_bf16_kernel(const ScoreParams p) {
+template <int D, int NT, int kHeadGroups>
+__global__ void __launch_bounds__(64 * kHeadGroups, 8 / kHeadGroups) score_bf16_kernel(const ScoreParams p) {
   constexpr int KB = D / 32;
+  constexpr int kScoreThreads = 64 * kHeadGroups;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint4* q_frag = reinterpret_cast<uint4*>(smem_raw);
   float* lam2 = reinterpret_cast<float*>(q_frag + (size_t)p.N_h * KB * NT * 32);
@@ -66,7 +65,8 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_bf16_kernel(const Scor
   const int64_t act0 = (int64_t)p.n_obs + (int64_t)p.F * p.N_s;
   const int64_t tok = (int64_t)p.N_h * D;
 
-  // stage this frame's query group as MMA B fragments (zero beyond the group)
+  // stage this frame's query group as MMA B fragments (zero beyond the group): asynchronous 16-byte copies, all in
+  // flight at once, overlapped with the first key loads below
   const int n_frag = p.N_h * KB * NT * 32;
   for (int i = tid; i < n_frag; i += kScoreThreads) {
     const int ln = i & 31;
@@ -74,19 +74,17 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_bf16_kernel(const Scor
     const int kb = ((i >> 5) / NT) % KB;
     const int h = (i >> 5) / (NT * KB);
     const int n = nt * 8 + (ln >> 2), t = ln & 3;
-    uint4 val = make_uint4(0, 0, 0, 0);
-    if (n < p.g) {
-      const __nv_bfloat16* src = p.q + ((int64_t)b * p.L + act0 + (int64_t)f * p.g + n) * tok + (int64_t)h * D +
-                                 kb * 32 + t * 8;
-      val = *reinterpret_cast<const uint4*>(src);
-    }
-    q_frag[i] = val;
+    const bool in = n < p.g;
+    const __nv_bfloat16* src = p.q + ((int64_t)b * p.L + act0 + (int64_t)f * p.g + (in ? n : 0)) * tok + (int64_t)h * D +
+                               kb * 32 + t * 8;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(q_frag + i)),
+                 "l"(src), "r"(in ? 16 : 0) : "memory");
   }
+  asm volatile("cp.async.commit_group;" ::: "memory");
   for (int i = tid; i < p.N_h * NT * 8; i += kScoreThreads) {
     const int n = i % (NT * 8), h = i / (NT * 8);
     lam2[i] = (n < p.g) ? p.lse[((int64_t)b * p.N_h + h) * p.H + f * p.g + n] * kLog2e : 0.f;
   }
-  __syncthreads();
 
   const int mt = warp & 1, hg = warp >> 1;
   const int gq = lane >> 2, t = lane & 3;
@@ -137,9 +135,12 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_bf16_kernel(const Scor
   // heads hg, hg+4, ... with the next head's keys in flight while this head's products run
   int h = hg;
   if (h < p.N_h) load(h, 0);
+  if (h + kHeadGroups < p.N_h) load(h + kHeadGroups, 1);
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
   for (; h < p.N_h; h += 2 * kHeadGroups) {
     const int h1 = h + kHeadGroups, h2 = h + 2 * kHeadGroups;
-    if (h1 < p.N_h) load(h1, 1);
+    if (h != hg && h1 < p.N_h) load(h1, 1);
     compute(h, 0);
     if (h1 < p.N_h) {
       if (h2 < p.N_h) load(h2, 0);
@@ -157,7 +158,11 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_bf16_kernel(const Scor
   }
   __syncthreads();
   if (tid < kScoreKeys && key0 + tid < p.N_s) {
-    const float s = (red[tid] + red[kScoreKeys + tid]) + (red[2 * kScoreKeys + tid] + red[3 * kScoreKeys + tid]);
+    float s = 0.f;
+#pragma unroll
+    for (int q = 0; q < kHeadGroups; q += 4)
+      s += (red[q * kScoreKeys + tid] + red[(q + 1) * kScoreKeys + tid]) +
+           (red[(q + 2) * kScoreKeys + tid] + red[(q + 3) * kScoreKeys + tid]);
     p.scores[((int64_t)b * p.F + f) * p.N_s + key0 + tid] = s * p.inv_nh;
   }
 }
@@ -197,38 +202,41 @@ __global__ void __launch_bounds__(256) score_f32_kernel(const ScoreParamsF32 p) 
 }
 
 // ---- layer quality (Eq. 9): R = sum S / F, E = mean normalised spatial entropy, Q = R (1 - E) ----------
-__device__ double block_sum(double v, double* sh) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  __syncthreads();
-  if (lane == 0) sh[warp] = v;
-  __syncthreads();
-  double tot = 0.0;
-  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += sh[w];
-  return tot;
-}
+// One CTA per sample, one pass over the scores: with a_f = sum_j s and b_f = sum_j s ln s the entropy of frame f is
+// ln a_f - b_f / a_f.  Warps take (frame, part) units; partial sums are combined in a fixed order.
+constexpr int kQualThreads = 1024;
 
-__global__ void __launch_bounds__(256) quality_kernel(const float* scores, float* quality, int F, int N_s) {
-  __shared__ double sh[8];
-  const int b = blockIdx.x;
+__global__ void __launch_bounds__(kQualThreads) quality_kernel(const float* scores, float* quality, int F, int N_s,
+                                                               int parts) {
+  extern __shared__ double2 part_sums[];  // [F * parts]
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, b = blockIdx.x;
   const float* s = scores + (int64_t)b * F * N_s;
-  double total = 0.0, ent = 0.0;
-  for (int f = 0; f < F; ++f) {
-    double part = 0.0;
-    for (int j = threadIdx.x; j < N_s; j += blockDim.x) part += (double)s[f * N_s + j];
-    const double fs = block_sum(part, sh);
-    total += fs;
-    double e = 0.0;
-    if (fs > 0.0) {
-      for (int j = threadIdx.x; j < N_s; j += blockDim.x) {
-        const double pj = (double)s[f * N_s + j] / fs;
-        if (pj > 0.0) e -= pj * log(pj);
-      }
+  const int per = (N_s + parts - 1) / parts;
+  for (int u = warp; u < F * parts; u += kQualThreads / 32) {
+    const int f = u / parts, part = u % parts;
+    const int j1 = min(N_s, (part + 1) * per);
+    double a = 0.0, bq = 0.0;
+    for (int j = part * per + lane; j < j1; j += 32) {
+      const float v = s[f * N_s + j];
+      a += (double)v;
+      if (v > 0.f) bq += (double)(v * logf(v));
     }
-    ent += block_sum(e, sh);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      a += __shfl_xor_sync(0xffffffffu, a, o);
+      bq += __shfl_xor_sync(0xffffffffu, bq, o);
+    }
+    if (lane == 0) part_sums[u] = make_double2(a, bq);
   }
+  __syncthreads();
   if (threadIdx.x == 0) {
+    double total = 0.0, ent = 0.0;
+    for (int f = 0; f < F; ++f) {
+      double a = 0.0, bq = 0.0;
+      for (int q = 0; q < parts; ++q) { a += part_sums[f * parts + q].x; bq += part_sums[f * parts + q].y; }
+      total += a;
+      if (a > 0.0) ent += log(a) - bq / a;
+    }
     const double R = total / (double)F;
     const double E = ent / ((double)F * log((double)N_s));
     quality[b * 3 + 0] = (float)R;
@@ -386,17 +394,22 @@ __global__ void __launch_bounds__(128) lse_f32_kernel(const float* q, const floa
   }
 }
 
-template <int D, int NT>
-cudaError_t launch_score_bf16(const Dims& d, const ScoreParams& p, cudaStream_t st) {
+template <int D, int NT, int HG>
+cudaError_t launch_score_bf16_hg(const Dims& d, const ScoreParams& p, cudaStream_t st) {
   const size_t smem = (size_t)d.N_h * (D / 32) * NT * 32 * sizeof(uint4) + (size_t)d.N_h * NT * 8 * sizeof(float) +
-                      kHeadGroups * kScoreKeys * sizeof(float);
+                      HG * kScoreKeys * sizeof(float);
   if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
-  cudaError_t e = cudaFuncSetAttribute(score_bf16_kernel<D, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(score_bf16_kernel<D, NT, HG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid((d.N_s + kScoreKeys - 1) / kScoreKeys, d.F, d.B);
-  score_bf16_kernel<D, NT><<<grid, kScoreThreads, smem, st>>>(p);
+  score_bf16_kernel<D, NT, HG><<<grid, 64 * HG, smem, st>>>(p);
   return cudaGetLastError();
+}
+
+template <int D, int NT>
+cudaError_t launch_score_bf16(const Dims& d, const ScoreParams& p, cudaStream_t st) {
+  return launch_score_bf16_hg<D, NT, 4>(d, p, st);
 }
 
 template <int D>
@@ -434,7 +447,9 @@ cudaError_t launch_score(const Dims& d, const Alpha& alpha, const void* q, const
 
 cudaError_t launch_quality(const Dims& d, const float* scores, float* quality, cudaStream_t st, int* launches) {
   ++*launches;
-  quality_kernel<<<d.B, 256, 0, st>>>(scores, quality, d.F, d.N_s);
+  int parts = 32 / d.F;
+  if (parts < 1) parts = 1;
+  quality_kernel<<<d.B, kQualThreads, (size_t)d.F * parts * sizeof(double2), st>>>(scores, quality, d.F, d.N_s, parts);
   return cudaGetLastError();
 }
 

@@ -52,13 +52,29 @@ __device__ void radix_select(const GroupCtx& g, int n, int k, KeyFn key, CandFn 
   KeyT prefix = 0, mask = 0;
   int remaining = k;
   if (k > 0) {
+    for (int i = g.tid; i < 256; i += g.n_threads) g.hist[i] = 0;
+    group_sync(g.bar_id, g.n_threads);
     for (int shift = kBits - 8; shift >= 0; shift -= 8) {
-      for (int i = g.tid; i < 256; i += g.n_threads) g.hist[i] = 0;
-      group_sync(g.bar_id, g.n_threads);
-      for (int i = g.tid; i < n; i += g.n_threads) {
-        if (cand(i)) {
+      for (int i0 = 0; i0 < n; i0 += g.n_threads) {
+        const int i = i0 + g.tid;
+        bool act = false;
+        int digit = 0;
+        if (i < n && cand(i)) {
           const KeyT kv = key(i);
-          if ((kv & mask) == prefix) atomicAdd(&g.hist[(int)((kv >> shift) & 0xFF)], 1);
+          act = (kv & mask) == prefix;
+          digit = (int)((kv >> shift) & 0xFF);
+        }
+        // keys often share their leading digits: when the whole warp agrees on the digit, one atomic serves it
+        const unsigned live = __ballot_sync(0xffffffffu, act);
+        if (live) {
+          const int lead = __ffs(live) - 1;
+          const int d0 = __shfl_sync(0xffffffffu, digit, lead);
+          const bool same = __all_sync(0xffffffffu, !act || digit == d0);
+          if (same) {
+            if (lane == lead) atomicAdd(&g.hist[d0], __popc(live));
+          } else if (act) {
+            atomicAdd(&g.hist[digit], 1);
+          }
         }
       }
       group_sync(g.bar_id, g.n_threads);
@@ -66,7 +82,7 @@ __device__ void radix_select(const GroupCtx& g, int n, int k, KeyFn key, CandFn 
         // lane owns bins [8*lane, 8*lane+8); suffix = number of keys in bins above the lane's
         int local[8], sum = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { local[j] = g.hist[lane * 8 + j]; sum += local[j]; }
+        for (int j = 0; j < 8; ++j) { local[j] = g.hist[lane * 8 + j]; sum += local[j]; g.hist[lane * 8 + j] = 0; }
         int incl = sum;  // inclusive suffix sum over lanes >= lane
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -97,7 +113,8 @@ __device__ void radix_select(const GroupCtx& g, int n, int k, KeyFn key, CandFn 
       prefix |= (KeyT)g.scal[0] << shift;
       mask |= (KeyT)0xFF << shift;
       remaining = g.scal[1];
-      // (the next pass's histogram reset is followed by a barrier before scal is rewritten)
+      // (warp 0 cleared the bins it read, and the barrier above orders that before the next pass's atomics; scal is
+      // rewritten only after the next pass's histogram barrier)
     }
   }
   // prefix is now the k-th largest key; admit keys above it, and the first `remaining` keys equal to it
@@ -184,12 +201,14 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
   GroupCtx all{0, kSelThreads, tid, hist, scal, warp_tot};
 
   // candidate pool: top (N_s - K_s) of max_f S(f, j)                                   (Eq. 4)
-  auto pool_key = [&](int j) {
+  uint32_t* keyM = reinterpret_cast<uint32_t*>(keyA);  // the anchor keys are built later in the same storage
+  for (int j = tid; j < N; j += kSelThreads) {
     float m = S[j];
     for (int f = 1; f < F; ++f) m = fmaxf(m, S[f * N + j]);
-    return key32(m);
-  };
-  radix_select<uint32_t>(all, N, N - p.Ks, pool_key, [](int) { return true; }, pool);
+    keyM[j] = key32(m);
+  }
+  __syncthreads();
+  radix_select<uint32_t>(all, N, N - p.Ks, [&](int j) { return keyM[j]; }, [](int) { return true; }, pool);
 
   // frame-specific core tokens: top K_c of S(f, .) inside the pool                      (Eq. 5)
   {
