@@ -1,22 +1,30 @@
-// Token selection (Eq. 4-6, 10-11) and packing metadata, one CTA per sample.
+// Token selection (Eq. 4-6, 10-11) and packing metadata: one thread-block cluster per sample.
 //
 // Every TopK is a radix select in shared memory: keys are mapped to unsigned integers whose order is the
 // order of the floating-point values, 8-bit digits are histogrammed from the top, and the digit holding the
-// k-th largest key is located with a warp-shuffle suffix scan.  What remains after the last digit is the
-// exact value of the k-th key; keys equal to it are admitted in ascending index order (ballot/popc ranks),
-// which is the "ties go to the lower index" rule.  The per-frame core selections run concurrently in thread
-// groups synchronised by named barriers; pool and anchor selections use the whole CTA.
+// k-th largest key is located with a warp-shuffle suffix scan.  The passes stop as soon as the bin that holds
+// the k-th key is taken whole; otherwise what remains after the last digit is the exact value of the k-th key and
+// keys equal to it are admitted in ascending index order (ballot/popc ranks), which is the "ties go to the lower
+// index" rule.
+//
+// The CTAs of a cluster (up to 8) each hold the sample's scores in shared memory.  The candidate pool and the anchor
+// selection are small and are computed by every CTA; the per-frame core selections and the map construction are
+// split by frame; core flags and anchor keys are exchanged through distributed shared memory.
 //
 // The anchor statistic is evaluated in fp64 with individually rounded operations (no fused multiply-add) in
 // a fixed order: sum over frames ascending, mean, sum of squared deviations ascending, population standard
 // deviation, CV = sd / mu (0 when mu = 0), key = mu / (1 + beta * CV).
+#include <cooperative_groups.h>
+
 #include "swam_internal.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace swam {
 namespace {
 
 constexpr int kSelThreads = 1024;
-constexpr int kMaxGroups = 8;
+constexpr int kMaxCluster = 8;
 
 __device__ __forceinline__ uint32_t key32(float x) {
   x = x + 0.0f;  // -0 -> +0 so that equal values have equal keys
@@ -29,34 +37,40 @@ __device__ __forceinline__ uint64_t key64(double x) {
   return (u & 0x8000000000000000ull) ? ~u : (u | 0x8000000000000000ull);
 }
 
-// barrier among the `count` threads of one group (count is a multiple of 32); id 0 is the CTA barrier
-__device__ __forceinline__ void group_sync(int id, int count) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
-}
-
-struct GroupCtx {
-  int bar_id;      // named barrier
-  int n_threads;   // threads in the group
-  int tid;         // thread index within the group
-  int* hist;       // [256] shared
-  int* scal;       // [4] shared scalars: digit, remaining
-  int* warp_tot;   // [32] shared
+struct Scratch {
+  int* hist;      // [256] shared
+  int* scal;      // [4] shared: digit, remaining, whole-bin flag
+  int* warp_tot;  // [32] shared
 };
 
-// Radix select among candidates. key(i) -> KeyT for i in [0,n); cand(i) -> bool.
+// exclusive prefix of this warp and the total over all warps of the per-warp counts in s.warp_tot
+__device__ __forceinline__ void warp_bases(const Scratch& s, int warp, int lane, int& wbase, int& total) {
+  const int v = s.warp_tot[lane];
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  wbase = __shfl_sync(0xffffffffu, incl - v, warp);
+  total = __shfl_sync(0xffffffffu, incl, 31);
+}
+
+// Radix select among candidates (whole CTA). key(i) -> KeyT for i in [0,n); cand(i) -> bool.
 // Writes flag_out[i] = 1 for the k selected candidates (0 otherwise, for all i in [0,n)).
 template <typename KeyT, typename KeyFn, typename CandFn>
-__device__ void radix_select(const GroupCtx& g, int n, int k, KeyFn key, CandFn cand, uint8_t* flag_out) {
+__device__ void radix_select(const Scratch& s, int n, int k, KeyFn key, CandFn cand, uint8_t* flag_out) {
   constexpr int kBits = sizeof(KeyT) * 8;
-  const int lane = g.tid & 31, warp = g.tid >> 5, n_warps = g.n_threads >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   KeyT prefix = 0, mask = 0;
   int remaining = k;
+  bool whole_bin = false;  // every key that matches the prefix so far is selected
   if (k > 0) {
-    for (int i = g.tid; i < 256; i += g.n_threads) g.hist[i] = 0;
-    group_sync(g.bar_id, g.n_threads);
+    for (int i = tid; i < 256; i += kSelThreads) s.hist[i] = 0;
+    __syncthreads();
     for (int shift = kBits - 8; shift >= 0; shift -= 8) {
-      for (int i0 = 0; i0 < n; i0 += g.n_threads) {
-        const int i = i0 + g.tid;
+      for (int i0 = 0; i0 < n; i0 += kSelThreads) {
+        const int i = i0 + tid;
         bool act = false;
         int digit = 0;
         if (i < n && cand(i)) {
@@ -71,18 +85,18 @@ __device__ void radix_select(const GroupCtx& g, int n, int k, KeyFn key, CandFn 
           const int d0 = __shfl_sync(0xffffffffu, digit, lead);
           const bool same = __all_sync(0xffffffffu, !act || digit == d0);
           if (same) {
-            if (lane == lead) atomicAdd(&g.hist[d0], __popc(live));
+            if (lane == lead) atomicAdd(&s.hist[d0], __popc(live));
           } else if (act) {
-            atomicAdd(&g.hist[digit], 1);
+            atomicAdd(&s.hist[digit], 1);
           }
         }
       }
-      group_sync(g.bar_id, g.n_threads);
+      __syncthreads();
       if (warp == 0) {
         // lane owns bins [8*lane, 8*lane+8); suffix = number of keys in bins above the lane's
         int local[8], sum = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { local[j] = g.hist[lane * 8 + j]; sum += local[j]; g.hist[lane * 8 + j] = 0; }
+        for (int j = 0; j < 8; ++j) { local[j] = s.hist[lane * 8 + j]; sum += local[j]; s.hist[lane * 8 + j] = 0; }
         int incl = sum;  // inclusive suffix sum over lanes >= lane
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -93,75 +107,75 @@ __device__ void radix_select(const GroupCtx& g, int n, int k, KeyFn key, CandFn 
         const int total = __shfl_sync(0xffffffffu, incl, 0);
         const int want = remaining < total ? remaining : total;  // fewer candidates than k: take them all
         if (want <= 0) {
-          if (lane == 0) { g.scal[0] = 0xFF; g.scal[1] = 0; }
+          if (lane == 0) { s.scal[0] = 0xFF; s.scal[1] = 0; s.scal[2] = 0; }
         } else if (above < want && want <= above + sum) {
           // the want-th largest key lies in this lane's bins
-          int digit = lane * 8, rem = want;
+          int digit = lane * 8, rem = want, in_bin = 0;
           bool found = false;
 #pragma unroll
           for (int j = 7; j >= 0; --j) {
             if (!found) {
-              if (want <= above + local[j]) { digit = lane * 8 + j; rem = want - above; found = true; }
+              if (want <= above + local[j]) { digit = lane * 8 + j; rem = want - above; in_bin = local[j]; found = true; }
               else above += local[j];
             }
           }
-          g.scal[0] = digit;
-          g.scal[1] = rem;
+          s.scal[0] = digit;
+          s.scal[1] = rem;
+          s.scal[2] = (in_bin == rem) ? 1 : 0;
         }
       }
-      group_sync(g.bar_id, g.n_threads);
-      prefix |= (KeyT)g.scal[0] << shift;
+      __syncthreads();
+      prefix |= (KeyT)s.scal[0] << shift;
       mask |= (KeyT)0xFF << shift;
-      remaining = g.scal[1];
-      // (warp 0 cleared the bins it read, and the barrier above orders that before the next pass's atomics; scal is
-      // rewritten only after the next pass's histogram barrier)
+      remaining = s.scal[1];
+      whole_bin = s.scal[2] != 0;
+      // (warp 0 cleared the bins it read before the barrier above; scal is rewritten only after the next pass's
+      // histogram barrier)
+      if (whole_bin) break;
     }
   }
-  // prefix is now the k-th largest key; admit keys above it, and the first `remaining` keys equal to it
+  // keys above the prefix are in; of the keys that match it, all (whole bin) or the first `remaining` by index
   int base = 0;
-  for (int start = 0; start < n; start += g.n_threads) {
-    const int i = start + g.tid;
-    bool c = false, eq = false, gt = false;
-    if (i < n && k > 0) {
-      c = cand(i);
-      if (c) { const KeyT kv = key(i); gt = kv > prefix; eq = kv == prefix; }
+  for (int start = 0; start < n; start += kSelThreads) {
+    const int i = start + tid;
+    bool eq = false, gt = false;
+    if (i < n && k > 0 && cand(i)) {
+      const KeyT kv = key(i) & mask;
+      gt = kv > prefix;
+      eq = kv == prefix;
+    }
+    if (whole_bin) {
+      if (i < n) flag_out[i] = (gt || eq) ? 1 : 0;
+      continue;
     }
     const unsigned bal = __ballot_sync(0xffffffffu, eq);
     const int before = __popc(bal & ((1u << lane) - 1u));
-    group_sync(g.bar_id, g.n_threads);  // warp_tot free to overwrite
-    if (lane == 0) g.warp_tot[warp] = __popc(bal);
-    group_sync(g.bar_id, g.n_threads);
-    int wbase = 0, total = 0;
-    for (int w = 0; w < n_warps; ++w) {
-      const int tw = g.warp_tot[w];
-      if (w < warp) wbase += tw;
-      total += tw;
-    }
+    __syncthreads();  // warp_tot free to overwrite
+    if (lane == 0) s.warp_tot[warp] = __popc(bal);
+    __syncthreads();
+    int wbase, total;
+    warp_bases(s, warp, lane, wbase, total);
     if (i < n) flag_out[i] = (gt || (eq && (base + wbase + before) < remaining)) ? 1 : 0;
     base += total;
   }
-  group_sync(g.bar_id, g.n_threads);
+  __syncthreads();
 }
 
-// Ascending compaction of flagged positions: calls emit(i, rank) for each flagged i; returns the count.
+// Ascending compaction of flagged positions: calls emit(i, rank) for each i (rank -1 when not flagged); returns the count.
 template <typename FlagFn, typename EmitFn>
-__device__ int ranked_emit(const GroupCtx& g, int n, FlagFn flag, EmitFn emit) {
-  const int lane = g.tid & 31, warp = g.tid >> 5, n_warps = g.n_threads >> 5;
+__device__ int ranked_emit(const Scratch& s, int n, FlagFn flag, EmitFn emit) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   int base = 0;
-  for (int start = 0; start < n; start += g.n_threads) {
-    const int i = start + g.tid;
+  for (int start = 0; start < n; start += kSelThreads) {
+    const int i = start + tid;
     const bool fl = (i < n) && flag(i);
     const unsigned bal = __ballot_sync(0xffffffffu, fl);
     const int before = __popc(bal & ((1u << lane) - 1u));
-    group_sync(g.bar_id, g.n_threads);
-    if (lane == 0) g.warp_tot[warp] = __popc(bal);
-    group_sync(g.bar_id, g.n_threads);
-    int wbase = 0, total = 0;
-    for (int w = 0; w < n_warps; ++w) {
-      const int tw = g.warp_tot[w];
-      if (w < warp) wbase += tw;
-      total += tw;
-    }
+    __syncthreads();
+    if (lane == 0) s.warp_tot[warp] = __popc(bal);
+    __syncthreads();
+    int wbase, total;
+    warp_bases(s, warp, lane, wbase, total);
     if (i < n) emit(i, fl ? base + wbase + before : -1);
     base += total;
   }
@@ -174,63 +188,76 @@ struct SelectParams {
   int32_t* pack_map;
   int32_t* inv_map;
   int* status;
-  int n_obs, F, N_s, H, Kc, Ks, L, Lp, n_groups;
+  int n_obs, F, N_s, H, Kc, Ks, L, Lp;
   double beta;
 };
 
+// shared-memory layout (bytes), identical in every CTA of the cluster
+struct SelLayout {
+  size_t keyA, S, keyM, hist, warp_tot, scal, pool, anchor, anycore, core, total;
+};
+__host__ __device__ inline SelLayout sel_layout(int F, int N) {
+  SelLayout l;
+  size_t o = 0;
+  l.keyA = o; o += (size_t)N * 8;
+  l.S = o; o += (size_t)F * N * 4;
+  l.keyM = o; o += (size_t)N * 4;
+  l.hist = o; o += 256 * 4;
+  l.warp_tot = o; o += 32 * 4;
+  l.scal = o; o += 4 * 4;
+  l.pool = o; o += (size_t)N;
+  l.anchor = o; o += (size_t)N;
+  l.anycore = o; o += (size_t)N;
+  o = (o + 3) & ~(size_t)3;
+  l.core = o; o += ((size_t)N + 3) / 4 * 4 * F;   // each frame's flags start on a 4-byte boundary
+  l.total = (o + 15) & ~(size_t)15;
+  return l;
+}
+
 __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int C = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
   const int F = p.F, N = p.N_s, K = p.Kc + p.Ks;
-  // layout: keyA u64[N] | S f32[F*N] | hist int[(groups+1)*256] | warp_tot int[(groups+1)*32] | scal int[(groups+1)*4]
-  //         | pool u8[N] | anchor u8[N] | anycore u8[N] | core u8[F*N]
-  uint64_t* keyA = reinterpret_cast<uint64_t*>(smem_raw);
-  float* S = reinterpret_cast<float*>(keyA + N);
-  int* hist = reinterpret_cast<int*>(S + (size_t)F * N);
-  int* warp_tot = hist + (kMaxGroups + 1) * 256;
-  int* scal = warp_tot + (kMaxGroups + 1) * 32;
-  uint8_t* pool = reinterpret_cast<uint8_t*>(scal + (kMaxGroups + 1) * 4);
-  uint8_t* anchor = pool + N;
-  uint8_t* anycore = anchor + N;
-  uint8_t* core = anycore + N;
+  const int Npad = (N + 3) / 4 * 4;
+  const SelLayout lay = sel_layout(F, N);
+  uint64_t* keyA = reinterpret_cast<uint64_t*>(smem_raw + lay.keyA);
+  float* S = reinterpret_cast<float*>(smem_raw + lay.S);
+  uint32_t* keyM = reinterpret_cast<uint32_t*>(smem_raw + lay.keyM);
+  Scratch sc{reinterpret_cast<int*>(smem_raw + lay.hist), reinterpret_cast<int*>(smem_raw + lay.scal),
+             reinterpret_cast<int*>(smem_raw + lay.warp_tot)};
+  uint8_t* pool = smem_raw + lay.pool;
+  uint8_t* anchor = smem_raw + lay.anchor;
+  uint8_t* anycore = smem_raw + lay.anycore;
+  uint8_t* core = smem_raw + lay.core;  // [F][Npad]
 
-  const int tid = threadIdx.x, b = blockIdx.x;
+  const int tid = threadIdx.x, b = blockIdx.y;
   const float* sg = p.scores + (int64_t)b * F * N;
   for (int i = tid; i < F * N; i += kSelThreads) S[i] = sg[i];
   __syncthreads();
 
-  GroupCtx all{0, kSelThreads, tid, hist, scal, warp_tot};
-
   // candidate pool: top (N_s - K_s) of max_f S(f, j)                                   (Eq. 4)
-  uint32_t* keyM = reinterpret_cast<uint32_t*>(keyA);  // the anchor keys are built later in the same storage
   for (int j = tid; j < N; j += kSelThreads) {
     float m = S[j];
     for (int f = 1; f < F; ++f) m = fmaxf(m, S[f * N + j]);
     keyM[j] = key32(m);
   }
   __syncthreads();
-  radix_select<uint32_t>(all, N, N - p.Ks, [&](int j) { return keyM[j]; }, [](int) { return true; }, pool);
+  radix_select<uint32_t>(sc, N, N - p.Ks, [&](int j) { return keyM[j]; }, [](int) { return true; }, pool);
 
-  // frame-specific core tokens: top K_c of S(f, .) inside the pool                      (Eq. 5)
-  {
-    const int gt = kSelThreads / p.n_groups;
-    const int grp = tid / gt;
-    GroupCtx gc{1 + grp, gt, tid - grp * gt, hist + (1 + grp) * 256, scal + (1 + grp) * 4, warp_tot + (1 + grp) * 32};
-    for (int f = grp; f < F; f += p.n_groups) {
-      const float* Sf = S + (size_t)f * N;
-      radix_select<uint32_t>(gc, N, p.Kc, [&](int j) { return key32(Sf[j]); }, [&](int j) { return pool[j] != 0; },
-                             core + (size_t)f * N);
-    }
+  // frame-specific core tokens of this CTA's frames: top K_c of S(f, .) inside the pool   (Eq. 5)
+  for (int f = rank; f < F; f += C) {
+    const float* Sf = S + (size_t)f * N;
+    radix_select<uint32_t>(sc, N, p.Kc, [&](int j) { return key32(Sf[j]); }, [&](int j) { return pool[j] != 0; },
+                           core + (size_t)f * Npad);
   }
-  __syncthreads();
 
-  // positions that are core in no frame (Eq. 10) and the anchor key mu / (1 + beta CV)   (Eq. 11, Eq. 6)
-  for (int j = tid; j < N; j += kSelThreads) {
-    uint8_t any = 0;
+  // this CTA's share of the anchor keys mu / (1 + beta CV)                               (Eq. 11, Eq. 6)
+  const int share = (N + C - 1) / C;
+  const int j_lo = rank * share, j_hi = min(N, j_lo + share);
+  for (int j = j_lo + tid; j < j_hi; j += kSelThreads) {
     double sum = 0.0;
-    for (int f = 0; f < F; ++f) {
-      any |= core[(size_t)f * N + j];
-      sum = __dadd_rn(sum, (double)S[f * N + j]);
-    }
+    for (int f = 0; f < F; ++f) sum = __dadd_rn(sum, (double)S[f * N + j]);
     const double mu = __ddiv_rn(sum, (double)F);
     double ss = 0.0;
     for (int f = 0; f < F; ++f) {
@@ -239,22 +266,45 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
     }
     const double sd = __dsqrt_rn(__ddiv_rn(ss, (double)F));
     const double cv = (mu == 0.0) ? 0.0 : __ddiv_rn(sd, mu);
-    const double a = __ddiv_rn(mu, __dadd_rn(1.0, __dmul_rn(p.beta, cv)));
-    anycore[j] = any;
-    keyA[j] = key64(a);
+    keyA[j] = key64(__ddiv_rn(mu, __dadd_rn(1.0, __dmul_rn(p.beta, cv))));
   }
   __syncthreads();
-  radix_select<uint64_t>(all, N, p.Ks, [&](int j) { return keyA[j]; }, [&](int j) { return anycore[j] == 0; }, anchor);
 
-  // retained positions ascending, and the maps
+  // exchange through distributed shared memory: my frames' core flags and my anchor keys go to every other CTA
+  if (C > 1) {
+    cluster.sync();  // every CTA of the cluster is resident before its shared memory is written remotely
+    for (int peer = 1; peer < C; ++peer) {
+      const int dst = (rank + peer) % C;
+      uint8_t* rbase = cluster.map_shared_rank(smem_raw, dst);
+      uint64_t* rkeyA = reinterpret_cast<uint64_t*>(rbase + lay.keyA);
+      for (int j = j_lo + tid; j < j_hi; j += kSelThreads) rkeyA[j] = keyA[j];
+      for (int f = rank; f < F; f += C) {
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(core + (size_t)f * Npad);
+        uint32_t* rdst = reinterpret_cast<uint32_t*>(rbase + lay.core + (size_t)f * Npad);
+        for (int w = tid; w < Npad / 4; w += kSelThreads) rdst[w] = src[w];
+      }
+    }
+    cluster.sync();
+  }
+
+  // positions that are core in no frame (Eq. 10), then the shared anchors
+  for (int j = tid; j < N; j += kSelThreads) {
+    uint8_t any = 0;
+    for (int f = 0; f < F; ++f) any |= core[(size_t)f * Npad + j];
+    anycore[j] = any;
+  }
+  __syncthreads();
+  radix_select<uint64_t>(sc, N, p.Ks, [&](int j) { return keyA[j]; }, [&](int j) { return anycore[j] == 0; }, anchor);
+
+  // retained positions ascending, and the maps, for this CTA's frames
   int32_t* sel = p.sel_idx ? p.sel_idx + (int64_t)b * F * K : nullptr;
   int32_t* pm = p.pack_map ? p.pack_map + (int64_t)b * p.Lp : nullptr;
   int32_t* im = p.inv_map ? p.inv_map + (int64_t)b * p.L : nullptr;
   bool bad = false;
-  for (int f = 0; f < F; ++f) {
-    const uint8_t* cf = core + (size_t)f * N;
+  for (int f = rank; f < F; f += C) {
+    const uint8_t* cf = core + (size_t)f * Npad;
     const int cnt = ranked_emit(
-        all, N, [&](int j) { return (cf[j] | anchor[j]) != 0; },
+        sc, N, [&](int j) { return (cf[j] | anchor[j]) != 0; },
         [&](int j, int r) {
           if (r >= 0 && r < K) {
             if (sel) sel[f * K + r] = j;
@@ -264,24 +314,26 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
         });
     bad |= (cnt != K);
   }
-  for (int t = tid; t < p.n_obs; t += kSelThreads) {
+  for (int t = rank * kSelThreads + tid; t < p.n_obs; t += C * kSelThreads) {
     if (pm) pm[t] = t;
     if (im) im[t] = t;
   }
-  for (int t = tid; t < p.H; t += kSelThreads) {
+  for (int t = rank * kSelThreads + tid; t < p.H; t += C * kSelThreads) {
     if (pm) pm[p.n_obs + F * K + t] = p.n_obs + F * N + t;
     if (im) im[p.n_obs + F * N + t] = p.n_obs + F * K + t;
   }
   if (bad && tid == 0) atomicOr(p.status, ST_BAD_COUNT);
 }
 
+int cluster_size(const Dims& d) {
+  int c = 1;
+  while (c * 2 <= d.F && c * 2 <= kMaxCluster) c *= 2;
+  return c;
+}
+
 }  // namespace
 
-size_t select_smem_bytes(const Dims& d) {
-  const size_t N = d.N_s, F = d.F;
-  size_t bytes = N * 8 + F * N * 4 + (size_t)(kMaxGroups + 1) * (256 + 32 + 4) * 4 + 3 * N + F * N;
-  return (bytes + 15) & ~(size_t)15;
-}
+size_t select_smem_bytes(const Dims& d) { return sel_layout(d.F, d.N_s).total; }
 
 cudaError_t select_prepare(const Dims& d) {
   const size_t smem = select_smem_bytes(d);
@@ -291,13 +343,23 @@ cudaError_t select_prepare(const Dims& d) {
 
 cudaError_t launch_select(const Dims& d, const float* scores, int32_t* sel_idx, int32_t* pack_map,
                           int32_t* inv_map, int* status, cudaStream_t st, int* launches) {
-  int groups = 1;
-  while (groups * 2 <= d.F && groups * 2 <= kMaxGroups) groups *= 2;
   SelectParams p{scores, sel_idx, pack_map, inv_map, status, d.n_obs, d.F, d.N_s, d.H,
-                 d.Kc, d.Ks, d.L, d.Lp, groups, (double)d.beta};
+                 d.Kc, d.Ks, d.L, d.Lp, (double)d.beta};
+  const int C = cluster_size(d);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(C, d.B, 1);
+  cfg.blockDim = dim3(kSelThreads, 1, 1);
+  cfg.dynamicSmemBytes = select_smem_bytes(d);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = C;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   ++*launches;
-  select_kernel<<<d.B, kSelThreads, select_smem_bytes(d), st>>>(p);
-  return cudaGetLastError();
+  return cudaLaunchKernelEx(&cfg, select_kernel, p);
 }
 
 }  // namespace swam
