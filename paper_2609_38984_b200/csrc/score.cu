@@ -267,15 +267,18 @@ __device__ __forceinline__ void merge_ms(float& m, float& s, float m2, float s2)
   m = mn;
 }
 
+constexpr int kLseHeads = 4;  // heads per CTA
+
 template <int D>
 __global__ void __launch_bounds__(kLseThreads) lse_partial_bf16_kernel(const LseParams p) {
   constexpr int KB = D / 32;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  uint4* q_frag = reinterpret_cast<uint4*>(smem_raw);                        // [KB][NT][32]
-  float2* wpart = reinterpret_cast<float2*>(q_frag + (size_t)KB * p.NT * 32);  // [8 warps][NT*8]
+  const int n_frag = KB * p.NT * 32;
+  uint4* q_frag = reinterpret_cast<uint4*>(smem_raw);                     // [2][KB][NT][32]
+  float2* wpart = reinterpret_cast<float2*>(q_frag + (size_t)2 * n_frag);  // [8 warps][NT*8]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int chunk = blockIdx.x, b = blockIdx.y;
+  const int chunk = blockIdx.x, h0 = blockIdx.y * kLseHeads, b = blockIdx.z;
   const int64_t tok = (int64_t)p.N_h * D;
   const int gq = lane >> 2, t = lane & 3;
   const int r0 = chunk * kLseKeys + warp * 16 + gq, r1 = r0 + 8;
@@ -283,50 +286,70 @@ __global__ void __launch_bounds__(kLseThreads) lse_partial_bf16_kernel(const Lse
   const __nv_bfloat16* k0 = p.k + ((int64_t)b * p.L + (v0 ? r0 : 0)) * tok + t * 8;
   const __nv_bfloat16* k1 = p.k + ((int64_t)b * p.L + (v1 ? r1 : 0)) * tok + t * 8;
   const int64_t act0 = (int64_t)p.L - p.H;
-  const int n_frag = KB * p.NT * 32;
   const uint4 zero = make_uint4(0, 0, 0, 0);
 
-  for (int h = 0; h < p.N_h; ++h) {
-    __syncthreads();  // previous head's fragments and partials are no longer read
+  auto stage_q = [&](int h, int buf) {  // this head's H queries as B fragments, asynchronously
     for (int i = tid; i < n_frag; i += kLseThreads) {
       const int ln = i & 31;
       const int nt = (i >> 5) % p.NT;
       const int kb = (i >> 5) / p.NT;
       const int n = nt * 8 + (ln >> 2);
-      uint4 val = zero;
-      if (n < p.H)
-        val = *reinterpret_cast<const uint4*>(p.q + ((int64_t)b * p.L + act0 + n) * tok + (int64_t)h * D + kb * 32 +
-                                              (ln & 3) * 8);
-      q_frag[i] = val;
+      const bool in = n < p.H;
+      const __nv_bfloat16* src = p.q + ((int64_t)b * p.L + act0 + (in ? n : 0)) * tok + (int64_t)h * D + kb * 32 + (ln & 3) * 8;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                   ::"r"((uint32_t)__cvta_generic_to_shared(q_frag + (size_t)buf * n_frag + i)), "l"(src), "r"(in ? 16 : 0)
+                   : "memory");
     }
-    uint4 a0[KB], a1[KB];
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  uint4 a0[2][KB], a1[2][KB];
+  auto load_k = [&](int h, int buf) {
 #pragma unroll
     for (int kb = 0; kb < KB; ++kb) {
-      a0[kb] = v0 ? ldg_stream(k0 + (int64_t)h * D + kb * 32) : zero;
-      a1[kb] = v1 ? ldg_stream(k1 + (int64_t)h * D + kb * 32) : zero;
+      a0[buf][kb] = v0 ? ldg_stream(k0 + (int64_t)h * D + kb * 32) : zero;
+      a1[buf][kb] = v1 ? ldg_stream(k1 + (int64_t)h * D + kb * 32) : zero;
+    }
+  };
+
+  stage_q(h0, 0);
+  load_k(h0, 0);
+#pragma unroll
+  for (int hi = 0; hi < kLseHeads; ++hi) {
+    const int h = h0 + hi;
+    if (h >= p.N_h) break;
+    const bool more = (hi + 1 < kLseHeads) && (h + 1 < p.N_h);
+    if (more) {
+      stage_q(h + 1, (hi + 1) & 1);
+      load_k(h + 1, (hi + 1) & 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
     __syncthreads();
+    const uint4* qf = q_frag + (size_t)(hi & 1) * n_frag;
     for (int nt = 0; nt < p.NT; ++nt) {
       float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int kb = 0; kb < KB; ++kb) {
-        const uint4 bq = q_frag[(kb * p.NT + nt) * 32 + lane];
-        mma_bf16_16816(c, a0[kb].x, a1[kb].x, a0[kb].y, a1[kb].y, bq.x, bq.y);
-        mma_bf16_16816(c, a0[kb].z, a1[kb].z, a0[kb].w, a1[kb].w, bq.z, bq.w);
+        const uint4 bq = qf[(kb * p.NT + nt) * 32 + lane];
+        mma_bf16_16816(c, a0[hi & 1][kb].x, a1[hi & 1][kb].x, a0[hi & 1][kb].y, a1[hi & 1][kb].y, bq.x, bq.y);
+        mma_bf16_16816(c, a0[hi & 1][kb].z, a1[hi & 1][kb].z, a0[hi & 1][kb].w, a1[hi & 1][kb].w, bq.z, bq.w);
       }
-      // columns 2t, 2t+1; rows gq (c0, c1) and gq+8 (c2, c3)
-      float x00 = v0 ? c[0] * p.scale_log2 : -INFINITY, x01 = v0 ? c[1] * p.scale_log2 : -INFINITY;
-      float x10 = v1 ? c[2] * p.scale_log2 : -INFINITY, x11 = v1 ? c[3] * p.scale_log2 : -INFINITY;
-      float m0 = x00, s0 = (x00 == -INFINITY) ? 0.f : 1.f;
-      float m1 = x01, s1 = (x01 == -INFINITY) ? 0.f : 1.f;
-      merge_ms(m0, s0, x10, (x10 == -INFINITY) ? 0.f : 1.f);
-      merge_ms(m1, s1, x11, (x11 == -INFINITY) ? 0.f : 1.f);
+      // columns 2t, 2t+1; rows gq (c0, c1) and gq+8 (c2, c3): column max over the warp's 16 keys, then the sum
+      const float x00 = v0 ? c[0] * p.scale_log2 : -INFINITY, x01 = v0 ? c[1] * p.scale_log2 : -INFINITY;
+      const float x10 = v1 ? c[2] * p.scale_log2 : -INFINITY, x11 = v1 ? c[3] * p.scale_log2 : -INFINITY;
+      float m0 = fmaxf(x00, x10), m1 = fmaxf(x01, x11);
 #pragma unroll
       for (int o = 4; o < 32; o <<= 1) {
-        const float om0 = __shfl_xor_sync(0xffffffffu, m0, o), os0 = __shfl_xor_sync(0xffffffffu, s0, o);
-        const float om1 = __shfl_xor_sync(0xffffffffu, m1, o), os1 = __shfl_xor_sync(0xffffffffu, s1, o);
-        merge_ms(m0, s0, om0, os0);
-        merge_ms(m1, s1, om1, os1);
+        m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, o));
+        m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o));
+      }
+      float s0 = (m0 == -INFINITY) ? 0.f : exp2f(x00 - m0) + exp2f(x10 - m0);
+      float s1 = (m1 == -INFINITY) ? 0.f : exp2f(x01 - m1) + exp2f(x11 - m1);
+#pragma unroll
+      for (int o = 4; o < 32; o <<= 1) {
+        s0 += __shfl_xor_sync(0xffffffffu, s0, o);
+        s1 += __shfl_xor_sync(0xffffffffu, s1, o);
       }
       if (gq == 0) {
         wpart[warp * p.NT * 8 + nt * 8 + 2 * t] = make_float2(m0, s0);
@@ -335,27 +358,34 @@ __global__ void __launch_bounds__(kLseThreads) lse_partial_bf16_kernel(const Lse
     }
     __syncthreads();
     for (int n = tid; n < p.H; n += kLseThreads) {
-      float m = -INFINITY, s = 0.f;
+      float m = -INFINITY, sacc = 0.f;
       for (int w = 0; w < 8; ++w) {
         const float2 ws = wpart[w * p.NT * 8 + n];
-        merge_ms(m, s, ws.x, ws.y);
+        merge_ms(m, sacc, ws.x, ws.y);
       }
-      p.partial[(((int64_t)b * p.n_chunks + chunk) * p.N_h + h) * p.H + n] = make_float2(m, s);
+      p.partial[(((int64_t)b * p.n_chunks + chunk) * p.N_h + h) * p.H + n] = make_float2(m, sacc);
     }
+    // the next head's barrier (after its wait) orders these reads of wpart before its writes
   }
 }
 
-// merges the per-chunk partials: lambda = ln2 * (m + log2 s)
-__global__ void lse_merge_kernel(const float2* partial, float* lse, int n_chunks, int N_h, int H) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+// merges the per-chunk partials: lambda = ln2 * (m + log2 s); one warp per (sample, head, query)
+__global__ void __launch_bounds__(256) lse_merge_kernel(const float2* partial, float* lse, int n_chunks, int N_h, int H) {
+  const int lane = threadIdx.x & 31;
+  const int i = blockIdx.x * 8 + (threadIdx.x >> 5);
   const int b = blockIdx.y;
   if (i >= N_h * H) return;
   float m = -INFINITY, s = 0.f;
-  for (int c = 0; c < n_chunks; ++c) {
+  for (int c = lane; c < n_chunks; c += 32) {
     const float2 ms = partial[((int64_t)b * n_chunks + c) * N_h * H + i];
     merge_ms(m, s, ms.x, ms.y);
   }
-  lse[(int64_t)b * N_h * H + i] = (m + log2f(s)) * 0.6931471805599453f;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
+    merge_ms(m, s, om, os);
+  }
+  if (lane == 0) lse[(int64_t)b * N_h * H + i] = (m + log2f(s)) * 0.6931471805599453f;
 }
 
 // fp32: one CTA per (b, h, i); threads stride over keys with a running (max, sum) in natural-log units
@@ -499,9 +529,9 @@ cudaError_t launch_action_lse(const Dims& d, const void* q, const void* k, float
   const int NT = (d.H + 7) / 8;
   LseParams p{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (float2*)scratch, d.H, d.N_h, d.L, n_chunks, NT,
               d.scale * kLog2e};
-  const size_t smem = (size_t)(d.D / 32) * NT * 32 * sizeof(uint4) + (size_t)8 * NT * 8 * sizeof(float2);
+  const size_t smem = (size_t)2 * (d.D / 32) * NT * 32 * sizeof(uint4) + (size_t)8 * NT * 8 * sizeof(float2);
   if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
-  dim3 grid(n_chunks, d.B);
+  dim3 grid(n_chunks, (d.N_h + kLseHeads - 1) / kLseHeads, d.B);
   cudaError_t e = cudaSuccess;
   *launches += 2;
   switch (d.D) {
@@ -522,8 +552,8 @@ cudaError_t launch_action_lse(const Dims& d, const void* q, const void* k, float
   if (e != cudaSuccess) return e;
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  dim3 g2((d.N_h * d.H + 127) / 128, d.B);
-  lse_merge_kernel<<<g2, 128, 0, st>>>((const float2*)scratch, lse, n_chunks, d.N_h, d.H);
+  dim3 g2((d.N_h * d.H + 7) / 8, d.B);
+  lse_merge_kernel<<<g2, 256, 0, st>>>((const float2*)scratch, lse, n_chunks, d.N_h, d.H);
   return cudaGetLastError();
 }
 
