@@ -153,8 +153,13 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 struct TcParams {
   float* lse;
   int* status;
+  float* partial;      // split items: [slot][2 tiles][128 rows][D + 4]: unnormalised O, then reference max and sum
   int lse_row0, lse_rows;
   int n, N_h;
+  int pairs;           // query tile pairs per (sample, head)
+  int n_whole;         // work items that run over all keys and write the output themselves
+  int splits;          // pieces per split item (0 when nothing is split)
+  int tiles_per_split; // key tiles per piece
   float scale_log2;
 };
 
@@ -196,9 +201,23 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::kSmemData + 8 * (6 + 4 * ST) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int h = blockIdx.y, b = blockIdx.z;
-  const int row0 = blockIdx.x * 2 * kTile;
-  const int n_tiles = (p.n + kTile - 1) / kTile;
+  // work item = (sample, head, query tile pair), pair fastest.  Items below n_whole walk over all keys; the few items
+  // of the last, partly filled wave are cut into `splits` pieces over the keys so that they spread over idle SMs,
+  // each piece leaving an unnormalised partial result for the combine kernel.
+  int item = blockIdx.x, kv_begin = 0;
+  const int all_tiles = (p.n + kTile - 1) / kTile;
+  int kv_end = all_tiles;
+  int slot = -1;
+  if (item >= p.n_whole) {
+    slot = item - p.n_whole;
+    item = p.n_whole + slot / p.splits;
+    kv_begin = (slot % p.splits) * p.tiles_per_split;
+    kv_end = min(all_tiles, kv_begin + p.tiles_per_split);
+  }
+  const int pair = item % p.pairs;
+  const int h = (item / p.pairs) % p.N_h, b = item / (p.pairs * p.N_h);
+  const int row0 = pair * 2 * kTile;
+  const int n_tiles = kv_end - kv_begin;  // >= 1 by construction
 
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
@@ -251,12 +270,12 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (!ok) break;
         mbar_expect_tx(bar_k_full(st), C::kTileBytes);
         for (int db = 0; db < C::DB; ++db)
-          tma_load_4d(sK + st * C::kTileBytes + db * C::kSubTile, &map_k, bar_k_full(st), db * 64, j * kTile, h, b);
+          tma_load_4d(sK + st * C::kTileBytes + db * C::kSubTile, &map_k, bar_k_full(st), db * 64, (kv_begin + j) * kTile, h, b);
         ok = mbar_wait(bar_v_empty(st), par, abort_flag);
         if (!ok) break;
         mbar_expect_tx(bar_v_full(st), C::kTileBytes);
         for (int db = 0; db < C::DB; ++db)
-          tma_load_4d(sV + st * C::kTileBytes + db * C::kSubTile, &map_v, bar_v_full(st), db * 64, j * kTile, h, b);
+          tma_load_4d(sV + st * C::kTileBytes + db * C::kSubTile, &map_v, bar_v_full(st), db * 64, (kv_begin + j) * kTile, h, b);
       }
     }
    } else if (warp == 8) {
@@ -330,7 +349,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 #pragma unroll
       for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<float(*)[32]>(&sv[c * 32]));
       tmem_ld_wait();
-      const int valid = p.n - j * kTile;  // keys of this tile inside the sequence
+      const int valid = p.n - (kv_begin + j) * kTile;  // keys of this tile inside the sequence
       if (valid < kTile) {
 #pragma unroll
         for (int c = 0; c < kTile; ++c)
@@ -379,8 +398,27 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       tc_fence_before();
       mbar_arrive(bar_p_full(s));
     }
-    // epilogue: O / l -> bf16 -> swizzled staging in the (finished) Q tile -> TMA store; rows beyond n are clipped
+    // epilogue
     if (ok) ok = mbar_wait(bar_o_final, 0, abort_flag);
+    if (slot >= 0) {
+      // a piece of a split item: unnormalised O, reference max and sum go to scratch; the combine kernel finishes
+      if (ok) {
+        tc_fence_after();
+        float* dst = p.partial + (((size_t)slot * 2 + s) * kTile + r) * (D + 4);
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          float ov[32];
+          tmem_ld32(tO + c * 32, ov);
+          tmem_ld_wait();
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4)
+            *reinterpret_cast<float4*>(dst + c * 32 + q4 * 4) = make_float4(ov[q4 * 4], ov[q4 * 4 + 1], ov[q4 * 4 + 2], ov[q4 * 4 + 3]);
+        }
+        dst[D] = m_used;
+        dst[D + 1] = l_run;
+      }
+    } else {
+    // O / l -> bf16 -> swizzled staging in the (finished) Q tile -> TMA store; rows beyond n are clipped
     if (ok) {
       tc_fence_after();
       const float inv = 1.f / l_run;
@@ -413,6 +451,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tma_store_4d(&map_o, sQ + s * C::kTileBytes + db * C::kSubTile, db * 64, row0 + s * kTile, h, b);
       tma_store_commit_wait();
     }
+    }
   }
 
   tc_fence_before();
@@ -422,6 +461,43 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
   }
+}
+
+// Merges the pieces of the split items: out = sum_i 2^(m_i - m) O_i / sum_i 2^(m_i - m) l_i, one warp per query row.
+struct CombineParams {
+  const float* partial;
+  __nv_bfloat16* out;
+  float* lse;
+  int lse_row0, lse_rows;
+  int n, N_h, D, pairs, n_whole, splits, n_split_items;
+};
+
+__global__ void __launch_bounds__(256) attn_combine_kernel(const CombineParams p) {
+  const int lane = threadIdx.x & 31;
+  const int row_id = blockIdx.x * 8 + (threadIdx.x >> 5);  // (split item, tile, row)
+  if (row_id >= p.n_split_items * 2 * kTile) return;
+  const int si = row_id / (2 * kTile), tr = row_id % (2 * kTile);
+  const int item = p.n_whole + si;
+  const int pair = item % p.pairs, h = (item / p.pairs) % p.N_h, b = item / (p.pairs * p.N_h);
+  const int row = pair * 2 * kTile + tr;
+  if (row >= p.n) return;
+  const int stride = p.D + 4;
+  const float* base = p.partial + ((size_t)si * p.splits * 2 * kTile + tr) * stride;  // piece 0 of this row
+  const size_t piece = (size_t)2 * kTile * stride;
+  float m = -INFINITY;
+  for (int i = 0; i < p.splits; ++i) m = fmaxf(m, base[i * piece + p.D]);
+  float l = 0.f;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};  // D <= 128: four columns per lane
+  for (int i = 0; i < p.splits; ++i) {
+    const float w = exp2f(base[i * piece + p.D] - m);
+    l += w * base[i * piece + p.D + 1];
+    for (int c = 0; c < p.D / 32; ++c) acc[c] += w * base[i * piece + c * 32 + lane];
+  }
+  const float inv = 1.f / l;
+  __nv_bfloat16* o = p.out + (((int64_t)b * p.n + row) * p.N_h + h) * p.D;
+  for (int c = 0; c < p.D / 32; ++c) o[c * 32 + lane] = __float2bfloat16(acc[c] * inv);
+  if (p.lse && lane == 0 && row >= p.lse_row0 && row < p.lse_row0 + p.lse_rows)
+    p.lse[((int64_t)b * p.N_h + h) * p.lse_rows + (row - p.lse_row0)] = (m + log2f(l)) * 0.6931471805599453f;
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -456,27 +532,64 @@ bool make_map(CUtensorMap* map, const void* ptr, int B, int n, int N_h, int D) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+int sm_count_tc() {
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+  }
+  return sms;
+}
+
 template <int D>
-cudaError_t launch_tc_d(const AttnArgs& a, int* status, cudaStream_t st) {
+cudaError_t launch_tc_d(const AttnArgs& a, int* status, float* partial, size_t partial_bytes, cudaStream_t st, int* launches) {
   CUtensorMap mq, mk, mv, mo;
   if (!make_map(&mq, a.q, a.B, a.n, a.N_h, D) || !make_map(&mk, a.k, a.B, a.n, a.N_h, D) ||
       !make_map(&mv, a.v, a.B, a.n, a.N_h, D) || !make_map(&mo, a.out, a.B, a.n, a.N_h, D))
     return cudaErrorInvalidValue;
   cudaError_t e = cudaFuncSetAttribute(attn_bf16_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<D>::kSmemBytes);
   if (e != cudaSuccess) return e;
-  TcParams p{a.lse, status, a.lse_row0, a.lse_rows, a.n, a.N_h, a.scale * kLog2e};
-  dim3 grid((a.n + 2 * kTile - 1) / (2 * kTile), a.N_h, a.B);
+  const int pairs = (a.n + 2 * kTile - 1) / (2 * kTile);
+  const int items = pairs * a.N_h * a.B;
+  const int n_tiles = (a.n + kTile - 1) / kTile;
+  const int sms = sm_count_tc();
+  // one CTA per SM: the items beyond the last full wave are cut over the keys into pieces that fill the idle SMs
+  int rem = items % sms, splits = 0, per = n_tiles;
+  if (items > sms && rem > 0 && rem <= sms / 2 && n_tiles >= 4) {
+    int want = sms / rem;
+    if (want > 16) want = 16;
+    if (want > n_tiles / 2) want = n_tiles / 2;
+    per = (n_tiles + want - 1) / want;
+    splits = (n_tiles + per - 1) / per;
+    const size_t need = (size_t)rem * splits * 2 * kTile * (D + 4) * sizeof(float);
+    if (splits < 2 || !partial || need > partial_bytes) { splits = 0; per = n_tiles; }
+  }
+  const int n_whole = splits ? items - rem : items;
+  TcParams p{a.lse, status, partial, a.lse_row0, a.lse_rows, a.n, a.N_h, pairs, n_whole, splits, per, a.scale * kLog2e};
+  const int grid = n_whole + (splits ? rem * splits : 0);
+  ++*launches;
   attn_bf16_tc_kernel<D><<<grid, kThreadsTc, TcCfg<D>::kSmemBytes, st>>>(mq, mk, mv, mo, p);
+  e = cudaGetLastError();
+  if (e != cudaSuccess || !splits) return e;
+  CombineParams c{partial, (__nv_bfloat16*)a.out, a.lse, a.lse_row0, a.lse_rows, a.n, a.N_h, D, pairs, n_whole, splits, rem};
+  ++*launches;
+  attn_combine_kernel<<<(rem * 2 * kTile + 7) / 8, 256, 0, st>>>(c);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, cudaStream_t st, int* launches) {
-  ++*launches;
+size_t attn_tc_scratch_bytes(int D) {
+  // room for one piece per SM (the split pieces never outnumber the SMs); 160 covers the SM count of this part
+  return (size_t)160 * 2 * kTile * (D + 4) * sizeof(float);
+}
+
+cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, void* scratch, size_t scratch_bytes, cudaStream_t st,
+                                int* launches) {
   switch (a.D) {
-    case 64: return launch_tc_d<64>(a, status, st);
-    case 128: return launch_tc_d<128>(a, status, st);
+    case 64: return launch_tc_d<64>(a, status, (float*)scratch, scratch_bytes, st, launches);
+    case 128: return launch_tc_d<128>(a, status, (float*)scratch, scratch_bytes, st, launches);
     default: return cudaErrorInvalidConfiguration;
   }
 }

@@ -18,7 +18,7 @@ struct swam_ctx {
   unsigned char* ws;
   size_t ws_bytes;
   size_t off_status, off_scores, off_quality, off_lse, off_sel, off_pack, off_inv, off_scratch, off_qp, off_kp,
-      off_vp, off_op, ws_need;
+      off_vp, off_op, off_attn, attn_scratch, ws_need;
   bool has_selection;
   int attn_variant;  // SWAM_ATTN_AUTO | SWAM_ATTN_WARP_MMA
   // host-io staging (device)
@@ -60,7 +60,7 @@ int run_attention(swam_ctx* c, const void* q, const void* k, const void* v, int 
     e = launch_attn_f32(a, st, &c->launches_i);
   } else if (c->d.D >= 64 && c->attn_variant == SWAM_ATTN_AUTO) {
     if (!c->ws) return fail(c, SWAM_ERR_WORKSPACE, "no workspace bound");
-    e = launch_attn_bf16_tc(a, (int*)(c->ws + c->off_status), st, &c->launches_i);
+    e = launch_attn_bf16_tc(a, (int*)(c->ws + c->off_status), c->ws + c->off_attn, c->attn_scratch, st, &c->launches_i);
   } else {
     e = launch_attn_bf16_mma(a, st, &c->launches_i);
   }
@@ -147,6 +147,8 @@ int swam_create(const swam_shape* s, swam_ctx** out_ctx) {
   c->off_kp = put(packed_bytes(d));
   c->off_vp = put(packed_bytes(d));
   c->off_op = put(packed_bytes(d));
+  c->attn_scratch = (d.dtype == SWAM_BF16 && d.D >= 64) ? attn_tc_scratch_bytes(d.D) : 0;
+  c->off_attn = put(c->attn_scratch);
   c->ws_need = off;
   c->io_need = 4 * align_up(full_bytes(d), 256);
   *out_ctx = c;

@@ -67,6 +67,9 @@ cudaError_t attn_prepare(int D, int dtype);
 cudaError_t launch_attn_f32(const AttnArgs& a, cudaStream_t st, int* launches);
 cudaError_t launch_attn_bf16_mma(const AttnArgs& a, cudaStream_t st, int* launches);
 // tcgen05 / TMEM / TMA kernel, head_dim 64 or 128; bounded waits report through the status word
-cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, cudaStream_t st, int* launches);
+// scratch: room for the partial results of the key-split tail items (attn_tc_scratch_bytes), may be nullptr
+size_t attn_tc_scratch_bytes(int D);
+cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, void* scratch, size_t scratch_bytes, cudaStream_t st,
+                                int* launches);
 
 }  // namespace swam
