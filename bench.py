@@ -237,12 +237,20 @@ def bench_swam(args):
         fut = wl.n_frames * wl.n_spatial
         reps = max(3, min(args.steps, 20))
 
-        def stage(make):
-            return per_launch_us([make(i) for i in range(N_ROT)], reps)
+        stage_clocks = {}
+
+        def stage(make, clock_key=None):
+            smp = ClockSampler(local_rank, period_s=0.005) if clock_key else None
+            if smp:
+                smp.start()
+            us = per_launch_us([make(i) for i in range(N_ROT)], reps)
+            if smp:
+                stage_clocks[clock_key] = smp.stop()
+            return us
 
         stage_us = {
             "attn_dense": stage(lambda i: lambda: lib.swam_sparse_attn(ctx.ctx, P(rot[i]["q"]), P(rot[i]["k"]), P(rot[i]["v"]), L,
-                                                                       P(outs[i]), None, S())),
+                                                                       P(outs[i]), None, S()), "attn_dense"),
             "score": stage(lambda i: lambda: lib.swam_score(ctx.ctx, P(rot[i]["q"]), P(rot[i]["k"]), P(lse_act), P(scores[i]),
                                                             None, S())),
             "score_with_lse": stage(lambda i: lambda: lib.swam_score(ctx.ctx, P(rot[i]["q"]), P(rot[i]["k"]), None,
@@ -310,7 +318,7 @@ def bench_swam(args):
                        "parallelism": f"sample-sharded x{world}"},
             "sparse_step_us": stages["sparse_step"]["us"], "full_step_us": stages["full_step"]["us"],
             "roofline": roofline, "stages": stages, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
-            "clocks": clocks, "impl": "swam",
+            "clocks": clocks, "stage_clocks": stage_clocks, "impl": "swam",
         }
     sd.barrier(device)
     sd.finalize()

@@ -150,7 +150,16 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   return d;
 }
 
+#ifdef SWAM_TC_TRACE
+#define TRACE(slot_, idx_) do { if (blockIdx.x == 0 && p.trace) p.trace[(slot_) * 4096 + (idx_)] = clock64(); } while (0)
+#else
+#define TRACE(slot_, idx_) do { } while (0)
+#endif
+
 struct TcParams {
+#ifdef SWAM_TC_TRACE
+  long long* trace;
+#endif
   float* lse;
   int* status;
   float* partial;      // split items: [slot][2 tiles][128 rows][D + 4]: unnormalised O, then reference max and sum
@@ -313,16 +322,20 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const uint32_t par_full = (j / ST) & 1, par_next = ((j + 1) / ST) & 1;
         ok = mbar_wait(bar_v_full(st), par_full, abort_flag);
         for (int s = 0; s < 2 && ok; ++s) {
+          TRACE(2, (j * 2 + s) * 4 + 0);
           ok = mbar_wait(bar_p_full(s), j & 1, abort_flag);
           if (!ok) break;
+          TRACE(2, (j * 2 + s) * 4 + 1);
           tc_fence_after();
           issue_pv(s, st, j > 0);
+          TRACE(2, (j * 2 + s) * 4 + 2);
           if (j + 1 < n_tiles) {
             if (s == 0) ok = mbar_wait(bar_k_full(st_next), par_next, abort_flag);
             if (!ok) break;
             tc_fence_after();
             issue_qk(s, st_next);
             tc_commit(bar_s_full(s));
+            TRACE(2, (j * 2 + s) * 4 + 3);
           }
         }
         if (!ok) break;
@@ -342,32 +355,62 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     float m_used = -INFINITY, l_run = 0.f;
     bool ok = true;
     for (int j = 0; j < n_tiles; ++j) {
+      if (r == 0) TRACE(s, j * 8 + 0);
       ok = mbar_wait(bar_s_full(s), j & 1, abort_flag);
       if (!ok) break;
+      if (r == 0) TRACE(s, j * 8 + 1);
       tc_fence_after();
       float sv[kTile];
 #pragma unroll
       for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<float(*)[32]>(&sv[c * 32]));
       tmem_ld_wait();
+      if (r == 0) TRACE(s, j * 8 + 2);
       const int valid = p.n - (kv_begin + j) * kTile;  // keys of this tile inside the sequence
       if (valid < kTile) {
 #pragma unroll
         for (int c = 0; c < kTile; ++c)
           if (c >= valid) sv[c] = -INFINITY;
       }
-      float mx = sv[0];
-#pragma unroll
-      for (int c = 1; c < kTile; ++c) mx = fmaxf(mx, sv[c]);
-      mx *= p.scale_log2;
-      // lazy rescale: only when some row of this warp outgrew its reference maximum by more than the threshold
-      const bool grow = mx > m_used + kRescaleThreshold;
       if (j == 0) {
-        m_used = mx;
-      } else if (__any_sync(0xffffffffu, grow)) {
-        const float m_new = fmaxf(m_used, mx);
-        const float f = ex2(m_used - m_new);
+        // the first tile fixes the reference maximum of the row (tree of independent partial maxima)
+        float m8[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) m8[i] = sv[i];
+#pragma unroll
+        for (int c = 8; c < kTile; c += 8) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) m8[i] = fmaxf(m8[i], sv[c + i]);
+        }
+        m_used = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])), fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7]))) *
+                 p.scale_log2;
+      }
+      // One pass: exponentials against the current reference maximum, with the row's own maximum tracked on the
+      // side.  Only if some row of the warp outgrew its reference by more than the threshold (rare after the first
+      // tiles) is the reference raised, O rescaled and the pass repeated; the result is exact either way.
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const float t0 = fmaf(sv[c * 32 + 2 * i], p.scale_log2, -m_used);
+          const float t1 = fmaf(sv[c * 32 + 2 * i + 1], p.scale_log2, -m_used);
+          mx4[i & 3] = fmaxf(mx4[i & 3], fmaxf(t0, t1));
+          const float p0 = ex2(t0), p1 = ex2(t1);
+          sum4[i & 3] += p0 + p1;
+          pk[i] = pack_bf16x2(p0, p1);
+        }
+        tmem_st16(tS + c * 16, pk);
+      }
+      float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+      const float t_max = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      if (__any_sync(0xffffffffu, t_max > kRescaleThreshold)) {
+        const float delta = fmaxf(t_max, 0.f);
+        const float f = ex2(-delta);
+        m_used += delta;
         l_run *= f;
-        m_used = m_new;
+        tmem_st_wait();
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
           float ov[32];
@@ -378,25 +421,26 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           for (int i = 0; i < 32; ++i) ou[i] = __float_as_uint(ov[i] * f);
           tmem_st32(tO + c * 32, ou);
         }
-        tmem_st_wait();
-      }
-      float sum = 0.f;
+        sum = 0.f;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t pk[16];
+        for (int c = 0; c < 4; ++c) {
+          uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const float p0 = ex2(fmaf(sv[c * 32 + 2 * i], p.scale_log2, -m_used));
-          const float p1 = ex2(fmaf(sv[c * 32 + 2 * i + 1], p.scale_log2, -m_used));
-          sum += p0 + p1;
-          pk[i] = pack_bf16x2(p0, p1);
+          for (int i = 0; i < 16; ++i) {
+            const float p0 = ex2(fmaf(sv[c * 32 + 2 * i], p.scale_log2, -m_used));
+            const float p1 = ex2(fmaf(sv[c * 32 + 2 * i + 1], p.scale_log2, -m_used));
+            sum += p0 + p1;
+            pk[i] = pack_bf16x2(p0, p1);
+          }
+          tmem_st16(tS + c * 16, pk);
         }
-        tmem_st16(tS + c * 16, pk);
       }
       l_run += sum;
+      if (r == 0) TRACE(s, j * 8 + 3);
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(bar_p_full(s));
+      if (r == 0) TRACE(s, j * 8 + 4);
     }
     // epilogue
     if (ok) ok = mbar_wait(bar_o_final, 0, abort_flag);
@@ -532,6 +576,14 @@ bool make_map(CUtensorMap* map, const void* ptr, int B, int n, int N_h, int D) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+#ifdef SWAM_TC_TRACE
+void* g_trace = nullptr;
+void* partial_trace_buffer() {
+  if (!g_trace) { cudaMalloc(&g_trace, 3 * 4096 * 8); cudaMemset(g_trace, 0, 3 * 4096 * 8); }
+  return g_trace;
+}
+#endif
+
 int sm_count_tc() {
   static int sms = 0;
   if (!sms) {
@@ -566,7 +618,11 @@ cudaError_t launch_tc_d(const AttnArgs& a, int* status, float* partial, size_t p
     if (splits < 2 || !partial || need > partial_bytes) { splits = 0; per = n_tiles; }
   }
   const int n_whole = splits ? items - rem : items;
-  TcParams p{a.lse, status, partial, a.lse_row0, a.lse_rows, a.n, a.N_h, pairs, n_whole, splits, per, a.scale * kLog2e};
+  TcParams p{
+#ifdef SWAM_TC_TRACE
+      (long long*)partial_trace_buffer(),
+#endif
+      a.lse, status, partial, a.lse_row0, a.lse_rows, a.n, a.N_h, pairs, n_whole, splits, per, a.scale * kLog2e};
   const int grid = n_whole + (splits ? rem * splits : 0);
   ++*launches;
   attn_bf16_tc_kernel<D><<<grid, kThreadsTc, TcCfg<D>::kSmemBytes, st>>>(mq, mk, mv, mo, p);
@@ -579,6 +635,10 @@ cudaError_t launch_tc_d(const AttnArgs& a, int* status, float* partial, size_t p
 }
 
 }  // namespace
+
+#ifdef SWAM_TC_TRACE
+extern "C" void swam_debug_trace(long long* host) { cudaMemcpy(host, g_trace, 3 * 4096 * 8, cudaMemcpyDeviceToHost); }
+#endif
 
 size_t attn_tc_scratch_bytes(int D) {
   // room for one piece per SM (the split pieces never outnumber the SMs); 160 covers the SM count of this part
