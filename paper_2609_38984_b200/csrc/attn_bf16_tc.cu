@@ -132,6 +132,25 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
+// packed pairs of fp32 (one instruction for two elements)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -387,25 +406,36 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       // One pass: exponentials against the current reference maximum, with the row's own maximum tracked on the
       // side.  Only if some row of the warp outgrew its reference by more than the threshold (rare after the first
       // tiles) is the reference raised, O rescaled and the pass repeated; the result is exact either way.
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      // packed fp32 pairs halve the FMA-pipe instruction count; growth of the row maximum shows up in the tile's sum
+      // (an exponent above the threshold pushes the sum beyond 2^threshold), so no per-element maximum is kept
+      const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), negm2 = pack2(-m_used, -m_used);
+      uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t pk[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-          const float t0 = fmaf(sv[c * 32 + 2 * i], p.scale_log2, -m_used);
-          const float t1 = fmaf(sv[c * 32 + 2 * i + 1], p.scale_log2, -m_used);
-          mx4[i & 3] = fmaxf(mx4[i & 3], fmaxf(t0, t1));
+          float t0, t1;
+          unpack2(fma2(pack2(sv[c * 32 + 2 * i], sv[c * 32 + 2 * i + 1]), scale2, negm2), t0, t1);
           const float p0 = ex2(t0), p1 = ex2(t1);
-          sum4[i & 3] += p0 + p1;
+          acc2[i & 3] = add2(acc2[i & 3], pack2(p0, p1));
           pk[i] = pack_bf16x2(p0, p1);
         }
         tmem_st16(tS + c * 16, pk);
       }
-      float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-      const float t_max = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      if (__any_sync(0xffffffffu, t_max > kRescaleThreshold)) {
+      float sum;
+      {
+        float a0, a1;
+        unpack2(add2(add2(acc2[0], acc2[1]), add2(acc2[2], acc2[3])), a0, a1);
+        sum = a0 + a1;
+      }
+      const bool grew = !(sum <= 256.f * 128.f);  // also catches inf and NaN
+      if (__any_sync(0xffffffffu, grew)) {
+        // rare: the row's true maximum relative to the reference
+        float mraw = sv[0];
+#pragma unroll
+        for (int c = 1; c < kTile; ++c) mraw = fmaxf(mraw, sv[c]);
+        const float t_max = fmaf(mraw, p.scale_log2, -m_used);
         const float delta = fmaxf(t_max, 0.f);
         const float f = ex2(-delta);
         m_used += delta;
