@@ -278,11 +278,11 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   // register budget: the softmax warpgroups hold a whole S row per thread, the third warpgroup (MMA issuer, TMA
   // producer, two idle warps) needs almost nothing
   // (setmaxnreg is a warpgroup-wide instruction: all four warps of a warpgroup execute the same one.  The kernel
-  // starts with 168 registers per thread (384 threads, one CTA per SM); lowering the third warpgroup to 64 releases
-  // 104 x 128 = 13312 registers, and raising the two softmax warpgroups to 216 takes 48 x 256 = 12288 of them.  An
+  // starts with 168 registers per thread (384 threads, one CTA per SM); lowering the third warpgroup to 48 releases
+  // 120 x 128 = 15360 registers, and raising the two softmax warpgroups to 224 takes 56 x 256 = 14336 of them.  An
   // increase beyond what was released would wait forever.)
   if (warp >= 8) {
-   asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+   asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
    if (warp == 9) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -365,7 +365,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     }
    }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
     // ------------------------------------------------------------------ softmax warps: one thread per query row
     const int s = warp >> 2;                 // query tile of this warpgroup
     const int r = (warp & 3) * 32 + lane;    // row inside the tile == TMEM lane
@@ -546,7 +546,9 @@ struct CombineParams {
   int n, N_h, D, pairs, n_whole, splits, n_split_items;
 };
 
+template <int D>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const CombineParams p) {
+  constexpr int CPL = D / 32;  // output columns per lane
   const int lane = threadIdx.x & 31;
   const int row_id = blockIdx.x * 8 + (threadIdx.x >> 5);  // (split item, tile, row)
   if (row_id >= p.n_split_items * 2 * kTile) return;
@@ -555,21 +557,40 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const CombineParams p
   const int pair = item % p.pairs, h = (item / p.pairs) % p.N_h, b = item / (p.pairs * p.N_h);
   const int row = pair * 2 * kTile + tr;
   if (row >= p.n) return;
-  const int stride = p.D + 4;
+  constexpr int stride = D + 4;
   const float* base = p.partial + ((size_t)si * p.splits * 2 * kTile + tr) * stride;  // piece 0 of this row
   const size_t piece = (size_t)2 * kTile * stride;
-  float m = -INFINITY;
-  for (int i = 0; i < p.splits; ++i) m = fmaxf(m, base[i * piece + p.D]);
-  float l = 0.f;
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};  // D <= 128: four columns per lane
-  for (int i = 0; i < p.splits; ++i) {
-    const float w = exp2f(base[i * piece + p.D] - m);
-    l += w * base[i * piece + p.D + 1];
-    for (int c = 0; c < p.D / 32; ++c) acc[c] += w * base[i * piece + c * 32 + lane];
+  // lane i holds piece i's reference maximum and sum (at most 16 pieces)
+  const float mi = (lane < p.splits) ? base[lane * piece + D] : -INFINITY;
+  const float li = (lane < p.splits) ? base[lane * piece + D + 1] : 0.f;
+  float m = mi;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  const float wi = (lane < p.splits) ? exp2f(mi - m) : 0.f;
+  float l = wi * li;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+  // all pieces' values are loaded before they are used, so the loads overlap
+  float v[16][CPL];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) v[i][c] = (i < p.splits) ? base[i * piece + lane * CPL + c] : 0.f;
+  }
+  float acc[CPL];
+#pragma unroll
+  for (int c = 0; c < CPL; ++c) acc[c] = 0.f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const float w = __shfl_sync(0xffffffffu, wi, i);
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) acc[c] += w * v[i][c];
   }
   const float inv = 1.f / l;
-  __nv_bfloat16* o = p.out + (((int64_t)b * p.n + row) * p.N_h + h) * p.D;
-  for (int c = 0; c < p.D / 32; ++c) o[c * 32 + lane] = __float2bfloat16(acc[c] * inv);
+  __nv_bfloat16* o = p.out + (((int64_t)b * p.n + row) * p.N_h + h) * D + lane * CPL;
+#pragma unroll
+  for (int c = 0; c < CPL; c += 2)
+    *reinterpret_cast<__nv_bfloat162*>(o + c) = __floats2bfloat162_rn(acc[c] * inv, acc[c + 1] * inv);
   if (p.lse && lane == 0 && row >= p.lse_row0 && row < p.lse_row0 + p.lse_rows)
     p.lse[((int64_t)b * p.N_h + h) * p.lse_rows + (row - p.lse_row0)] = (m + log2f(l)) * 0.6931471805599453f;
 }
@@ -660,7 +681,7 @@ cudaError_t launch_tc_d(const AttnArgs& a, int* status, float* partial, size_t p
   if (e != cudaSuccess || !splits) return e;
   CombineParams c{partial, (__nv_bfloat16*)a.out, a.lse, a.lse_row0, a.lse_rows, a.n, a.N_h, D, pairs, n_whole, splits, rem};
   ++*launches;
-  attn_combine_kernel<<<(rem * 2 * kTile + 7) / 8, 256, 0, st>>>(c);
+  attn_combine_kernel<D><<<(rem * 2 * kTile + 7) / 8, 256, 0, st>>>(c);
   return cudaGetLastError();
 }
 
