@@ -32,9 +32,9 @@ from paper_2609_38984_b200 import dist as sd  # noqa: E402
 from paper_2609_38984_b200 import workloads as W  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture summarised
-# under profiles/ (None until a capture of the current kernel exists)
-DOMINANT_KERNEL_DRAM_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel's launches in one cycle (dense launch + packed
+# launch), from the ncu capture summarised in profiles/attn_bf16_tc_larger_imagination.txt
+DOMINANT_KERNEL_DRAM_BYTES = {"larger_imagination": int((228.264192 + 57.030400 + 87.169280 + 13.018368) * 1e6)}
 
 
 def load_peaks():
