@@ -1,0 +1,132 @@
+"""Keep-ratio x refresh-interval sweep at the larger-imagination shape (seed 4).
+
+For each (keep, R) the workload's 10 denoising steps run through swam_step on one GPU; every stage is also timed
+on its own through the individual C-ABI calls.  Reported per configuration: the latency split over score, select,
+pack, attention (dense and packed) and scatter, the step latencies, packed tokens/s, the overlap of consecutive
+steps' selections (IoU of retained sets and the Eq. 13 overlap of the normalised score maps, from a diagnostic
+score + select at every step), and how far the sparse output is from the dense one (relative L2; a reported
+number, not a pass/fail: the paper gives no figure for it).
+
+  python -m paper_2609_38984_b200.sweep [--keeps 0.1,0.3] [--refresh 1,2,4] [--steps 10]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import numpy as np
+import torch
+
+from . import swam
+from . import workloads as W
+
+
+def _event_us(fn, reps=5):
+    ts = []
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        b.synchronize()
+        ts.append(a.elapsed_time(b) * 1e3)
+    return float(np.median(ts))
+
+
+def _graph_us(fn, launches=8, reps=3):
+    """Average device time of one fn() when `launches` of them are replayed back to back from a CUDA graph."""
+    fn()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for _ in range(launches):
+            fn()
+    g.replay()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        g.replay()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) * 1e3 / (launches * reps)
+
+
+def run_config(keep: float, refresh: int, n_steps: int, dev_steps, dense_outs) -> dict:
+    wl = W.sweep_workload(keep, refresh).with_(steps=n_steps)
+    ctx = swam.Swam.from_workload(wl)
+    diag = swam.Swam.from_workload(wl)          # diagnostic scoring/selection at every step
+    out = ctx.empty_full().zero_()
+    sched = W.refresh_schedule(n_steps, refresh)
+    step_us, rel_l2, ious, overlaps = [], [], [], []
+    prev_sel, prev_scores = None, None
+    for t, x in enumerate(dev_steps):
+        mode = swam.REFRESH_FULL if sched[t] else swam.REUSE
+        step_us.append(_event_us(lambda: ctx.step(x["q"], x["k"], x["v"], mode, out), reps=1))
+        ctx.check()
+        d = dense_outs[t].float()
+        rel_l2.append(float((out.float() - d).norm() / d.norm()))
+        s = diag.score(x["q"], x["k"])
+        sel, _, _ = diag.select(s)
+        sel_np, s_np = sel.cpu().numpy(), s.cpu().numpy().astype(np.float64)
+        if prev_sel is not None:
+            inter = [len(np.intersect1d(a, b)) for a, b in zip(prev_sel.reshape(-1, sel_np.shape[-1]),
+                                                               sel_np.reshape(-1, sel_np.shape[-1]))]
+            k = sel_np.shape[-1]
+            ious.append(float(np.mean([i / (2 * k - i) for i in inter])))
+            p = prev_scores / prev_scores.sum(-1, keepdims=True)
+            q = s_np / s_np.sum(-1, keepdims=True)
+            overlaps.append(float(np.minimum(p, q).sum(-1).mean()))      # Eq. 13 per (sample, frame)
+        prev_sel, prev_scores = sel_np, s_np
+    # stage split on the last step's inputs with the cached selection
+    x = dev_steps[-1]
+    _, lse_act, _ = ctx.cached_scores()
+    sel, pm, im = ctx.selection()
+    scores = ctx.score(x["q"], x["k"], lse_act)
+    qp, kp, vp = ctx.pack(x["q"], x["k"], x["v"], pm)
+    op = ctx.sparse_attn(qp, kp, vp)
+    lib, P, S = ctx.lib, swam._ptr, swam._stream
+    split = {
+        "score": _graph_us(lambda: lib.swam_score(ctx.ctx, P(x["q"]), P(x["k"]), P(lse_act), P(scores), None, S())),
+        "select": _graph_us(lambda: lib.swam_select(ctx.ctx, P(scores), P(sel), P(pm), P(im), S())),
+        "pack": _graph_us(lambda: lib.swam_pack(ctx.ctx, P(x["q"]), P(x["k"]), P(x["v"]), P(pm), P(qp), P(kp), P(vp), S())),
+        "attn_packed": _graph_us(lambda: lib.swam_sparse_attn(ctx.ctx, P(qp), P(kp), P(vp), wl.packed_len, P(op), None, S())),
+        "scatter": _graph_us(lambda: lib.swam_scatter(ctx.ctx, P(op), P(pm), P(im), P(out), P(out), S())),
+        "attn_dense": _graph_us(lambda: lib.swam_sparse_attn(ctx.ctx, P(x["q"]), P(x["k"]), P(x["v"]), wl.seq_len, P(out), None, S()),
+                                launches=4),
+    }
+    ctx.check()
+    full = [u for u, f in zip(step_us, sched) if f]
+    sparse = [u for u, f in zip(step_us, sched) if not f]
+    total_us = float(np.sum(step_us))
+    tokens = wl.batch * sum(wl.seq_len if f else wl.packed_len for f in sched)
+    return {
+        "keep": keep, "refresh": refresh, "k_core": wl.budgets[0], "k_anchor": wl.budgets[1], "packed_len": wl.packed_len,
+        "steps": n_steps, "full_steps": len(full), "stage_us": {k: round(v, 2) for k, v in split.items()},
+        "full_step_us": round(float(np.median(full)), 1), "sparse_step_us": round(float(np.median(sparse)), 1) if sparse else None,
+        "schedule_us": round(total_us, 1), "tokens_per_s": tokens / (total_us * 1e-6),
+        "iou_consecutive_steps": round(float(np.mean(ious)), 4), "overlap_eq13_consecutive_steps": round(float(np.mean(overlaps)), 4),
+        "rel_l2_vs_dense_per_step": [round(v, 4) for v in rel_l2],
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--keeps", default=",".join(str(k) for k in W.SWEEP_KEEPS))
+    ap.add_argument("--refresh", default=",".join(str(r) for r in W.SWEEP_REFRESH))
+    ap.add_argument("--steps", type=int, default=10)
+    args = ap.parse_args()
+    keeps = [float(k) for k in args.keeps.split(",")]
+    refreshes = [int(r) for r in args.refresh.split(",")]
+    base = W.sweep_workload(1.0, 1).with_(steps=args.steps)
+    host = W.generate_steps(base, args.steps)              # the inputs do not depend on keep or R
+    dev_steps = [{n: swam.to_device(x[n], base.dtype) for n in "qkv"} for x in host]
+    dense_ctx = swam.Swam.from_workload(base)
+    dense_outs = [dense_ctx.sparse_attn(x["q"], x["k"], x["v"]) for x in dev_steps]   # memoised dense results
+    for keep in keeps:
+        for r in refreshes:
+            print(json.dumps(run_config(keep, r, args.steps, dev_steps, dense_outs)), flush=True)
+
+
+if __name__ == "__main__":
+    main()
