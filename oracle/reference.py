@@ -150,6 +150,39 @@ def select(scores_f32: np.ndarray, k_core: int, k_anchor: int, beta: float = 1.0
     return res
 
 
+def aggregate(layer_scores: np.ndarray, layer_quality: np.ndarray, k_layer: int):
+    """Multi-layer aggregation (Eq. 3, Eq. 11): layer_scores [n_layers, B, F, N_s] float32, layer_quality
+    [n_layers, B, 3] float32 (R, E, Q per layer, Eq. 9).  Returns v_core, v_all [B, F, N_s] float32 and the chosen
+    core layers [B, k_layer] (ascending)."""
+    lib = _load()
+    ls = np.ascontiguousarray(layer_scores, dtype=np.float32)
+    nl, b, f, n = ls.shape
+    lq = np.ascontiguousarray(layer_quality, dtype=np.float32)
+    v_core = np.empty((b, f, n), np.float32)
+    v_all = np.empty((b, f, n), np.float32)
+    layers = np.empty((b, min(k_layer, nl)), np.int32)
+    for i in range(b):
+        si = np.ascontiguousarray(ls[:, i].reshape(nl, f * n))
+        qi = np.ascontiguousarray(lq[:, i, 2])
+        lib.oracle_aggregate(_p(si, ctypes.c_float), _p(qi, ctypes.c_float), ctypes.c_int(nl), ctypes.c_int(k_layer),
+                             ctypes.c_int(f * n), _p(v_core[i], ctypes.c_float), _p(v_all[i], ctypes.c_float),
+                             _p(layers[i], ctypes.c_int32))
+    return v_core, v_all, layers
+
+
+def select2(v_core: np.ndarray, v_all: np.ndarray, k_core: int, k_anchor: int, beta: float = 1.0) -> np.ndarray:
+    """Selection with the core score map V for pool and cores and V_all for the anchors; sel_idx [B, F, K]."""
+    lib = _load()
+    vc = np.ascontiguousarray(v_core, dtype=np.float32)
+    va = np.ascontiguousarray(v_all, dtype=np.float32)
+    b, f, n = vc.shape
+    sel = np.zeros((b, f, k_core + k_anchor), np.int32)
+    for i in range(b):
+        lib.oracle_select2(_p(vc[i], ctypes.c_float), _p(va[i], ctypes.c_float), ctypes.c_int(f), ctypes.c_int(n),
+                           ctypes.c_int(k_core), ctypes.c_int(k_anchor), ctypes.c_double(beta), _p(sel[i], ctypes.c_int32))
+    return sel
+
+
 def maps(sel_idx: np.ndarray, n_obs: int, n_spatial: int, n_action: int) -> Tuple[np.ndarray, np.ndarray]:
     """pack_map [B, L'] and inv_map [B, L] (Sec. 4.2 packing metadata)."""
     lib = _load()

@@ -250,3 +250,89 @@ void oracle_maps(const int32_t* sel_idx, int n_obs, int n_frames, int n_spatial,
     for (int t = 0; t < n_action; ++t) pack_map[p++] = n_obs + n_frames * n_spatial + t;
     for (int i = 0; i < p; ++i) inv_map[pack_map[i]] = i;
 }
+
+/* ------------------------------------------------------------------------
+ * Multi-layer aggregation for one sample (Eq. 3 and the first line of Eq. 11).
+ * layer_scores: [n_layers, F*N_s] stored fp32 scores S_l; layer_q: [n_layers] layer qualities Q_l (Eq. 9).
+ *   L_core = the k_layer layers with the largest Q_l (equal Q_l: lower layer index)
+ *   V      = sum_{l in L_core} Q_l S_l / sum_{l in L_core} Q_l        (Eq. 3)
+ *   V_all  = sum_l Q_l S_l / sum_l Q_l                               (Eq. 11)
+ * Sums run over layers in ascending order in double; results are stored as fp32.  When the weights of a set
+ * sum to zero (every layer uniform) the plain mean over that set is used.
+ * core_layers: [k_layer] ascending layer indices (may be NULL).
+ * ------------------------------------------------------------------------ */
+void oracle_aggregate(const float* layer_scores, const float* layer_q, int n_layers, int k_layer, int n_elems,
+                      float* v_core, float* v_all, int32_t* core_layers)
+{
+    keyed* cand = (keyed*)malloc(sizeof(keyed) * (size_t)n_layers);
+    uint8_t* in_core = (uint8_t*)calloc((size_t)n_layers, 1);
+    for (int l = 0; l < n_layers; ++l) { cand[l].key = (double)layer_q[l]; cand[l].idx = l; }
+    qsort(cand, (size_t)n_layers, sizeof(keyed), by_key_desc_idx_asc);
+    for (int r = 0; r < k_layer && r < n_layers; ++r) in_core[cand[r].idx] = 1;
+    double wc = 0.0, wa = 0.0;
+    int nc = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        wa = wa + (double)layer_q[l];
+        if (in_core[l]) { wc = wc + (double)layer_q[l]; ++nc; }
+    }
+    for (int e = 0; e < n_elems; ++e) {
+        double sc = 0.0, sa = 0.0;
+        for (int l = 0; l < n_layers; ++l) {
+            const double s = (double)layer_scores[(size_t)l * n_elems + e];
+            const double w = (double)layer_q[l];
+            const double wa_l = (wa == 0.0) ? 1.0 : w;
+            const double wc_l = (wc == 0.0) ? 1.0 : w;
+            sa = sa + wa_l * s;
+            if (in_core[l]) sc = sc + wc_l * s;
+        }
+        v_all[e] = (float)(sa / ((wa == 0.0) ? (double)n_layers : wa));
+        v_core[e] = (float)(sc / ((wc == 0.0) ? (double)nc : wc));
+    }
+    if (core_layers) { int n = 0; for (int l = 0; l < n_layers; ++l) if (in_core[l]) core_layers[n++] = l; }
+    free(cand); free(in_core);
+}
+
+/* Selection with separate score maps: pool and cores rank v_core (Eq. 4-5), anchors use v_all (Eq. 11, Eq. 6). */
+void oracle_select2(const float* v_core, const float* v_all, int n_frames, int n_spatial, int k_core, int k_anchor,
+                    double beta, int32_t* sel_idx)
+{
+    const int F = n_frames, N = n_spatial, K = k_core + k_anchor;
+    keyed* cand = (keyed*)malloc(sizeof(keyed) * (size_t)N);
+    uint8_t* pool = (uint8_t*)calloc((size_t)N, 1);
+    uint8_t* core = (uint8_t*)calloc((size_t)F * N, 1);
+    uint8_t* in_any_core = (uint8_t*)calloc((size_t)N, 1);
+    uint8_t* anchor = (uint8_t*)calloc((size_t)N, 1);
+    for (int j = 0; j < N; ++j) {
+        double m = (double)v_core[j];
+        for (int f = 1; f < F; ++f) if ((double)v_core[f * N + j] > m) m = (double)v_core[f * N + j];
+        cand[j].key = m; cand[j].idx = j;
+    }
+    topk_sorted(cand, N, N - k_anchor);
+    for (int r = 0; r < N - k_anchor; ++r) pool[cand[r].idx] = 1;
+    for (int f = 0; f < F; ++f) {
+        int nc = 0;
+        for (int j = 0; j < N; ++j) if (pool[j]) { cand[nc].key = (double)v_core[f * N + j]; cand[nc].idx = j; ++nc; }
+        topk_sorted(cand, nc, k_core);
+        for (int r = 0; r < k_core; ++r) { core[f * N + cand[r].idx] = 1; in_any_core[cand[r].idx] = 1; }
+    }
+    int ne = 0;
+    for (int j = 0; j < N; ++j) {
+        if (in_any_core[j]) continue;
+        double sum = 0.0;
+        for (int f = 0; f < F; ++f) sum = sum + (double)v_all[f * N + j];
+        const double mu = sum / (double)F;
+        double ss = 0.0;
+        for (int f = 0; f < F; ++f) { const double d = (double)v_all[f * N + j] - mu; ss = ss + d * d; }
+        const double sd = sqrt(ss / (double)F);
+        const double cv = (mu == 0.0) ? 0.0 : sd / mu;
+        cand[ne].key = mu / (1.0 + beta * cv); cand[ne].idx = j; ++ne;
+    }
+    topk_sorted(cand, ne, k_anchor);
+    for (int r = 0; r < k_anchor; ++r) anchor[cand[r].idx] = 1;
+    for (int f = 0; f < F; ++f) {
+        int n = 0;
+        for (int j = 0; j < N; ++j) if (core[f * N + j] || anchor[j]) { if (n < K) sel_idx[f * K + n] = j; ++n; }
+        if (n != K) sel_idx[0] = -1;
+    }
+    free(cand); free(pool); free(core); free(in_any_core); free(anchor);
+}

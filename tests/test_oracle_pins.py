@@ -368,3 +368,57 @@ def test_overlap_measure():
     assert abs(ora.overlap(p, p * 7) - 1.0) < 1e-15
     assert ora.overlap(np.array([1.0, 0, 0]), np.array([0, 2.0, 1.0])) == 0.0
     assert abs(ora.overlap(np.array([1.0, 1.0]), np.array([3.0, 1.0])) - 0.75) < 1e-15
+
+
+# ------------------------------------------------------------------ multi-layer aggregation (Eq. 3, Eq. 9, Eq. 11)
+def _layers(seed, nl, b, f, n):
+    s = np.stack([W.random_scores(seed + l, b, f, n) for l in range(nl)])
+    q = np.stack([ora.quality(s[l]) for l in range(nl)]).astype(np.float32)
+    return s, q
+
+
+def test_aggregate_single_layer_is_the_layer_itself():
+    s, q = _layers(40, 1, 2, 3, 17)
+    vc, va, layers = ora.aggregate(s, q, 1)
+    assert np.array_equal(vc, s[0]) and np.array_equal(va, s[0]) and layers.tolist() == [[0], [0]]
+    # and the selection from (V, V_all) equals the single-map selection
+    assert np.array_equal(ora.select2(vc, va, 4, 5), ora.select(s[0], 4, 5)["sel_idx"])
+
+
+def test_aggregate_against_direct_weighted_mean():
+    nl, b, f, n, kl = 5, 2, 3, 19, 2
+    s, q = _layers(50, nl, b, f, n)
+    q[:, :, 2] = np.array([[0.1, 0.4], [0.5, 0.2], [0.3, 0.6], [0.05, 0.1], [0.5, 0.3]], np.float32)   # with a tie in sample 0
+    vc, va, layers = ora.aggregate(s, q, kl)
+    assert layers.tolist() == [[1, 4], [0, 2]]                      # top-2 by Q (sample 0: the 0.5/0.5 tie beats 0.3)
+    for i in range(b):
+        w = q[:, i, 2].astype(np.float64)
+        want_all = np.tensordot(w, s[:, i].astype(np.float64), axes=1) / w.sum()
+        sel = layers[i]
+        want_core = np.tensordot(w[sel], s[sel, i].astype(np.float64), axes=1) / w[sel].sum()
+        # results are stored as fp32: half an ulp at these magnitudes is below 4e-9
+        assert np.abs(va[i] - want_all).max() <= 5e-9 and np.abs(vc[i] - want_core).max() <= 5e-9
+    # all layers selected: V equals V_all
+    vc2, va2, _ = ora.aggregate(s, q, nl)
+    assert np.array_equal(vc2, va2)
+    # equal qualities: plain mean over layers; zero qualities fall back to the plain mean as well
+    q[:, :, 2] = 0.25
+    _, va3, _ = ora.aggregate(s, q, nl)
+    assert np.abs(va3 - s.astype(np.float64).mean(0)).max() <= 5e-9
+    q[:, :, 2] = 0.0
+    _, va4, _ = ora.aggregate(s, q, nl)
+    assert np.abs(va4 - s.astype(np.float64).mean(0)).max() <= 5e-9
+
+
+def test_select2_uses_core_map_for_cores_and_all_map_for_anchors():
+    f, n, kc, ks = 2, 12, 2, 3
+    v_core = np.zeros((1, f, n), np.float32)
+    v_all = np.zeros((1, f, n), np.float32)
+    v_core[0, 0, [3, 7]] = [0.9, 0.8]          # frame 0 cores
+    v_core[0, 1, [5, 1]] = [0.9, 0.7]          # frame 1 cores
+    v_all[0, :, 10] = 0.5                      # strong and steady in V_all only
+    v_all[0, :, 11] = 0.4
+    v_all[0, :, 2] = 0.3
+    v_all[0, :, 3] = 0.95                      # core position: must not become an anchor
+    sel = ora.select2(v_core, v_all, kc, ks)
+    assert sel[0, 0].tolist() == [2, 3, 7, 10, 11] and sel[0, 1].tolist() == [1, 2, 5, 10, 11]
