@@ -103,6 +103,19 @@ int swam_score_noalloc(swam_ctx* ctx, const void* q, const void* k, float* score
 int swam_select(swam_ctx* ctx, const float* scores, int32_t* sel_idx, int32_t* pack_map, int32_t* inv_map,
                 void* stream);
 
+/* (2b) Several profiled layers (Sec. 4.1, App. A.1).  swam_aggregate forms the core score map
+ *   V = sum_{l in L_core} Q_l S_l / sum_{l in L_core} Q_l (Eq. 3), L_core = the k_layer layers with the largest Q_l,
+ * and the anchor score map V_all, the same sum over all layers (Eq. 11), from per-layer scores and qualities as
+ * swam_score writes them: layer_scores dev float [n_layers, B, F, N_s], layer_quality dev float [n_layers, B, 3]
+ * (R, E, Q of Eq. 9; only Q is used).  fp64 accumulation in ascending layer order, results stored as fp32; equal
+ * qualities go to the lower layer index; if the weights of a set sum to zero the plain mean is used.  v_core, v_all:
+ * dev float [B, F, N_s]; core_layers: dev int32 [B, k_layer] ascending, or NULL.  n_layers <= 256.
+ * swam_select_maps is call (2) with pool and cores ranked on core_scores (V) and anchors on anchor_scores (V_all). */
+int swam_aggregate(swam_ctx* ctx, const float* layer_scores, const float* layer_quality, int32_t n_layers,
+                   int32_t k_layer, float* v_core, float* v_all, int32_t* core_layers, void* stream);
+int swam_select_maps(swam_ctx* ctx, const float* core_scores, const float* anchor_scores, int32_t* sel_idx,
+                     int32_t* pack_map, int32_t* inv_map, void* stream);
+
 /* (3) Packing (Sec. 4.2): xp[b, p, :] = x[b, pack_map[b, p], :] for x in {q, k, v}; xp: dev [B, L', N_h, D].
  * Any of the three pairs may be NULL/NULL.  Out-of-range map entries are skipped and flagged in the status word. */
 int swam_pack(swam_ctx* ctx, const void* q, const void* k, const void* v, const int32_t* pack_map,

@@ -183,7 +183,8 @@ __device__ int ranked_emit(const Scratch& s, int n, FlagFn flag, EmitFn emit) {
 }
 
 struct SelectParams {
-  const float* scores;
+  const float* scores;      // core score map V: pool and cores
+  const float* scores_all;  // anchor score map V_all (may equal scores)
   int32_t* sel_idx;
   int32_t* pack_map;
   int32_t* inv_map;
@@ -194,13 +195,14 @@ struct SelectParams {
 
 // shared-memory layout (bytes), identical in every CTA of the cluster
 struct SelLayout {
-  size_t keyA, S, keyM, hist, warp_tot, scal, pool, anchor, anycore, core, total;
+  size_t keyA, S, Sall, keyM, hist, warp_tot, scal, pool, anchor, anycore, core, total;
 };
 __host__ __device__ inline SelLayout sel_layout(int F, int N) {
   SelLayout l;
   size_t o = 0;
   l.keyA = o; o += (size_t)N * 8;
   l.S = o; o += (size_t)F * N * 4;
+  l.Sall = o; o += (size_t)F * N * 4;
   l.keyM = o; o += (size_t)N * 4;
   l.hist = o; o += 256 * 4;
   l.warp_tot = o; o += 32 * 4;
@@ -234,6 +236,13 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
   const int tid = threadIdx.x, b = blockIdx.y;
   const float* sg = p.scores + (int64_t)b * F * N;
   for (int i = tid; i < F * N; i += kSelThreads) S[i] = sg[i];
+  const float* Sall = S;  // the anchor statistic reads V_all; with one profiled layer it is the same map
+  if (p.scores_all != p.scores) {
+    float* sa = reinterpret_cast<float*>(smem_raw + lay.Sall);
+    const float* sag = p.scores_all + (int64_t)b * F * N;
+    for (int i = tid; i < F * N; i += kSelThreads) sa[i] = sag[i];
+    Sall = sa;
+  }
   __syncthreads();
 
   // candidate pool: top (N_s - K_s) of max_f S(f, j)                                   (Eq. 4)
@@ -257,11 +266,11 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
   const int j_lo = rank * share, j_hi = min(N, j_lo + share);
   for (int j = j_lo + tid; j < j_hi; j += kSelThreads) {
     double sum = 0.0;
-    for (int f = 0; f < F; ++f) sum = __dadd_rn(sum, (double)S[f * N + j]);
+    for (int f = 0; f < F; ++f) sum = __dadd_rn(sum, (double)Sall[f * N + j]);
     const double mu = __ddiv_rn(sum, (double)F);
     double ss = 0.0;
     for (int f = 0; f < F; ++f) {
-      const double dv = __dadd_rn((double)S[f * N + j], -mu);
+      const double dv = __dadd_rn((double)Sall[f * N + j], -mu);
       ss = __dadd_rn(ss, __dmul_rn(dv, dv));
     }
     const double sd = __dsqrt_rn(__ddiv_rn(ss, (double)F));
@@ -325,6 +334,54 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
   if (bad && tid == 0) atomicOr(p.status, ST_BAD_COUNT);
 }
 
+// Multi-layer aggregation (Eq. 3, Eq. 11): V = sum over the k_layer best layers of Q_l S_l / sum Q_l and V_all the
+// same over all layers, in fp64 with individually rounded operations, layers in ascending order, stored as fp32.
+// Equal qualities go to the lower layer index; weights that sum to zero fall back to the plain mean.
+constexpr int kMaxLayers = 256;
+
+__global__ void __launch_bounds__(256) aggregate_kernel(const float* layer_scores, const float* layer_quality, int n_layers,
+                                                        int k_layer, int B, int n_elems, float* v_core, float* v_all,
+                                                        int32_t* core_layers) {
+  __shared__ double q[kMaxLayers];
+  __shared__ uint8_t in_core[kMaxLayers];
+  __shared__ double wsum[2];
+  __shared__ int n_core;
+  const int b = blockIdx.y, tid = threadIdx.x;
+  for (int l = tid; l < n_layers; l += 256) q[l] = (double)layer_quality[((size_t)l * B + b) * 3 + 2];
+  __syncthreads();
+  for (int l = tid; l < n_layers; l += 256) {
+    int rank = 0;
+    for (int m = 0; m < n_layers; ++m) rank += (q[m] > q[l] || (q[m] == q[l] && m < l)) ? 1 : 0;
+    in_core[l] = rank < k_layer ? 1 : 0;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    double wc = 0.0, wa = 0.0;
+    int nc = 0;
+    for (int l = 0; l < n_layers; ++l) {
+      wa = __dadd_rn(wa, q[l]);
+      if (in_core[l]) {
+        wc = __dadd_rn(wc, q[l]);
+        if (core_layers && blockIdx.x == 0) core_layers[(size_t)b * min(k_layer, n_layers) + nc] = l;
+        ++nc;
+      }
+    }
+    wsum[0] = wc; wsum[1] = wa; n_core = nc;
+  }
+  __syncthreads();
+  const double wc = wsum[0], wa = wsum[1];
+  const int e = blockIdx.x * 256 + tid;
+  if (e >= n_elems) return;
+  double sc = 0.0, sa = 0.0;
+  for (int l = 0; l < n_layers; ++l) {
+    const double s = (double)layer_scores[((size_t)l * B + b) * n_elems + e];
+    sa = __dadd_rn(sa, __dmul_rn(wa == 0.0 ? 1.0 : q[l], s));
+    if (in_core[l]) sc = __dadd_rn(sc, __dmul_rn(wc == 0.0 ? 1.0 : q[l], s));
+  }
+  v_all[(size_t)b * n_elems + e] = (float)__ddiv_rn(sa, wa == 0.0 ? (double)n_layers : wa);
+  v_core[(size_t)b * n_elems + e] = (float)__ddiv_rn(sc, wc == 0.0 ? (double)n_core : wc);
+}
+
 int cluster_size(const Dims& d) {
   int c = 1;
   while (c * 2 <= d.F && c * 2 <= kMaxCluster) c *= 2;
@@ -335,15 +392,27 @@ int cluster_size(const Dims& d) {
 
 size_t select_smem_bytes(const Dims& d) { return sel_layout(d.F, d.N_s).total; }
 
+int max_layers() { return kMaxLayers; }
+
+cudaError_t launch_aggregate(const Dims& d, const float* layer_scores, const float* layer_quality, int n_layers, int k_layer,
+                             float* v_core, float* v_all, int32_t* core_layers, cudaStream_t st, int* launches) {
+  const int n_elems = d.F * d.N_s;
+  dim3 grid((n_elems + 255) / 256, d.B);
+  ++*launches;
+  aggregate_kernel<<<grid, 256, 0, st>>>(layer_scores, layer_quality, n_layers, k_layer, d.B, n_elems, v_core, v_all,
+                                         core_layers);
+  return cudaGetLastError();
+}
+
 cudaError_t select_prepare(const Dims& d) {
   const size_t smem = select_smem_bytes(d);
   if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
   return cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
 
-cudaError_t launch_select(const Dims& d, const float* scores, int32_t* sel_idx, int32_t* pack_map,
-                          int32_t* inv_map, int* status, cudaStream_t st, int* launches) {
-  SelectParams p{scores, sel_idx, pack_map, inv_map, status, d.n_obs, d.F, d.N_s, d.H,
+cudaError_t launch_select(const Dims& d, const float* scores, const float* scores_all, int32_t* sel_idx,
+                          int32_t* pack_map, int32_t* inv_map, int* status, cudaStream_t st, int* launches) {
+  SelectParams p{scores, scores_all ? scores_all : scores, sel_idx, pack_map, inv_map, status, d.n_obs, d.F, d.N_s, d.H,
                  d.Kc, d.Ks, d.L, d.Lp, (double)d.beta};
   const int C = cluster_size(d);
   cudaLaunchConfig_t cfg = {};

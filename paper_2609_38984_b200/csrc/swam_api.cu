@@ -247,7 +247,30 @@ int swam_score_noalloc(swam_ctx* c, const void* q, const void* k, float* scores,
 int swam_select(swam_ctx* c, const float* scores, int32_t* sel_idx, int32_t* pack_map, int32_t* inv_map, void* stream) {
   if (!c || !scores) return fail(c, SWAM_ERR_INVALID_ARG, "swam_select: null argument");
   if (int r = need_ws(c)) return r;
-  cudaError_t e = launch_select(c->d, scores, sel_idx, pack_map, inv_map, (int*)(c->ws + c->off_status),
+  cudaError_t e = launch_select(c->d, scores, nullptr, sel_idx, pack_map, inv_map, (int*)(c->ws + c->off_status),
+                                (cudaStream_t)stream, &c->launches_i);
+  count(c);
+  if (e != cudaSuccess) return fail_cuda(c, e, "select launch");
+  return SWAM_OK;
+}
+
+int swam_aggregate(swam_ctx* c, const float* layer_scores, const float* layer_quality, int32_t n_layers, int32_t k_layer,
+                   float* v_core, float* v_all, int32_t* core_layers, void* stream) {
+  if (!c || !layer_scores || !layer_quality || !v_core || !v_all) return fail(c, SWAM_ERR_INVALID_ARG, "swam_aggregate: null argument");
+  if (n_layers <= 0 || k_layer <= 0 || k_layer > n_layers) return fail(c, SWAM_ERR_INVALID_ARG, "swam_aggregate: need 0 < k_layer <= n_layers");
+  if (n_layers > max_layers()) return fail(c, SWAM_ERR_UNSUPPORTED, "swam_aggregate: too many layers");
+  cudaError_t e = launch_aggregate(c->d, layer_scores, layer_quality, n_layers, k_layer, v_core, v_all, core_layers,
+                                   (cudaStream_t)stream, &c->launches_i);
+  count(c);
+  if (e != cudaSuccess) return fail_cuda(c, e, "aggregate launch");
+  return SWAM_OK;
+}
+
+int swam_select_maps(swam_ctx* c, const float* core_scores, const float* anchor_scores, int32_t* sel_idx, int32_t* pack_map,
+                     int32_t* inv_map, void* stream) {
+  if (!c || !core_scores || !anchor_scores) return fail(c, SWAM_ERR_INVALID_ARG, "swam_select_maps: null argument");
+  if (int r = need_ws(c)) return r;
+  cudaError_t e = launch_select(c->d, core_scores, anchor_scores, sel_idx, pack_map, inv_map, (int*)(c->ws + c->off_status),
                                 (cudaStream_t)stream, &c->launches_i);
   count(c);
   if (e != cudaSuccess) return fail_cuda(c, e, "select launch");

@@ -40,8 +40,13 @@ cudaError_t static_scratch(const Dims& d, float** lse, void** partial);
 // ---- select.cu ------------------------------------------------------------
 size_t select_smem_bytes(const Dims& d);
 cudaError_t select_prepare(const Dims& d);  // opt in to the dynamic shared memory the kernel needs
-cudaError_t launch_select(const Dims& d, const float* scores, int32_t* sel_idx, int32_t* pack_map,
-                          int32_t* inv_map, int* status, cudaStream_t st, int* launches);
+// scores: core map (pool, cores); scores_all: anchor map, nullptr => same as scores
+cudaError_t launch_select(const Dims& d, const float* scores, const float* scores_all, int32_t* sel_idx,
+                          int32_t* pack_map, int32_t* inv_map, int* status, cudaStream_t st, int* launches);
+int max_layers();
+// V and V_all from per-layer scores [n_layers, B, F, N_s] and qualities [n_layers, B, 3]
+cudaError_t launch_aggregate(const Dims& d, const float* layer_scores, const float* layer_quality, int n_layers, int k_layer,
+                             float* v_core, float* v_all, int32_t* core_layers, cudaStream_t st, int* launches);
 
 // ---- pack_scatter.cu ------------------------------------------------------
 // dst[b, p] = src[b, map[b,p]] for up to three tensor pairs (row_bytes per row).

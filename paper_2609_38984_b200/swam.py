@@ -25,7 +25,7 @@ ATTN_AUTO, ATTN_WARP_MMA = 0, 1
 
 EXPORTS = [
     "swam_create", "swam_destroy", "swam_workspace_bytes", "swam_bind_workspace", "swam_score", "swam_score_noalloc",
-    "swam_select",
+    "swam_select", "swam_aggregate", "swam_select_maps",
     "swam_pack", "swam_sparse_attn", "swam_scatter", "swam_step", "swam_host_io_bytes", "swam_bind_host_io",
     "swam_step_host", "swam_get_selection", "swam_get_scores", "swam_check", "swam_set_option", "swam_launch_count",
     "swam_last_error", "swam_version",
@@ -69,6 +69,8 @@ def load_library() -> ctypes.CDLL:
         lib.swam_score.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         lib.swam_score_noalloc.argtypes = [vp, vp, vp, vp, vp]
         lib.swam_select.argtypes = [vp, vp, vp, vp, vp, vp]
+        lib.swam_aggregate.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp]
+        lib.swam_select_maps.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         lib.swam_pack.argtypes = [vp] * 9
         lib.swam_sparse_attn.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp]
         lib.swam_scatter.argtypes = [vp] * 7
@@ -201,6 +203,24 @@ class Swam:
         pack = torch.empty((self.B, self.Lp), dtype=torch.int32, device=self.device)
         inv = torch.empty((self.B, self.L), dtype=torch.int32, device=self.device)
         self._chk(self.lib.swam_select(self.ctx, _ptr(scores), _ptr(sel), _ptr(pack), _ptr(inv), _stream()))
+        return sel, pack, inv
+
+    def aggregate(self, layer_scores, layer_quality, k_layer: int):
+        """V, V_all and the chosen core layers from per-layer scores [n_layers, B, F, N_s] and qualities [n_layers, B, 3]."""
+        n_layers = layer_scores.shape[0]
+        v_core = torch.empty((self.B, self.F, self.N_s), dtype=torch.float32, device=self.device)
+        v_all = torch.empty_like(v_core)
+        layers = torch.empty((self.B, k_layer), dtype=torch.int32, device=self.device)
+        self._chk(self.lib.swam_aggregate(self.ctx, _ptr(layer_scores), _ptr(layer_quality), n_layers, k_layer,
+                                          _ptr(v_core), _ptr(v_all), _ptr(layers), _stream()))
+        return v_core, v_all, layers
+
+    def select_maps(self, core_scores, anchor_scores):
+        sel = torch.empty((self.B, self.F, self.K), dtype=torch.int32, device=self.device)
+        pack = torch.empty((self.B, self.Lp), dtype=torch.int32, device=self.device)
+        inv = torch.empty((self.B, self.L), dtype=torch.int32, device=self.device)
+        self._chk(self.lib.swam_select_maps(self.ctx, _ptr(core_scores), _ptr(anchor_scores), _ptr(sel), _ptr(pack),
+                                            _ptr(inv), _stream()))
         return sel, pack, inv
 
     def pack(self, q, k, v, pack_map):

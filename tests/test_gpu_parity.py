@@ -349,3 +349,55 @@ def test_host_buffer_step_matches_device_step():
         ctx_b.step_host(hq, hk, hv, mode, out_host)
         ctx_b.check()
         assert torch.equal(out_dev.cpu(), out_host)
+
+
+# ------------------------------------------------------------------ several profiled layers (Eq. 3, Eq. 9, Eq. 11)
+@pytest.mark.parametrize("wl,n_layers,k_layer", [
+    (small(batch=2), 5, 2),
+    (small("larger_imagination", n_obs=40, grid_h=7, grid_w=9, n_heads=2), 6, 6),
+], ids=["5_layers_top2", "6_layers_all"])
+def test_multi_layer_aggregation_and_selection(wl, n_layers, k_layer):
+    swam = _swam()
+    layers = W.generate_steps(wl.with_(rho=0.5), n_layers)          # one (q, k) pair per profiled layer
+    ctx = swam.Swam.from_workload(wl)
+    kc, ks = wl.budgets
+    s_dev, q_dev = [], []
+    for x in layers:
+        s, qual = ctx.score(dev(x["q"], wl), dev(x["k"], wl), quality=True)
+        s_dev.append(s)
+        q_dev.append(qual)
+    ls, lq = torch.stack(s_dev).contiguous(), torch.stack(q_dev).contiguous()
+    v_core, v_all, core_layers = ctx.aggregate(ls, lq, k_layer)
+    sel, pm, im = ctx.select_maps(v_core, v_all)
+    ctx.check()
+    # stage-isolated: the oracle on the device's own per-layer arrays must agree bit for bit
+    wc, wa, wl_layers = ora.aggregate(ls.cpu().numpy(), lq.cpu().numpy(), k_layer)
+    assert np.array_equal(core_layers.cpu().numpy(), wl_layers)
+    assert np.array_equal(v_core.cpu().numpy(), wc) and np.array_equal(v_all.cpu().numpy(), wa)
+    want_sel = ora.select2(wc, wa, kc, ks)
+    wpm, wim = ora.maps(want_sel, wl.n_obs, wl.n_spatial, wl.n_action)
+    assert np.array_equal(sel.cpu().numpy(), want_sel)
+    assert np.array_equal(pm.cpu().numpy(), wpm) and np.array_equal(im.cpu().numpy(), wim)
+    # end to end from the oracle's own scores and qualities
+    os_ = np.stack([ora.score(x["q"], x["k"], wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action).astype(np.float32)
+                    for x in layers])
+    oq = np.stack([ora.quality(s) for s in os_]).astype(np.float32)
+    ec, ea, el = ora.aggregate(os_, oq, k_layer)
+    assert np.array_equal(el, wl_layers)
+    assert (np.abs(v_core.cpu().numpy() - ec) / ec).max() <= 1e-4 and (np.abs(v_all.cpu().numpy() - ea) / ea).max() <= 1e-4
+    if k_layer == n_layers:
+        assert torch.equal(v_core, v_all)
+
+
+def test_single_layer_aggregation_is_identity():
+    swam = _swam()
+    wl = small()
+    x = W.generate_steps(wl, 1)[0]
+    ctx = swam.Swam.from_workload(wl)
+    s, qual = ctx.score(dev(x["q"], wl), dev(x["k"], wl), quality=True)
+    v_core, v_all, _ = ctx.aggregate(s.unsqueeze(0).contiguous(), qual.unsqueeze(0).contiguous(), 1)
+    assert torch.equal(v_core, s) and torch.equal(v_all, s)
+    a = ctx.select(s)
+    b = ctx.select_maps(v_core, v_all)
+    for t, u in zip(a, b):
+        assert torch.equal(t, u)
