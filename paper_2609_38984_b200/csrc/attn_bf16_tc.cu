@@ -77,17 +77,23 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// The issuing thread's own instruction count per MMA matters (one MMA of this size executes in 32-64 clk), so the
+// 64-bit shared-memory descriptors are kept as a constant high word and a low word that only needs an add.
 // D[tmem] (+)= A[smem desc] * B[smem desc]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
+template <bool kAccum>
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc) {
   asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accum) : "memory");
+      "{\n .reg .pred p;\n .reg .b64 da, db;\n setp.ne.b32 p, %5, 0;\n mov.b64 da, {%1, %3};\n mov.b64 db, {%2, %3};\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "n"(kAccum ? 1 : 0) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem desc]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                       uint32_t accum) {
   asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accum) : "memory");
+      "{\n .reg .pred p;\n .reg .b64 db;\n setp.ne.b32 p, %5, 0;\n mov.b64 db, {%2, %3};\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accum) : "memory");
 }
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
@@ -157,16 +163,13 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// Shared-memory matrix descriptor, 128-byte swizzle, tile rows of 128 bytes, 8-row groups 1024 bytes apart.
-// lbo: byte distance between 64-element blocks along the MN dimension (MN-major operands only).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr & 0x3FFFF) >> 4);
-  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
-  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
-  d |= (uint64_t)1 << 46;  // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;  // SWIZZLE_128B
-  return d;
+// Shared-memory matrix descriptor, 128-byte swizzle, tile rows of 128 bytes, 8-row groups 1024 bytes apart:
+// high word = stride between 8-row groups (1024 B >> 4), descriptor version bit, SWIZZLE_128B layout type;
+// low word = start address >> 4, and (bits 16-29) the byte distance >> 4 between 64-element blocks along the MN
+// dimension, which only MN-major operands use.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
+  return ((addr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
 }
 
 #ifdef SWAM_TC_TRACE
@@ -310,22 +313,26 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       bool ok = mbar_wait(bar_q, 0, abort_flag);
+      const uint32_t q_lo0 = desc_lo(sQ, 16), k_lo0 = desc_lo(sK, 16), v_lo0 = desc_lo(sV, C::kSubTile);
       auto issue_qk = [&](int s, int st) {
         // S_s = Q_s K^T : K dimension = D, 16 elements (32 bytes) per instruction inside the 128-byte swizzle row
+        const uint32_t a_lo = q_lo0 + ((uint32_t)(s * C::kTileBytes) >> 4), b_lo = k_lo0 + ((uint32_t)(st * C::kTileBytes) >> 4);
+        const uint32_t d = tm_S(s);
+        mma_ss<false>(d, a_lo, b_lo, kDescHi, C::kIdescQK);
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-          const uint32_t off = (ks >> 2) * C::kSubTile + (ks & 3) * 32;
-          mma_ss(tm_S(s), smem_desc(sQ + s * C::kTileBytes + off, 16, 1024), smem_desc(sK + st * C::kTileBytes + off, 16, 1024),
-                 C::kIdescQK, ks > 0);
+        for (int ks = 1; ks < D / 16; ++ks) {
+          constexpr int kSub16 = C::kSubTile >> 4;
+          const uint32_t off = (uint32_t)((ks >> 2) * kSub16 + (ks & 3) * 2);
+          mma_ss<true>(d, a_lo + off, b_lo + off, kDescHi, C::kIdescQK);
         }
       };
       auto issue_pv = [&](int s, int st, bool accum) {
         // O_s += P_s V : K dimension = 128 keys, 16 keys (two 8-row groups) per instruction; V is MN-major
+        const uint32_t b_lo = v_lo0 + ((uint32_t)(st * C::kTileBytes) >> 4);
+        const uint32_t d = tm_O(s), a = tm_S(s);
+        mma_ts(d, a, b_lo, kDescHi, C::kIdescPV, accum ? 1u : 0u);
 #pragma unroll
-        for (int kk = 0; kk < kTile / 16; ++kk) {
-          mma_ts(tm_O(s), tm_S(s) + kk * 8, smem_desc(sV + st * C::kTileBytes + kk * 2048, C::kSubTile, 1024), C::kIdescPV,
-                 (accum || kk > 0) ? 1u : 0u);
-        }
+        for (int kk = 1; kk < kTile / 16; ++kk) mma_ts(d, a + kk * 8, b_lo + kk * (2048 >> 4), kDescHi, C::kIdescPV, 1u);
       };
       if (ok) ok = mbar_wait(bar_k_full(0), 0, abort_flag);
       if (ok) {
