@@ -200,6 +200,9 @@ struct TcCfg {
   static constexpr int kSubTile = kTile * 128;      // bytes of one [128 rows x 64 cols] block
   static constexpr int kTileBytes = DB * kSubTile;  // one 128 x D tile
   static constexpr int kStages = (D == 128) ? 2 : 4;
+  // score buffers in TMEM: two at D = 128 (S0, S1, O0, O1 fill all 512 columns); at D = 64 the outputs need only 128
+  // columns, which leaves room for a third score buffer and lets Q K^T run one tile further ahead of the softmax
+  static constexpr int kSBufs = (D == 128) ? 2 : 3;
   static constexpr int kSmemData = 2 * kTileBytes + 2 * kStages * kTileBytes;
   static constexpr int kSmemBytes = kSmemData + 1024 /*alignment slack*/ + 256 /*barriers*/;
   static constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
@@ -225,11 +228,12 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   auto bar_k_empty = [&](int s) { return bars + 8 * (1 + ST + s); };
   auto bar_v_full = [&](int s) { return bars + 8 * (1 + 2 * ST + s); };
   auto bar_v_empty = [&](int s) { return bars + 8 * (1 + 3 * ST + s); };
-  auto bar_s_full = [&](int s) { return bars + 8 * (1 + 4 * ST + s); };
-  auto bar_p_full = [&](int s) { return bars + 8 * (3 + 4 * ST + s); };
-  const uint32_t bar_o_final = bars + 8 * (5 + 4 * ST);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + C::kSmemData + 8 * (6 + 4 * ST));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::kSmemData + 8 * (6 + 4 * ST) + 8);
+  constexpr int NB = C::kSBufs;
+  auto bar_s_full = [&](int buf) { return bars + 8 * (1 + 4 * ST + buf); };
+  auto bar_p_full = [&](int buf) { return bars + 8 * (4 + 4 * ST + buf); };
+  const uint32_t bar_o_final = bars + 8 * (7 + 4 * ST);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + C::kSmemData + 8 * (8 + 4 * ST));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::kSmemData + 8 * (8 + 4 * ST) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // work item = (sample, head, query tile pair), pair fastest.  Items below n_whole walk over all keys; the few items
@@ -258,9 +262,9 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       mbar_init(bar_v_full(s), 1);
       mbar_init(bar_v_empty(s), 1);
     }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(bar_s_full(s), 1);
-      mbar_init(bar_p_full(s), kTile);
+    for (int buf = 0; buf < NB; ++buf) {
+      mbar_init(bar_s_full(buf), 1);
+      mbar_init(bar_p_full(buf), kTile);
     }
     mbar_init(bar_o_final, 1);
     *abort_flag = 0;
@@ -274,9 +278,11 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+D) O1 [256+D, 256+2D); P_s overlays the first 64 columns of S_s
-  auto tm_S = [&](int s) { return tmem + (uint32_t)(s * kTile); };
-  auto tm_O = [&](int s) { return tmem + (uint32_t)(2 * kTile + s * D); };
+  // TMEM columns: NB score buffers of 128 columns, then O0 and O1 (D columns each): 512 in total for both head
+  // dims.  Work is a sequence of items i = 2 * tile + query tile; item i uses score buffer i % NB, and its P (bf16)
+  // overlays the first 64 columns of that buffer.
+  auto tm_S = [&](int buf) { return tmem + (uint32_t)(buf * kTile); };
+  auto tm_O = [&](int s) { return tmem + (uint32_t)(NB * kTile + s * D); };
 
   // register budget: the softmax warpgroups hold a whole S row per thread, the third warpgroup (MMA issuer, TMA
   // producer, two idle warps) needs almost nothing
@@ -314,10 +320,10 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     if (lane == 0) {
       bool ok = mbar_wait(bar_q, 0, abort_flag);
       const uint32_t q_lo0 = desc_lo(sQ, 16), k_lo0 = desc_lo(sK, 16), v_lo0 = desc_lo(sV, C::kSubTile);
-      auto issue_qk = [&](int s, int st) {
-        // S_s = Q_s K^T : K dimension = D, 16 elements (32 bytes) per instruction inside the 128-byte swizzle row
+      auto issue_qk = [&](int s, int buf, int st) {
+        // S = Q_s K^T : K dimension = D, 16 elements (32 bytes) per instruction inside the 128-byte swizzle row
         const uint32_t a_lo = q_lo0 + ((uint32_t)(s * C::kTileBytes) >> 4), b_lo = k_lo0 + ((uint32_t)(st * C::kTileBytes) >> 4);
-        const uint32_t d = tm_S(s);
+        const uint32_t d = tm_S(buf);
         mma_ss<false>(d, a_lo, b_lo, kDescHi, C::kIdescQK);
 #pragma unroll
         for (int ks = 1; ks < D / 16; ++ks) {
@@ -326,47 +332,50 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           mma_ss<true>(d, a_lo + off, b_lo + off, kDescHi, C::kIdescQK);
         }
       };
-      auto issue_pv = [&](int s, int st, bool accum) {
-        // O_s += P_s V : K dimension = 128 keys, 16 keys (two 8-row groups) per instruction; V is MN-major
+      auto issue_pv = [&](int s, int buf, int st, bool accum) {
+        // O_s += P V : K dimension = 128 keys, 16 keys (two 8-row groups) per instruction; V is MN-major
         const uint32_t b_lo = v_lo0 + ((uint32_t)(st * C::kTileBytes) >> 4);
-        const uint32_t d = tm_O(s), a = tm_S(s);
+        const uint32_t d = tm_O(s), a = tm_S(buf);
         mma_ts(d, a, b_lo, kDescHi, C::kIdescPV, accum ? 1u : 0u);
 #pragma unroll
         for (int kk = 1; kk < kTile / 16; ++kk) mma_ts(d, a + kk * 8, b_lo + kk * (2048 >> 4), kDescHi, C::kIdescPV, 1u);
       };
-      if (ok) ok = mbar_wait(bar_k_full(0), 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        issue_qk(0, 0);
-        tc_commit(bar_s_full(0));
-        issue_qk(1, 0);
-        tc_commit(bar_s_full(1));
-        tc_commit(bar_k_empty(0));
-      }
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int st = j % ST, st_next = (j + 1) % ST;
-        const uint32_t par_full = (j / ST) & 1, par_next = ((j + 1) / ST) & 1;
-        ok = mbar_wait(bar_v_full(st), par_full, abort_flag);
-        for (int s = 0; s < 2 && ok; ++s) {
-          TRACE(2, (j * 2 + s) * 4 + 0);
-          ok = mbar_wait(bar_p_full(s), j & 1, abort_flag);
-          if (!ok) break;
-          TRACE(2, (j * 2 + s) * 4 + 1);
+      // Items are issued in order: Q K^T of the first NB items up front, then for each item its P V followed by the
+      // Q K^T of item i + NB into the score buffer that P V has just consumed (the tensor pipe executes in issue
+      // order).  With three buffers the scores of a query tile's next key tile are ready before its softmax
+      // warpgroup has finished the current one.
+      const int n_items = 2 * n_tiles;
+      int k_waited = 0, v_waited = 0;
+      auto qk_item = [&](int it) -> bool {
+        const int j = it >> 1, sq = it & 1, st = j % ST;
+        if (j >= k_waited) {
+          if (!mbar_wait(bar_k_full(st), (j / ST) & 1, abort_flag)) return false;
+          k_waited = j + 1;
           tc_fence_after();
-          issue_pv(s, st, j > 0);
-          TRACE(2, (j * 2 + s) * 4 + 2);
-          if (j + 1 < n_tiles) {
-            if (s == 0) ok = mbar_wait(bar_k_full(st_next), par_next, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-            issue_qk(s, st_next);
-            tc_commit(bar_s_full(s));
-            TRACE(2, (j * 2 + s) * 4 + 3);
-          }
         }
+        issue_qk(sq, it % NB, st);
+        tc_commit(bar_s_full(it % NB));
+        if (sq == 1) tc_commit(bar_k_empty(st));   // both query tiles have used this key tile
+        return true;
+      };
+      for (int it = 0; it < NB && it < n_items && ok; ++it) ok = qk_item(it);
+      for (int it = 0; it < n_items && ok; ++it) {
+        const int j = it >> 1, sq = it & 1, st = j % ST, buf = it % NB;
+        if (j >= v_waited) {
+          ok = mbar_wait(bar_v_full(st), (j / ST) & 1, abort_flag);
+          if (!ok) break;
+          v_waited = j + 1;
+        }
+        TRACE(2, it * 4 + 0);
+        ok = mbar_wait(bar_p_full(buf), (it / NB) & 1, abort_flag);
         if (!ok) break;
-        tc_commit(bar_v_empty(st));
-        if (j + 1 < n_tiles) tc_commit(bar_k_empty(st_next));
+        TRACE(2, it * 4 + 1);
+        tc_fence_after();
+        issue_pv(sq, buf, st, j > 0);
+        TRACE(2, it * 4 + 2);
+        if (sq == 1) tc_commit(bar_v_empty(st));
+        if (it + NB < n_items) ok = qk_item(it + NB);
+        TRACE(2, it * 4 + 3);
       }
       if (ok) tc_commit(bar_o_final);
     }
@@ -377,12 +386,14 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const int s = warp >> 2;                 // query tile of this warpgroup
     const int r = (warp & 3) * 32 + lane;    // row inside the tile == TMEM lane
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tS = tm_S(s) + lane_off, tO = tm_O(s) + lane_off;
+    const uint32_t tO = tm_O(s) + lane_off;
     float m_used = -INFINITY, l_run = 0.f;
     bool ok = true;
     for (int j = 0; j < n_tiles; ++j) {
+      const int item = 2 * j + s, buf = item % NB;
+      const uint32_t tS = tm_S(buf) + lane_off;
       if (r == 0) TRACE(s, j * 8 + 0);
-      ok = mbar_wait(bar_s_full(s), j & 1, abort_flag);
+      ok = mbar_wait(bar_s_full(buf), (item / NB) & 1, abort_flag);
       if (!ok) break;
       if (r == 0) TRACE(s, j * 8 + 1);
       tc_fence_after();
@@ -476,7 +487,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       if (r == 0) TRACE(s, j * 8 + 3);
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(bar_p_full(s));
+      mbar_arrive(bar_p_full(buf));
       if (r == 0) TRACE(s, j * 8 + 4);
     }
     // epilogue
