@@ -70,3 +70,10 @@ def test_null_context_calls_fail_cleanly(lib):
     assert lib.swam_step(None, None, None, None, 0, None, None) == swam.ERR_INVALID_ARG
     assert lib.swam_check(None, None) == swam.ERR_INVALID_ARG
     assert lib.swam_last_error(None) == b"null context"
+
+
+def test_shapes_beyond_the_selection_kernels_shared_memory_are_rejected(lib):
+    from paper_2609_38984_b200 import swam
+    # F * N_s scores (two maps) + keys + flags must fit one SM's shared memory
+    assert _create(lib, n_frames=8, n_spatial=8192, n_action=32, k_core=10, k_anchor=10) == swam.ERR_UNSUPPORTED
+    assert _create(lib, n_obs=1 << 25) == swam.ERR_UNSUPPORTED            # sequence length limit

@@ -401,3 +401,50 @@ def test_single_layer_aggregation_is_identity():
     b = ctx.select_maps(v_core, v_all)
     for t, u in zip(a, b):
         assert torch.equal(t, u)
+
+
+# ------------------------------------------------------------------ more edge cases
+def test_cycle_replayed_from_a_cuda_graph_equals_eager():
+    """The step has a fixed shape, so a refresh cycle can be captured once and replayed (what bench.py times)."""
+    swam = _swam()
+    wl = small(batch=2)
+    steps = W.generate_steps(wl, 2)
+    d = [{n: dev(x[n], wl) for n in "qkv"} for x in steps]
+    eager, graphed = swam.Swam.from_workload(wl), swam.Swam.from_workload(wl)
+    out_e, out_g = eager.empty_full().zero_(), graphed.empty_full().zero_()
+
+    def cycle(ctx, out):
+        ctx.step(d[0]["q"], d[0]["k"], d[0]["v"], swam.REFRESH_FULL, out)
+        ctx.step(d[1]["q"], d[1]["k"], d[1]["v"], swam.REUSE, out)
+
+    cycle(eager, out_e)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        cycle(graphed, out_g)                      # warm-up outside capture
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    out_g.zero_()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        cycle(graphed, out_g)
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    graphed.check()
+    assert torch.equal(out_e, out_g)
+    for a, b in zip(eager.selection(), graphed.selection()):
+        assert torch.equal(a, b)
+
+
+def test_keep_nothing_leaves_only_observed_and_action_rows():
+    swam = _swam()
+    wl = small(k_core=0, k_anchor=0)
+    assert wl.packed_len == wl.n_obs + wl.n_action
+    steps = W.generate_steps(wl, 2)
+    ctx = swam.Swam.from_workload(wl)
+    compare_schedule(wl, steps, 2, run_schedule(ctx, wl, steps, 2))
+    _, pm, im = ctx.selection()
+    L = wl.seq_len
+    assert pm.cpu().numpy()[0].tolist() == list(range(wl.n_obs)) + list(range(L - wl.n_action, L))
+    assert int((im < 0).sum()) == wl.batch * wl.n_frames * wl.n_spatial
