@@ -21,7 +21,6 @@ namespace {
 constexpr int kTile = 128;          // query rows per tile and keys per tile
 constexpr int kThreadsTc = 384;     // 8 softmax warps + MMA warp + TMA warp + 2 idle warps (three full warpgroups)
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kRescaleThreshold = 8.0f;
 constexpr unsigned long long kWaitCycles = 4000000000ull;  // about two seconds at 1.9 GHz
 
 // ---------------------------------------------------------------------------------------------------------
@@ -447,7 +446,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         unpack2(add2(add2(acc2[0], acc2[1]), add2(acc2[2], acc2[3])), a0, a1);
         sum = a0 + a1;
       }
-      const bool grew = !(sum <= 256.f * 128.f);  // also catches inf and NaN
+      const bool grew = !(sum <= 256.f * 128.f);  // some exponent above 2^8 (or 128 of them near it); also catches inf, NaN
       if (__any_sync(0xffffffffu, grew)) {
         // rare: the row's true maximum relative to the reference
         float mraw = sv[0];

@@ -71,8 +71,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) row_copy_bulk_kernel(const Row
   long long issued = 0, stored = 0;  // lane 0's counters over valid units
   bool ok = true;
   // lane 0 keeps up to kStages - 1 loads in flight; src/dst offsets of issued-but-not-stored units
-  long long pend_dst[kStages];
-  int pend_z[kStages];
+  long long pend_dst[kStages] = {};
+  int pend_z[kStages] = {};
 
   auto retire_one = [&]() {  // wait for the oldest load, send it out, free one ring slot
     const int st = (int)(stored % kStages);
