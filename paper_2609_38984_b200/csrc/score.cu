@@ -47,13 +47,13 @@ struct ScoreParams {
   Alpha alpha;
 };
 
-constexpr int kScoreKeys = 32;  // keys per CTA: 2 m-tiles of 16
 
 // smem: query fragments [N_h][D/32][NT][32] uint4, lambda*log2e [N_h][NT*8], partial sums [4][32]
-template <int D, int NT, int kHeadGroups>
-__global__ void __launch_bounds__(64 * kHeadGroups, 8 / kHeadGroups) score_bf16_kernel(const ScoreParams p) {
+template <int D, int NT, int kHeadGroups, int MT>
+__global__ void __launch_bounds__(32 * MT * kHeadGroups, 16 / (MT * kHeadGroups)) score_bf16_kernel(const ScoreParams p) {
   constexpr int KB = D / 32;
-  constexpr int kScoreThreads = 64 * kHeadGroups;
+  constexpr int kScoreThreads = 32 * MT * kHeadGroups;
+  constexpr int kScoreKeys = 16 * MT;  // keys per CTA: MT m-tiles of 16
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint4* q_frag = reinterpret_cast<uint4*>(smem_raw);
   float* lam2 = reinterpret_cast<float*>(q_frag + (size_t)p.N_h * KB * NT * 32);
@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(64 * kHeadGroups, 8 / kHeadGroups) score_bf16_
     lam2[i] = (n < p.g) ? p.lse[((int64_t)b * p.N_h + h) * p.H + f * p.g + n] * kLog2e : 0.f;
   }
 
-  const int mt = warp & 1, hg = warp >> 1;
+  const int mt = warp % MT, hg = warp / MT;
   const int gq = lane >> 2, t = lane & 3;
   const int r0 = key0 + mt * 16 + gq, r1 = r0 + 8;
   const bool v0 = r0 < p.N_s, v1 = r1 < p.N_s;
@@ -424,22 +424,33 @@ __global__ void __launch_bounds__(128) lse_f32_kernel(const float* q, const floa
   }
 }
 
-template <int D, int NT, int HG>
+template <int D, int NT, int HG, int MT>
 cudaError_t launch_score_bf16_hg(const Dims& d, const ScoreParams& p, cudaStream_t st) {
+  constexpr int kScoreKeys = 16 * MT;
   const size_t smem = (size_t)d.N_h * (D / 32) * NT * 32 * sizeof(uint4) + (size_t)d.N_h * NT * 8 * sizeof(float) +
                       HG * kScoreKeys * sizeof(float);
   if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
-  cudaError_t e = cudaFuncSetAttribute(score_bf16_kernel<D, NT, HG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(score_bf16_kernel<D, NT, HG, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid((d.N_s + kScoreKeys - 1) / kScoreKeys, d.F, d.B);
-  score_bf16_kernel<D, NT, HG><<<grid, 64 * HG, smem, st>>>(p);
+  score_bf16_kernel<D, NT, HG, MT><<<grid, 32 * MT * HG, smem, st>>>(p);
   return cudaGetLastError();
 }
 
 template <int D, int NT>
 cudaError_t launch_score_bf16(const Dims& d, const ScoreParams& p, cudaStream_t st) {
-  return launch_score_bf16_hg<D, NT, 4>(d, p, st);
+  // 32 keys per CTA, except when that gives between one and two CTAs per SM: then 64-key CTAs (one per SM, half the
+  // query-fragment staging) finish sooner
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+  }
+  const long long n32 = (long long)((d.N_s + 31) / 32) * d.F * d.B;
+  if (n32 > sms && n32 <= 2 * sms) return launch_score_bf16_hg<D, NT, 4, 4>(d, p, st);
+  return launch_score_bf16_hg<D, NT, 4, 2>(d, p, st);
 }
 
 template <int D>
