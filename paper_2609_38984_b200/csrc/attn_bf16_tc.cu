@@ -65,9 +65,10 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t sr
   asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
                ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
+// the staging tile only has to stay alive until the copy engine has read it; the writes complete with the grid
 __device__ __forceinline__ void tma_store_commit_wait() {
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -172,6 +173,12 @@ __device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
 }
 
 #ifdef SWAM_TC_TRACE
+__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define CTA_T(k_) do { if (p.trace) p.trace[3 * 4096 + blockIdx.x * 4 + (k_)] = gtime(); } while (0)
+#else
+#define CTA_T(k_) do { } while (0)
+#endif
+#ifdef SWAM_TC_TRACE
 #define TRACE(slot_, idx_) do { if (blockIdx.x == 0 && p.trace) p.trace[(slot_) * 4096 + (idx_)] = clock64(); } while (0)
 #else
 #define TRACE(slot_, idx_) do { } while (0)
@@ -253,6 +260,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const int row0 = pair * 2 * kTile;
   const int n_tiles = kv_end - kv_begin;  // >= 1 by construction
 
+  if (threadIdx.x == 0) CTA_T(0);
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
     for (int s = 0; s < ST; ++s) {
@@ -395,6 +403,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       ok = mbar_wait(bar_s_full(buf), (item / NB) & 1, abort_flag);
       if (!ok) break;
       if (r == 0) TRACE(s, j * 8 + 1);
+      if (r == 0 && s == 0 && j == 0) CTA_T(1);
       tc_fence_after();
       float sv[kTile];
 #pragma unroll
@@ -491,6 +500,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     }
     // epilogue
     if (ok) ok = mbar_wait(bar_o_final, 0, abort_flag);
+    if (r == 0 && s == 0) CTA_T(2);
     if (slot >= 0) {
       // a piece of a split item: unnormalised O, reference max and sum go to scratch; the combine kernel finishes
       if (ok) {
@@ -547,6 +557,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) CTA_T(3);
   if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, ST_TIMEOUT);
   if (warp == 8) {
     tc_fence_after();
@@ -647,7 +658,7 @@ bool make_map(CUtensorMap* map, const void* ptr, int B, int n, int N_h, int D) {
 #ifdef SWAM_TC_TRACE
 void* g_trace = nullptr;
 void* partial_trace_buffer() {
-  if (!g_trace) { cudaMalloc(&g_trace, 3 * 4096 * 8); cudaMemset(g_trace, 0, 3 * 4096 * 8); }
+  if (!g_trace) { cudaMalloc(&g_trace, 8 * 4096 * 8); cudaMemset(g_trace, 0, 8 * 4096 * 8); }
   return g_trace;
 }
 #endif
@@ -705,7 +716,7 @@ cudaError_t launch_tc_d(const AttnArgs& a, int* status, float* partial, size_t p
 }  // namespace
 
 #ifdef SWAM_TC_TRACE
-extern "C" void swam_debug_trace(long long* host) { cudaMemcpy(host, g_trace, 3 * 4096 * 8, cudaMemcpyDeviceToHost); }
+extern "C" void swam_debug_trace(long long* host) { cudaMemcpy(host, g_trace, 8 * 4096 * 8, cudaMemcpyDeviceToHost); }
 #endif
 
 size_t attn_tc_scratch_bytes(int D) {
