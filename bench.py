@@ -33,8 +33,11 @@ from paper_2609_38984_b200 import workloads as W  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel's launches in one cycle (dense launch + packed
-# launch), from the ncu capture summarised in profiles/attn_bf16_tc_larger_imagination.txt
-DOMINANT_KERNEL_DRAM_BYTES = {"larger_imagination": int((228.264192 + 57.030400 + 87.169280 + 13.018368) * 1e6)}
+# launch), from the ncu captures summarised in profiles/attn_bf16_tc_*.txt
+DOMINANT_KERNEL_DRAM_BYTES = {
+    "larger_imagination": int((228.174336 + 56.776192 + 87.152896 + 10.919168) * 1e6),
+    "multi_view": int((639.898880 + 198.045696 + 257.214464 + 71.534336) * 1e6),   # profiles/attn_bf16_tc_multi_view.txt
+}
 
 
 def load_peaks():
@@ -296,10 +299,15 @@ def bench_swam(args):
         att_flops = algo["attn_dense"][1] + (R - 1) * algo["attn_packed"][1]
         att_us = stage_us["attn_dense"] + (R - 1) * stage_us["attn_packed"]
         achieved = att_flops / (att_us * 1e-6) / 1e12
-        # fp32 tensors run on the FMA pipes; the tensor peak only applies to bf16
-        roofline = {"kernel": "joint attention (dense + packed launches of one cycle)", "bound": "tensor" if wl.dtype == W.BF16 else "alu",
-                    "achieved": round(achieved, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                    "frac": round(achieved / peaks["bf16_tflops"], 4), "peak_source": f"{peak_kind} (burst)",
+        # fp32 tensors run on the FMA pipes: peak = 148 SMs x 128 FP32 lanes x 2 flop x 1.965 GHz (nominal unit counts
+        # and the maximum SM clock); the measured tensor peak only applies to bf16
+        if wl.dtype == W.BF16:
+            bound, peak, src = "tensor", peaks["bf16_tflops"], f"{peak_kind} (burst)"
+        else:
+            bound, peak, src = "alu", 148 * 128 * 2 * 1.965e9 / 1e12, "derived: 148 SMs x 128 lanes x 2 x 1.965 GHz"
+        roofline = {"kernel": "joint attention (dense + packed launches of one cycle)", "bound": bound,
+                    "achieved": round(achieved, 2), "peak": round(peak, 1), "unit": "TFLOP/s",
+                    "frac": round(achieved / peak, 4), "peak_source": src,
                     "traffic": DOMINANT_KERNEL_DRAM_BYTES.get(wl0.name)}
         cpu = cpu_baseline(wl, host_steps, budget_s=args.cpu_seconds)
         line = {
