@@ -2,15 +2,19 @@
 //
 // One CTA owns two 128-row query tiles of one (sample, head) and walks over the keys in tiles of 128:
 //   warp 9      TMA producer: Q once, then K_j / V_j into a ring of shared-memory stages (128B-swizzled boxes)
-//   warp 8      one elected thread issues every tcgen05.mma: S_s = Q_s K_j^T (both operands K-major in shared
-//               memory) into TMEM, then O_s += P_s V_j with P_s read from TMEM and V_j as an MN-major operand
-//   warps 0-3   softmax of query tile 0: one thread per row reads its S row from TMEM, keeps the running max and
-//   warps 4-7   sum (exp2 domain), writes P as bf16 back over S; same for query tile 1
-// The two query tiles alternate on the tensor pipe, so one tile's exponentials overlap the other tile's MMAs.
-// O stays in TMEM for the whole key loop; it is rescaled only when a row's maximum has grown by more than 2^8
-// since the value its exponentials refer to (the result is exact either way: sums and outputs share the same
-// reference maximum).  Every wait on an mbarrier is bounded; when a wait runs out the kernel raises the timeout
-// bit of the status word, stops issuing work, and every role falls through to the common exit.
+//   warp 8      one elected thread issues every tcgen05.mma: S = Q_s K_j^T (both operands K-major in shared
+//               memory) into a TMEM score buffer, then O_s += P V_j with P read from TMEM and V_j as an MN-major
+//               operand
+//   warps 0-3   softmax of query tile 0: one thread per row reads its S row from TMEM, keeps the reference maximum
+//   warps 4-7   and the running sum (exp2 domain), writes P as bf16 back over S; same for query tile 1
+//   warps 10-11 idle (they complete the third warpgroup, which hands most of its registers to the softmax warps)
+// Work is a sequence of items (key tile, query tile); item i uses score buffer i mod NB (NB = 2 at head dim 128,
+// 3 at head dim 64) and the issuing thread keeps Q K^T NB items ahead of P V, so one tile's exponentials overlap the
+// other tile's MMAs.  O stays in TMEM for the whole key loop; it is rescaled only when a row's maximum has grown by
+// more than 2^8 beyond the value its exponentials refer to (the result is exact either way: sums and outputs share
+// the same reference maximum).  Work items left over after the last full wave of CTAs are cut over the keys and
+// merged by a small combine kernel.  Every wait on an mbarrier is bounded; when a wait runs out the kernel raises
+// the timeout bit of the status word, stops issuing work, and every role falls through to the common exit.
 #include <cuda.h>
 
 #include "swam_internal.cuh"
