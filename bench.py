@@ -144,9 +144,10 @@ def per_launch_us(fns, reps):
 
 def bench_swam(args):
     from paper_2609_38984_b200 import swam
-    rank, local_rank, world = sd.init("nccl")
-    torch.cuda.set_device(local_rank)
+    _, local_rank, _ = sd.env_rank()
+    torch.cuda.set_device(local_rank)            # before the process group, so NCCL binds this rank to its own GPU
     device = torch.device("cuda", local_rank)
+    rank, local_rank, world = sd.init("nccl")
     wl0 = W.WORKLOADS[args.workload]
     wl = sd.rank_workload(wl0, rank, world)
     R = wl.refresh
