@@ -211,6 +211,7 @@ def bench_swam(args):
     e0.record()
     for _ in range(e2e_steps):
         cycle_host()
+    ctx.host_join()      # the timed region ends when the last result has arrived in host memory
     e1.record()
     torch.cuda.synchronize()
     sd.barrier(device)

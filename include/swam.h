@@ -141,14 +141,22 @@ int swam_scatter(swam_ctx* ctx, const void* out_p, const int32_t* pack_map, cons
  * then runs the sparse step with the new maps. */
 int swam_step(swam_ctx* ctx, const void* q, const void* k, const void* v, int32_t mode, void* out, void* stream);
 
-/* The same step for callers whose tensors live in (pinned) host memory: copies q, k, v into a device staging
- * area, runs swam_step, copies out back; all on `stream`, no synchronisation.  The staging area (4 full
- * tensors, caller-allocated, dev) is bound once; on SWAM_REUSE steps the staged out of the previous step is
- * the cache, so staging must not be touched between steps. */
+/* The same step for callers whose tensors live in (pinned) host memory.  The call enqueues a three-stage pipeline
+ * and does not synchronise: q, k, v travel to a device staging slot on an internal copy stream, swam_step runs on
+ * `stream`, and out leaves for out_host on a second internal copy stream, so that consecutive calls overlap one
+ * step's copies with the neighbouring steps' compute and the two PCIe directions with each other.  The staging area
+ * (7 full tensors: two input slots and the persistent out; caller-allocated, dev) is bound once; binding creates the
+ * internal streams and events.  The host input buffers of a call must stay unchanged, and out_host is complete,
+ * once swam_check (which also waits for the internal streams) or a device-wide synchronisation has returned.  On
+ * SWAM_REUSE steps the staged out of the previous step is the cache, so the staging area must not be touched between
+ * steps.  Not capturable in a CUDA graph. */
 int swam_host_io_bytes(const swam_ctx* ctx, size_t* bytes);
 int swam_bind_host_io(swam_ctx* ctx, void* dev_ptr, size_t bytes);
 int swam_step_host(swam_ctx* ctx, const void* q_host, const void* k_host, const void* v_host, int32_t mode,
                    void* out_host, void* stream);
+/* Makes `stream` wait (on the device, without blocking the host) until the result of the most recent
+ * swam_step_host call has arrived in its out_host; work enqueued on `stream` afterwards may read out_host. */
+int swam_host_join(swam_ctx* ctx, void* stream);
 
 /* Device pointers (inside the workspace) of the state swam_step keeps; any argument may be NULL. */
 int swam_get_selection(const swam_ctx* ctx, const int32_t** sel_idx, const int32_t** pack_map,

@@ -21,9 +21,13 @@ struct swam_ctx {
       off_vp, off_op, off_attn, attn_scratch, ws_need;
   bool has_selection;
   int attn_variant;  // SWAM_ATTN_AUTO | SWAM_ATTN_WARP_MMA
-  // host-io staging (device)
+  // host-io staging (device): two input slots of (q, k, v) and the persistent output, plus the copy pipeline
   unsigned char* io;
   size_t io_need;
+  cudaStream_t s_in, s_out;           // host-to-device and device-to-host copy streams
+  cudaEvent_t ev_h2d[2], ev_done[2];  // per input slot: inputs arrived / step finished with the slot
+  cudaEvent_t ev_d2h;                 // the previous result has left the staged output
+  int64_t host_steps;
   int launches_i;
   int64_t launches;
   char err[256];
@@ -150,12 +154,18 @@ int swam_create(const swam_shape* s, swam_ctx** out_ctx) {
   c->attn_scratch = (d.dtype == SWAM_BF16 && d.D >= 64) ? attn_tc_scratch_bytes(d.D) : 0;
   c->off_attn = put(c->attn_scratch);
   c->ws_need = off;
-  c->io_need = 4 * align_up(full_bytes(d), 256);
+  c->io_need = 7 * align_up(full_bytes(d), 256);
   *out_ctx = c;
   return SWAM_OK;
 }
 
 int swam_destroy(swam_ctx* ctx) {
+  if (ctx && ctx->s_in) {
+    cudaStreamDestroy(ctx->s_in);
+    cudaStreamDestroy(ctx->s_out);
+    for (int i = 0; i < 2; ++i) { cudaEventDestroy(ctx->ev_h2d[i]); cudaEventDestroy(ctx->ev_done[i]); }
+    cudaEventDestroy(ctx->ev_d2h);
+  }
   delete ctx;
   return SWAM_OK;
 }
@@ -191,7 +201,19 @@ int swam_bind_host_io(swam_ctx* c, void* dev_ptr, size_t bytes) {
   if (!c || !dev_ptr) return SWAM_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(dev_ptr) & 255u) != 0) return fail(c, SWAM_ERR_INVALID_ARG, "staging not 256-byte aligned");
   if (bytes < c->io_need) return fail(c, SWAM_ERR_WORKSPACE, "staging area too small");
+  if (int r = check_device(c)) return r;
+  if (!c->s_in) {
+    cudaError_t e = cudaStreamCreateWithFlags(&c->s_in, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->s_out, cudaStreamNonBlocking);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+      e = cudaEventCreateWithFlags(&c->ev_h2d[i], cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_done[i], cudaEventDisableTiming);
+    }
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_d2h, cudaEventDisableTiming);
+    if (e != cudaSuccess) return fail_cuda(c, e, "swam_bind_host_io: stream/event creation");
+  }
   c->io = (unsigned char*)dev_ptr;
+  c->host_steps = 0;
   return SWAM_OK;
 }
 
@@ -361,17 +383,38 @@ int swam_step_host(swam_ctx* c, const void* q_host, const void* k_host, const vo
   if (!c->io) return fail(c, SWAM_ERR_WORKSPACE, "swam_step_host: no staging area bound");
   cudaStream_t st = (cudaStream_t)stream;
   const size_t fb = full_bytes(c->d), stride = align_up(fb, 256);
-  void* dq = c->io;
-  void* dk = c->io + stride;
-  void* dv = c->io + 2 * stride;
-  void* dout = c->io + 3 * stride;
-  cudaError_t e = cudaMemcpyAsync(dq, q_host, fb, cudaMemcpyHostToDevice, st);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(dk, k_host, fb, cudaMemcpyHostToDevice, st);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v_host, fb, cudaMemcpyHostToDevice, st);
+  // Three-stage pipeline over two input slots: this step's inputs travel on the copy-in stream while the previous
+  // step still computes, the step runs on the caller's stream, and the result leaves on the copy-out stream while
+  // the next inputs arrive (PCIe is full duplex).
+  const int slot = (int)(c->host_steps & 1);
+  unsigned char* in = c->io + (size_t)slot * 3 * stride;
+  void* dq = in;
+  void* dk = in + stride;
+  void* dv = in + 2 * stride;
+  void* dout = c->io + 6 * stride;
+  cudaError_t e = cudaStreamWaitEvent(c->s_in, c->ev_done[slot], 0);   // the step two calls ago has read this slot
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dq, q_host, fb, cudaMemcpyHostToDevice, c->s_in);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dk, k_host, fb, cudaMemcpyHostToDevice, c->s_in);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v_host, fb, cudaMemcpyHostToDevice, c->s_in);
+  if (e == cudaSuccess) e = cudaEventRecord(c->ev_h2d[slot], c->s_in);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_h2d[slot], 0);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_d2h, 0);     // the previous result has been copied out
   if (e != cudaSuccess) return fail_cuda(c, e, "host to device copy");
   if (int r = swam_step(c, dq, dk, dv, mode, dout, stream)) return r;
-  e = cudaMemcpyAsync(out_host, dout, fb, cudaMemcpyDeviceToHost, st);
+  e = cudaEventRecord(c->ev_done[slot], st);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(c->s_out, c->ev_done[slot], 0);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(out_host, dout, fb, cudaMemcpyDeviceToHost, c->s_out);
+  if (e == cudaSuccess) e = cudaEventRecord(c->ev_d2h, c->s_out);
   if (e != cudaSuccess) return fail_cuda(c, e, "device to host copy");
+  ++c->host_steps;
+  return SWAM_OK;
+}
+
+int swam_host_join(swam_ctx* c, void* stream) {
+  if (!c) return SWAM_ERR_INVALID_ARG;
+  if (!c->s_in) return fail(c, SWAM_ERR_WORKSPACE, "swam_host_join: no staging area bound");
+  cudaError_t e = cudaStreamWaitEvent((cudaStream_t)stream, c->ev_d2h, 0);
+  if (e != cudaSuccess) return fail_cuda(c, e, "swam_host_join");
   return SWAM_OK;
 }
 
@@ -395,6 +438,8 @@ int swam_check(swam_ctx* c, void* stream) {
   if (!c) return SWAM_ERR_INVALID_ARG;
   if (int r = need_ws(c)) return r;
   cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e == cudaSuccess && c->s_in) e = cudaStreamSynchronize(c->s_in);
+  if (e == cudaSuccess && c->s_out) e = cudaStreamSynchronize(c->s_out);
   if (e != cudaSuccess) return fail_cuda(c, e, "cudaStreamSynchronize");
   int word = 0;
   e = cudaMemcpy(&word, c->ws + c->off_status, sizeof(int), cudaMemcpyDeviceToHost);

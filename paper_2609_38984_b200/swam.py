@@ -27,7 +27,7 @@ EXPORTS = [
     "swam_create", "swam_destroy", "swam_workspace_bytes", "swam_bind_workspace", "swam_score", "swam_score_noalloc",
     "swam_select", "swam_aggregate", "swam_select_maps",
     "swam_pack", "swam_sparse_attn", "swam_scatter", "swam_step", "swam_host_io_bytes", "swam_bind_host_io",
-    "swam_step_host", "swam_get_selection", "swam_get_scores", "swam_check", "swam_set_option", "swam_launch_count",
+    "swam_step_host", "swam_host_join", "swam_get_selection", "swam_get_scores", "swam_check", "swam_set_option", "swam_launch_count",
     "swam_last_error", "swam_version",
 ]
 
@@ -76,6 +76,7 @@ def load_library() -> ctypes.CDLL:
         lib.swam_scatter.argtypes = [vp] * 7
         lib.swam_step.argtypes = [vp, vp, vp, vp, i32, vp, vp]
         lib.swam_step_host.argtypes = [vp, vp, vp, vp, i32, vp, vp]
+        lib.swam_host_join.argtypes = [vp, vp]
         lib.swam_get_selection.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
         lib.swam_get_scores.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
         lib.swam_check.argtypes = [vp, vp]
@@ -253,6 +254,10 @@ class Swam:
         self._chk(self.lib.swam_step_host(self.ctx, _ptr(q_host), _ptr(k_host), _ptr(v_host), mode, _ptr(out_host),
                                           _stream()))
         return out_host
+
+    def host_join(self):
+        """The current stream waits for the last step_host result to arrive in its host buffer."""
+        self._chk(self.lib.swam_host_join(self.ctx, _stream()))
 
     def _view(self, ptr: ctypes.c_void_p, shape, dtype) -> torch.Tensor:
         off = ptr.value - self.workspace.data_ptr()

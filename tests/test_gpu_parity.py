@@ -351,6 +351,27 @@ def test_host_buffer_step_matches_device_step():
         assert torch.equal(out_dev.cpu(), out_host)
 
 
+def test_host_buffer_steps_pipeline_without_synchronising_in_between():
+    swam = _swam()
+    wl = small(steps=5)
+    steps = W.generate_steps(wl)
+    ctx_a, ctx_b = swam.Swam.from_workload(wl), swam.Swam.from_workload(wl)
+    out_dev = ctx_a.empty_full()
+    tdt = out_dev.dtype
+    host_in = [[torch.from_numpy(x[n]).to(tdt).pin_memory() for n in "qkv"] for x in steps]
+    host_out = [torch.empty(out_dev.shape, dtype=tdt).pin_memory() for _ in steps]
+    want = []
+    for t, (hq, hk, hv) in enumerate(host_in):
+        mode = swam.REFRESH_FULL if t % 2 == 0 else swam.REUSE
+        ctx_a.step(hq.cuda(), hk.cuda(), hv.cuda(), mode, out_dev)
+        want.append(out_dev.cpu().clone())
+    for t, (hq, hk, hv) in enumerate(host_in):          # five calls enqueued back to back
+        ctx_b.step_host(hq, hk, hv, swam.REFRESH_FULL if t % 2 == 0 else swam.REUSE, host_out[t])
+    ctx_b.check()
+    for t in range(len(steps)):
+        assert torch.equal(want[t], host_out[t]), t
+
+
 # ------------------------------------------------------------------ several profiled layers (Eq. 3, Eq. 9, Eq. 11)
 @pytest.mark.parametrize("wl,n_layers,k_layer", [
     (small(batch=2), 5, 2),
