@@ -195,6 +195,8 @@ struct TcParams {
   float* lse;
   int* status;
   float* partial;      // split items: [slot][2 tiles][128 rows][D + 4]: unnormalised O, then reference max and sum
+  const int32_t* pack_map;  // scatter mode: [B, n] row of the full output tensor that each attended row is written to
+  int n_full;               // scatter mode: rows per sample of the full output tensor
   int lse_row0, lse_rows;
   int n, N_h;
   int pairs;           // query tile pairs per (sample, head)
@@ -219,7 +221,11 @@ struct TcCfg {
   static constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(D >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
 };
 
-template <int D>
+// SCATTER = false: map_o covers the [B, n, N_h, D] output in boxes of 128 rows, one store per query tile.
+// SCATTER = true (Eq. 7 fused into the packed attention): map_o covers the FULL [B, n_full, N_h, D] output in boxes of
+// one row, and each attended row goes straight to its original position pack_map[b, row]; the rows the packed sequence
+// omits are never touched and keep the cached values they hold.
+template <int D, bool SCATTER>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o, const TcParams p) {
@@ -550,11 +556,28 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         p.lse[((int64_t)b * p.N_h + h) * p.lse_rows + (row - p.lse_row0)] = (m_used + log2f(l_run)) * 0.6931471805599453f;
       fence_proxy_async();
     }
-    asm volatile("bar.sync %0, 128;" ::"r"(1 + s) : "memory");  // the four warps of this query tile
-    if (ok && (warp & 3) == 0 && lane == 0 && row0 + s * kTile < p.n) {
-      for (int db = 0; db < C::DB; ++db)
-        tma_store_4d(&map_o, sQ + s * C::kTileBytes + db * C::kSubTile, db * 64, row0 + s * kTile, h, b);
-      tma_store_commit_wait();
+    if (SCATTER) {
+      // each thread sends the row it has just staged (it reads only its own writes, so its own proxy fence is all the
+      // ordering the copy engine needs); the 128-byte swizzle is a function of the shared-memory address, so a
+      // one-row box at the row's offset reads the same bytes the 128-row box would
+      const int prow = row0 + s * kTile + r;
+      if (ok && prow < p.n) {
+        const int orow = p.pack_map[(int64_t)b * p.n + prow];
+        if (orow >= 0 && orow < p.n_full) {
+          for (int db = 0; db < C::DB; ++db)
+            tma_store_4d(&map_o, sQ + s * C::kTileBytes + db * C::kSubTile + r * 128, db * 64, orow, h, b);
+          tma_store_commit_wait();
+        } else {
+          atomicOr(p.status, ST_BAD_MAP);
+        }
+      }
+    } else {
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + s) : "memory");  // the four warps of this query tile
+      if (ok && (warp & 3) == 0 && lane == 0 && row0 + s * kTile < p.n) {
+        for (int db = 0; db < C::DB; ++db)
+          tma_store_4d(&map_o, sQ + s * C::kTileBytes + db * C::kSubTile, db * 64, row0 + s * kTile, h, b);
+        tma_store_commit_wait();
+      }
     }
     }
   }
@@ -572,6 +595,9 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 // Merges the pieces of the split items: out = sum_i 2^(m_i - m) O_i / sum_i 2^(m_i - m) l_i, one warp per query row.
 struct CombineParams {
   const float* partial;
+  const int32_t* pack_map;  // scatter mode: out is the full tensor and row goes to pack_map[b, row]; nullptr otherwise
+  int n_full;
+  int* status;
   __nv_bfloat16* out;
   float* lse;
   int lse_row0, lse_rows;
@@ -619,7 +645,16 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const CombineParams p
     for (int c = 0; c < CPL; ++c) acc[c] += w * v[i][c];
   }
   const float inv = 1.f / l;
-  __nv_bfloat16* o = p.out + (((int64_t)b * p.n + row) * p.N_h + h) * D + lane * CPL;
+  int64_t out_row = (int64_t)b * p.n + row;
+  if (p.pack_map) {
+    const int orow = p.pack_map[(int64_t)b * p.n + row];
+    if (orow < 0 || orow >= p.n_full) {
+      if (lane == 0) atomicOr(p.status, ST_BAD_MAP);
+      return;
+    }
+    out_row = (int64_t)b * p.n_full + orow;
+  }
+  __nv_bfloat16* o = p.out + (out_row * p.N_h + h) * D + lane * CPL;
 #pragma unroll
   for (int c = 0; c < CPL; c += 2)
     *reinterpret_cast<__nv_bfloat162*>(o + c) = __floats2bfloat162_rn(acc[c] * inv, acc[c + 1] * inv);
@@ -646,13 +681,13 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// [B, n, N_h, D] bf16 viewed as a 4-D tensor (d, row, head, sample); box = 64 columns x 128 rows, 128-byte swizzle
-bool make_map(CUtensorMap* map, const void* ptr, int B, int n, int N_h, int D) {
+// [B, n, N_h, D] bf16 viewed as a 4-D tensor (d, row, head, sample); box = 64 columns x box_rows rows, 128-byte swizzle
+bool make_map(CUtensorMap* map, const void* ptr, int B, int n, int N_h, int D, int box_rows = kTile) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)n, (cuuint64_t)N_h, (cuuint64_t)B};
   const cuuint64_t strides[3] = {(cuuint64_t)N_h * D * 2, (cuuint64_t)D * 2, (cuuint64_t)n * N_h * D * 2};
-  const cuuint32_t box[4] = {64, (cuuint32_t)kTile, 1, 1};
+  const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -677,13 +712,16 @@ int sm_count_tc() {
   return sms;
 }
 
-template <int D>
-cudaError_t launch_tc_d(const AttnArgs& a, int* status, float* partial, size_t partial_bytes, cudaStream_t st, int* launches) {
+// SCATTER: a.out is the full [B, n_full, N_h, D] tensor and pack_map [B, a.n] names the row each attended row goes to.
+template <int D, bool SCATTER>
+cudaError_t launch_tc_d(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, float* partial,
+                        size_t partial_bytes, cudaStream_t st, int* launches) {
   CUtensorMap mq, mk, mv, mo;
   if (!make_map(&mq, a.q, a.B, a.n, a.N_h, D) || !make_map(&mk, a.k, a.B, a.n, a.N_h, D) ||
-      !make_map(&mv, a.v, a.B, a.n, a.N_h, D) || !make_map(&mo, a.out, a.B, a.n, a.N_h, D))
+      !make_map(&mv, a.v, a.B, a.n, a.N_h, D) ||
+      !(SCATTER ? make_map(&mo, a.out, a.B, n_full, a.N_h, D, 1) : make_map(&mo, a.out, a.B, a.n, a.N_h, D)))
     return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(attn_bf16_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<D>::kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(attn_bf16_tc_kernel<D, SCATTER>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<D>::kSmemBytes);
   if (e != cudaSuccess) return e;
   const int pairs = (a.n + 2 * kTile - 1) / (2 * kTile);
   const int items = pairs * a.N_h * a.B;
@@ -705,13 +743,15 @@ cudaError_t launch_tc_d(const AttnArgs& a, int* status, float* partial, size_t p
 #ifdef SWAM_TC_TRACE
       (long long*)partial_trace_buffer(),
 #endif
-      a.lse, status, partial, a.lse_row0, a.lse_rows, a.n, a.N_h, pairs, n_whole, splits, per, a.scale * kLog2e};
+      a.lse, status, partial, pack_map, n_full, a.lse_row0, a.lse_rows, a.n, a.N_h, pairs, n_whole, splits, per,
+      a.scale * kLog2e};
   const int grid = n_whole + (splits ? rem * splits : 0);
   ++*launches;
-  attn_bf16_tc_kernel<D><<<grid, kThreadsTc, TcCfg<D>::kSmemBytes, st>>>(mq, mk, mv, mo, p);
+  attn_bf16_tc_kernel<D, SCATTER><<<grid, kThreadsTc, TcCfg<D>::kSmemBytes, st>>>(mq, mk, mv, mo, p);
   e = cudaGetLastError();
   if (e != cudaSuccess || !splits) return e;
-  CombineParams c{partial, (__nv_bfloat16*)a.out, a.lse, a.lse_row0, a.lse_rows, a.n, a.N_h, D, pairs, n_whole, splits, rem};
+  CombineParams c{partial, SCATTER ? pack_map : nullptr, n_full, status, (__nv_bfloat16*)a.out, a.lse, a.lse_row0, a.lse_rows,
+                  a.n, a.N_h, D, pairs, n_whole, splits, rem};
   ++*launches;
   attn_combine_kernel<D><<<(rem * 2 * kTile + 7) / 8, 256, 0, st>>>(c);
   return cudaGetLastError();
@@ -731,8 +771,17 @@ size_t attn_tc_scratch_bytes(int D) {
 cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, void* scratch, size_t scratch_bytes, cudaStream_t st,
                                 int* launches) {
   switch (a.D) {
-    case 64: return launch_tc_d<64>(a, status, (float*)scratch, scratch_bytes, st, launches);
-    case 128: return launch_tc_d<128>(a, status, (float*)scratch, scratch_bytes, st, launches);
+    case 64: return launch_tc_d<64, false>(a, nullptr, a.n, status, (float*)scratch, scratch_bytes, st, launches);
+    case 128: return launch_tc_d<128, false>(a, nullptr, a.n, status, (float*)scratch, scratch_bytes, st, launches);
+    default: return cudaErrorInvalidConfiguration;
+  }
+}
+
+cudaError_t launch_attn_bf16_tc_scatter(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, void* scratch,
+                                        size_t scratch_bytes, cudaStream_t st, int* launches) {
+  switch (a.D) {
+    case 64: return launch_tc_d<64, true>(a, pack_map, n_full, status, (float*)scratch, scratch_bytes, st, launches);
+    case 128: return launch_tc_d<128, true>(a, pack_map, n_full, status, (float*)scratch, scratch_bytes, st, launches);
     default: return cudaErrorInvalidConfiguration;
   }
 }

@@ -21,6 +21,7 @@ struct swam_ctx {
       off_vp, off_op, off_attn, attn_scratch, ws_need;
   bool has_selection;
   int attn_variant;  // SWAM_ATTN_AUTO | SWAM_ATTN_WARP_MMA
+  int sparse_path;   // SWAM_SPARSE_FUSED | SWAM_SPARSE_STAGED
   // host-io staging (device): two input slots of (q, k, v) and the persistent output, plus the copy pipeline
   unsigned char* io;
   size_t io_need;
@@ -365,7 +366,20 @@ int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t 
     if (int r = swam_select(c, scores, sel, pm, im, stream)) return r;
     c->has_selection = true;
   }
-  if (mode != SWAM_REFRESH_FULL) {
+  if (mode != SWAM_REFRESH_FULL && c->sparse_path == SWAM_SPARSE_FUSED && d.dtype == SWAM_BF16 && d.D >= 64 &&
+      c->attn_variant == SWAM_ATTN_AUTO) {
+    // packed attention writes each retained row straight to its place in `out`; the omitted rows keep the cached
+    // value they already hold (Eq. 7), so no packed output and no scatter pass exist
+    void* qp = c->ws + c->off_qp;
+    void* kp = c->ws + c->off_kp;
+    void* vp = c->ws + c->off_vp;
+    if (int r = swam_pack(c, q, k, v, pm, qp, kp, vp, stream)) return r;
+    AttnArgs a{qp, kp, vp, out, nullptr, 0, 0, d.B, d.Lp, d.N_h, d.D, d.scale};
+    cudaError_t e = launch_attn_bf16_tc_scatter(a, pm, d.L, (int*)(c->ws + c->off_status), c->ws + c->off_attn,
+                                                c->attn_scratch, st, &c->launches_i);
+    count(c);
+    if (e != cudaSuccess) return fail_cuda(c, e, "fused sparse attention launch");
+  } else if (mode != SWAM_REFRESH_FULL) {
     void* qp = c->ws + c->off_qp;
     void* kp = c->ws + c->off_kp;
     void* vp = c->ws + c->off_vp;
@@ -458,6 +472,10 @@ int swam_set_option(swam_ctx* c, int32_t option, int32_t value) {
   if (!c) return SWAM_ERR_INVALID_ARG;
   if (option == SWAM_OPT_ATTN_VARIANT && (value == SWAM_ATTN_AUTO || value == SWAM_ATTN_WARP_MMA)) {
     c->attn_variant = value;
+    return SWAM_OK;
+  }
+  if (option == SWAM_OPT_SPARSE_PATH && (value == SWAM_SPARSE_FUSED || value == SWAM_SPARSE_STAGED)) {
+    c->sparse_path = value;
     return SWAM_OK;
   }
   return fail(c, SWAM_ERR_INVALID_ARG, "swam_set_option: unknown option or value");

@@ -76,5 +76,10 @@ cudaError_t launch_attn_bf16_mma(const AttnArgs& a, cudaStream_t st, int* launch
 size_t attn_tc_scratch_bytes(int D);
 cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, void* scratch, size_t scratch_bytes, cudaStream_t st,
                                 int* launches);
+// Packed attention with Eq. 7's scatter fused into the epilogue: q, k, v are the packed tensors [B, a.n, N_h, D];
+// a.out is the FULL output tensor [B, n_full, N_h, D], and attended row i of sample b is written to row
+// pack_map[b, i] of it.  Rows that pack_map does not name are not touched.  a.lse is ignored.
+cudaError_t launch_attn_bf16_tc_scatter(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, void* scratch,
+                                        size_t scratch_bytes, cudaStream_t st, int* launches);
 
 }  // namespace swam

@@ -20,8 +20,9 @@ LIB_PATH = os.path.join(_HERE, "libswam.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_STATE, ERR_CUDA, ERR_DEVICE_CHECK, ERR_TIMEOUT = range(8)
 F32, BF16 = 0, 1
 REUSE, REFRESH_FULL, REFRESH_LIGHT = 0, 1, 2
-OPT_ATTN_VARIANT = 1
+OPT_ATTN_VARIANT, OPT_SPARSE_PATH = 1, 2
 ATTN_AUTO, ATTN_WARP_MMA = 0, 1
+SPARSE_FUSED, SPARSE_STAGED = 0, 1
 
 EXPORTS = [
     "swam_create", "swam_destroy", "swam_workspace_bytes", "swam_bind_workspace", "swam_score", "swam_score_noalloc",

@@ -104,6 +104,16 @@ def test_full_size_cycle_matches_oracle(name, wl, n_rows):
     got_p = out[rows_p[:, 0], orig].float().cpu().numpy().astype(np.float64)
     check_bf16(got_p, want_p)
 
+    # ---- the fused sparse step (scatter inside the attention kernel) equals the staged one bit for bit -------
+    staged = swam.Swam.from_workload(wl)
+    staged.set_option(swam.OPT_SPARSE_PATH, swam.SPARSE_STAGED)
+    out_s = out_full.clone()
+    staged.step(d0["q"], d0["k"], d0["v"], swam.REFRESH_FULL, out_s)
+    staged.step(d1["q"], d1["k"], d1["v"], swam.REUSE, out_s)
+    staged.check()
+    assert torch.equal(out_s, out)
+    del staged, out_s
+
     # ---- every element: tcgen05 kernel vs the independent mma.sync kernel ----------------------------------
     other = swam.Swam.from_workload(wl)
     other.set_option(swam.OPT_ATTN_VARIANT, swam.ATTN_WARP_MMA)

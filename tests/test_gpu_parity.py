@@ -325,6 +325,34 @@ def test_light_refresh_step():
     check_float(f64(out), st.out, wl.dtype)
 
 
+@pytest.mark.parametrize("wl", [
+    small(batch=2),
+    small("larger_imagination", n_obs=40, grid_h=7, grid_w=9, n_heads=2),
+    small("larger_imagination", n_obs=300, grid_h=12, grid_w=11, n_heads=2, keep=0.5),   # whole tiles of observed rows
+    small(keep=1.0),
+    small(keep=0.0),
+], ids=["d64", "d128", "d128_long_obs", "keep_all", "keep_none"])
+@pytest.mark.parametrize("mode", ["reuse", "light"])
+def test_fused_sparse_step_equals_staged_bit_for_bit(wl, mode):
+    """Packed attention with the scatter fused into its epilogue and pack -> attention -> scatter give the same bits."""
+    swam = _swam()
+    x0, x1 = W.generate_steps(wl, 2)
+    outs = []
+    for path in (swam.SPARSE_FUSED, swam.SPARSE_STAGED):
+        ctx = swam.Swam.from_workload(wl)
+        ctx.set_option(swam.OPT_SPARSE_PATH, path)
+        out = ctx.empty_full().zero_()
+        n0 = ctx.launch_count()
+        ctx.step(dev(x0["q"], wl), dev(x0["k"], wl), dev(x0["v"], wl), swam.REFRESH_FULL, out)
+        n1 = ctx.launch_count()
+        ctx.step(dev(x1["q"], wl), dev(x1["k"], wl), dev(x1["v"], wl),
+                 swam.REUSE if mode == "reuse" else swam.REFRESH_LIGHT, out)
+        ctx.check()
+        outs.append((out.clone(), ctx.launch_count() - n1))
+    assert torch.equal(outs[0][0], outs[1][0])
+    assert outs[0][1] < outs[1][1]          # the fused step launches fewer kernels
+
+
 def test_reuse_before_refresh_is_a_state_error():
     swam = _swam()
     wl = W.WORKLOADS["tiny"]
