@@ -171,11 +171,12 @@ int swam_check(swam_ctx* ctx, void* stream);
  * tcgen05/TMEM kernel for head_dim 64 and 128 and the warp-level mma.sync kernel for head_dim 32;
  * SWAM_ATTN_WARP_MMA forces the mma.sync kernel (an independent on-device second opinion used by the tests).
  *
- * SWAM_OPT_SPARSE_PATH selects how swam_step ends a REUSE or REFRESH_LIGHT step (Sec. 3.3, Eq. 7):
- * SWAM_SPARSE_FUSED (default) lets the tcgen05 attention kernel write each retained row straight to its original
- * position in `out`, so that the packed output and the scatter pass do not exist; SWAM_SPARSE_STAGED runs swam_pack,
- * swam_sparse_attn and swam_scatter one after the other.  The fused path needs bf16, head_dim 64 or 128 and
- * SWAM_ATTN_AUTO; every other configuration runs staged.  Both paths produce the same bits. */
+ * SWAM_OPT_SPARSE_PATH selects how swam_step runs a REUSE or REFRESH_LIGHT step (Sec. 4.2, Eq. 7):
+ * SWAM_SPARSE_FUSED (default) packs only K and V; the tcgen05 attention kernel fetches its query rows from the full
+ * Q through pack_map and writes each retained row straight to its original position in `out`, so that the packed Q,
+ * the packed output and the scatter pass do not exist; SWAM_SPARSE_STAGED runs swam_pack, swam_sparse_attn and
+ * swam_scatter one after the other.  The fused path needs bf16, head_dim 64 or 128 and SWAM_ATTN_AUTO; every other
+ * configuration runs staged.  Both paths produce the same bits. */
 enum { SWAM_OPT_ATTN_VARIANT = 1, SWAM_OPT_SPARSE_PATH = 2 };
 enum { SWAM_ATTN_AUTO = 0, SWAM_ATTN_WARP_MMA = 1 };
 enum { SWAM_SPARSE_FUSED = 0, SWAM_SPARSE_STAGED = 1 };

@@ -74,6 +74,16 @@ __device__ __forceinline__ void tma_store_commit_wait() {
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
   asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+// one arrival on `bar` once every cp.async this thread has issued so far has landed (counted in the barrier's
+// expected arrivals, not added to them)
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -195,8 +205,9 @@ struct TcParams {
   float* lse;
   int* status;
   float* partial;      // split items: [slot][2 tiles][128 rows][D + 4]: unnormalised O, then reference max and sum
-  const int32_t* pack_map;  // scatter mode: [B, n] row of the full output tensor that each attended row is written to
-  int n_full;               // scatter mode: rows per sample of the full output tensor
+  const int32_t* pack_map;  // scatter and gather modes: [B, n] row of the full tensors that each attended row stands for
+  int n_full;               // scatter and gather modes: rows per sample of the full tensors
+  const __nv_bfloat16* q_full;  // gather mode: the full [B, n_full, N_h, D] query tensor
   int lse_row0, lse_rows;
   int n, N_h;
   int pairs;           // query tile pairs per (sample, head)
@@ -221,11 +232,18 @@ struct TcCfg {
   static constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(D >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
 };
 
-// SCATTER = false: map_o covers the [B, n, N_h, D] output in boxes of 128 rows, one store per query tile.
-// SCATTER = true (Eq. 7 fused into the packed attention): map_o covers the FULL [B, n_full, N_h, D] output in boxes of
-// one row, and each attended row goes straight to its original position pack_map[b, row]; the rows the packed sequence
-// omits are never touched and keep the cached values they hold.
-template <int D, bool SCATTER>
+// MODE = kDirect: the tensor maps cover [B, n, N_h, D] tensors in boxes of 128 rows; one output store per query tile.
+// MODE = kScatter (Eq. 7 fused into the packed attention): inputs as before, but map_o covers the FULL
+// [B, n_full, N_h, D] output in boxes of one row, and each attended row goes straight to its original position
+// pack_map[b, row]; the rows the packed sequence omits are never touched and keep the cached values they hold.
+// MODE = kGather (the query third of Sec. 4.2's pack fused in as well): K and V are packed tensors as before, but Q is
+// the full tensor; two warps fetch the query rows pack_map names with 16-byte asynchronous copies, writing the same
+// swizzled tile layout the tensor map would, so the packed Q never exists in memory.  map_q is not used.  (K and V
+// are shared by every query tile pair of a head: packing them once is cheaper than gathering them in every CTA.)
+enum { kDirect = 0, kScatter = 1, kGather = 2 };
+constexpr int kGatherThreads = 64;   // warps 10 and 11
+
+template <int D, int MODE>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o, const TcParams p) {
@@ -272,7 +290,8 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 
   if (threadIdx.x == 0) CTA_T(0);
   if (threadIdx.x == 0) {
-    mbar_init(bar_q, 1);
+    // direct loads: one arrival (the expect_tx) plus the bytes; gathered loads: one arrival per producer thread
+    mbar_init(bar_q, (MODE == kGather) ? kGatherThreads : 1);
     for (int s = 0; s < ST; ++s) {
       mbar_init(bar_k_full(s), 1);
       mbar_init(bar_k_empty(s), 1);
@@ -309,14 +328,71 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   // increase beyond what was released would wait forever.)
   if (warp >= 8) {
    asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
-   if (warp == 9) {
+   if (MODE == kGather && warp >= 10) {
+    // ------------------------------------------------------------------ gathering producers of Q (64 threads)
+    // Tile row rr <- row pack_map[b, prow0 + rr] of the full tensor; 16-byte chunk cc of a row lands where the
+    // 128-byte-swizzled box layout puts it: sub-tile cc / 8, row rr, chunk (cc % 8) ^ (rr % 8).  Rows beyond the
+    // packed sequence, and rows whose map entry is out of range (flagged), are filled with zeros.
+    // Rows are handled in blocks of 32: a warp reads the 32 map entries of a block with one coalesced load and then
+    // hands them out by shuffle, so that the copy loop itself contains no loads.
+    constexpr int CPR = D / 8;                 // 16-byte chunks per row
+    constexpr int RPI = 32 / CPR;              // rows per warp instruction
+    const int pw = warp - 10;
+    const int cc = lane % CPR, sub = lane / CPR;
+    const int32_t* pm = p.pack_map + (int64_t)b * p.n;
+    const int64_t row_stride = (int64_t)p.N_h * D;
+    const int64_t base_off = ((int64_t)b * p.n_full * p.N_h + h) * D + cc * 8;
+    const uint32_t dst_cc = (uint32_t)((cc >> 3) * C::kSubTile);
+    // map entries of row block rb of the tile starting at packed row prow0: -1 = fill with zeros
+    auto block_rows = [&](int prow0, int rb) {
+      const int pr = prow0 + rb * 32 + lane;
+      int orow = -1;
+      if (pr < p.n) {
+        orow = pm[pr];
+        if (orow < 0 || orow >= p.n_full) {
+          atomicOr(p.status, ST_BAD_MAP);
+          orow = -1;
+        }
+      }
+      return orow;
+    };
+    // per-lane constants of the copy loop: the swizzled chunk position only depends on (row % 8), and a lane's rows
+    // advance by RPI per instruction, so the positions repeat every 8 / RPI instructions
+    uint32_t dst_lane[8 / RPI];
+#pragma unroll
+    for (int i = 0; i < 8 / RPI; ++i) {
+      const int rl = i * RPI + sub;
+      dst_lane[i] = dst_cc + (uint32_t)(rl * 128 + (((cc & 7) ^ (rl & 7)) << 4));
+    }
+    auto gather_block = [&](uint32_t dst, const __nv_bfloat16* src, int rb, int rows_reg) {
+      const __nv_bfloat16* src_lane = src + base_off;
+      const uint32_t dst_blk = dst + (uint32_t)(rb * 32 * 128);
+#pragma unroll
+      for (int i = 0; i < 32 / RPI; ++i) {
+        const int orow = __shfl_sync(0xffffffffu, rows_reg, i * RPI + sub);
+        cp_async_16(dst_blk + dst_lane[i % (8 / RPI)] + (uint32_t)((i / (8 / RPI)) * 8 * 128),
+                    src_lane + (orow < 0 ? 0 : orow) * row_stride, orow < 0 ? 0u : 16u);
+      }
+    };
+    // warp pw copies row blocks pw and pw + 2 of both query tiles
+    for (int s = 0; s < 2; ++s) {
+      const int prow0 = row0 + s * kTile;
+      const int r0 = block_rows(prow0, pw), r1 = block_rows(prow0, pw + 2);
+      gather_block(sQ + s * C::kTileBytes, p.q_full, pw, r0);
+      gather_block(sQ + s * C::kTileBytes, p.q_full, pw + 2, r1);
+    }
+    cp_async_arrive(bar_q);
+    cp_async_wait_all();   // nothing of this thread is still on its way into shared memory at exit
+   } else if (warp == 9) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       bool ok = true;
-      mbar_expect_tx(bar_q, 2 * C::kTileBytes);
-      for (int s = 0; s < 2; ++s)
-        for (int db = 0; db < C::DB; ++db)
-          tma_load_4d(sQ + s * C::kTileBytes + db * C::kSubTile, &map_q, bar_q, db * 64, row0 + s * kTile, h, b);
+      if (MODE != kGather) {
+        mbar_expect_tx(bar_q, 2 * C::kTileBytes);
+        for (int s = 0; s < 2; ++s)
+          for (int db = 0; db < C::DB; ++db)
+            tma_load_4d(sQ + s * C::kTileBytes + db * C::kSubTile, &map_q, bar_q, db * 64, row0 + s * kTile, h, b);
+      }
       for (int j = 0; j < n_tiles && ok; ++j) {
         const int st = j % ST;
         const uint32_t par = ((j / ST) & 1) ^ 1;  // first pass over the ring: slots start empty
@@ -335,7 +411,10 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
    } else if (warp == 8) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
+      // gathered query tiles were written through the generic proxy and are read by the tensor core through the
+      // async proxy: the reader fences after the wait
       bool ok = mbar_wait(bar_q, 0, abort_flag);
+      if (MODE == kGather) fence_proxy_async();
       const uint32_t q_lo0 = desc_lo(sQ, 16), k_lo0 = desc_lo(sK, 16), v_lo0 = desc_lo(sV, C::kSubTile);
       auto issue_qk = [&](int s, int buf, int st) {
         // S = Q_s K^T : K dimension = D, 16 elements (32 bytes) per instruction inside the 128-byte swizzle row
@@ -556,7 +635,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         p.lse[((int64_t)b * p.N_h + h) * p.lse_rows + (row - p.lse_row0)] = (m_used + log2f(l_run)) * 0.6931471805599453f;
       fence_proxy_async();
     }
-    if (SCATTER) {
+    if (MODE != kDirect) {
       // each thread sends the row it has just staged (it reads only its own writes, so its own proxy fence is all the
       // ordering the copy engine needs); the 128-byte swizzle is a function of the shared-memory address, so a
       // one-row box at the row's offset reads the same bytes the 128-row box would
@@ -712,16 +791,21 @@ int sm_count_tc() {
   return sms;
 }
 
-// SCATTER: a.out is the full [B, n_full, N_h, D] tensor and pack_map [B, a.n] names the row each attended row goes to.
-template <int D, bool SCATTER>
+// kScatter: a.out is the full [B, n_full, N_h, D] tensor and pack_map [B, a.n] names the row each attended row goes
+// to.  kGather: a.q is the full tensor as well and pack_map also names the query rows.
+template <int D, int MODE>
 cudaError_t launch_tc_d(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, float* partial,
                         size_t partial_bytes, cudaStream_t st, int* launches) {
   CUtensorMap mq, mk, mv, mo;
-  if (!make_map(&mq, a.q, a.B, a.n, a.N_h, D) || !make_map(&mk, a.k, a.B, a.n, a.N_h, D) ||
-      !make_map(&mv, a.v, a.B, a.n, a.N_h, D) ||
-      !(SCATTER ? make_map(&mo, a.out, a.B, n_full, a.N_h, D, 1) : make_map(&mo, a.out, a.B, a.n, a.N_h, D)))
+  if (!(MODE != kDirect ? make_map(&mo, a.out, a.B, n_full, a.N_h, D, 1) : make_map(&mo, a.out, a.B, a.n, a.N_h, D)))
     return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(attn_bf16_tc_kernel<D, SCATTER>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<D>::kSmemBytes);
+  if (!make_map(&mk, a.k, a.B, a.n, a.N_h, D) || !make_map(&mv, a.v, a.B, a.n, a.N_h, D)) return cudaErrorInvalidValue;
+  if (MODE == kGather) {
+    mq = mo;   // not used by the kernel
+  } else if (!make_map(&mq, a.q, a.B, a.n, a.N_h, D)) {
+    return cudaErrorInvalidValue;
+  }
+  cudaError_t e = cudaFuncSetAttribute(attn_bf16_tc_kernel<D, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<D>::kSmemBytes);
   if (e != cudaSuccess) return e;
   const int pairs = (a.n + 2 * kTile - 1) / (2 * kTile);
   const int items = pairs * a.N_h * a.B;
@@ -743,14 +827,14 @@ cudaError_t launch_tc_d(const AttnArgs& a, const int32_t* pack_map, int n_full, 
 #ifdef SWAM_TC_TRACE
       (long long*)partial_trace_buffer(),
 #endif
-      a.lse, status, partial, pack_map, n_full, a.lse_row0, a.lse_rows, a.n, a.N_h, pairs, n_whole, splits, per,
+      a.lse, status, partial, pack_map, n_full, (const __nv_bfloat16*)a.q, a.lse_row0, a.lse_rows, a.n, a.N_h, pairs, n_whole, splits, per,
       a.scale * kLog2e};
   const int grid = n_whole + (splits ? rem * splits : 0);
   ++*launches;
-  attn_bf16_tc_kernel<D, SCATTER><<<grid, kThreadsTc, TcCfg<D>::kSmemBytes, st>>>(mq, mk, mv, mo, p);
+  attn_bf16_tc_kernel<D, MODE><<<grid, kThreadsTc, TcCfg<D>::kSmemBytes, st>>>(mq, mk, mv, mo, p);
   e = cudaGetLastError();
   if (e != cudaSuccess || !splits) return e;
-  CombineParams c{partial, SCATTER ? pack_map : nullptr, n_full, status, (__nv_bfloat16*)a.out, a.lse, a.lse_row0, a.lse_rows,
+  CombineParams c{partial, MODE != kDirect ? pack_map : nullptr, n_full, status, (__nv_bfloat16*)a.out, a.lse, a.lse_row0, a.lse_rows,
                   a.n, a.N_h, D, pairs, n_whole, splits, rem};
   ++*launches;
   attn_combine_kernel<D><<<(rem * 2 * kTile + 7) / 8, 256, 0, st>>>(c);
@@ -771,8 +855,8 @@ size_t attn_tc_scratch_bytes(int D) {
 cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, void* scratch, size_t scratch_bytes, cudaStream_t st,
                                 int* launches) {
   switch (a.D) {
-    case 64: return launch_tc_d<64, false>(a, nullptr, a.n, status, (float*)scratch, scratch_bytes, st, launches);
-    case 128: return launch_tc_d<128, false>(a, nullptr, a.n, status, (float*)scratch, scratch_bytes, st, launches);
+    case 64: return launch_tc_d<64, kDirect>(a, nullptr, a.n, status, (float*)scratch, scratch_bytes, st, launches);
+    case 128: return launch_tc_d<128, kDirect>(a, nullptr, a.n, status, (float*)scratch, scratch_bytes, st, launches);
     default: return cudaErrorInvalidConfiguration;
   }
 }
@@ -780,8 +864,17 @@ cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, void* scratch, s
 cudaError_t launch_attn_bf16_tc_scatter(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, void* scratch,
                                         size_t scratch_bytes, cudaStream_t st, int* launches) {
   switch (a.D) {
-    case 64: return launch_tc_d<64, true>(a, pack_map, n_full, status, (float*)scratch, scratch_bytes, st, launches);
-    case 128: return launch_tc_d<128, true>(a, pack_map, n_full, status, (float*)scratch, scratch_bytes, st, launches);
+    case 64: return launch_tc_d<64, kScatter>(a, pack_map, n_full, status, (float*)scratch, scratch_bytes, st, launches);
+    case 128: return launch_tc_d<128, kScatter>(a, pack_map, n_full, status, (float*)scratch, scratch_bytes, st, launches);
+    default: return cudaErrorInvalidConfiguration;
+  }
+}
+
+cudaError_t launch_attn_bf16_tc_gather(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, void* scratch,
+                                       size_t scratch_bytes, cudaStream_t st, int* launches) {
+  switch (a.D) {
+    case 64: return launch_tc_d<64, kGather>(a, pack_map, n_full, status, (float*)scratch, scratch_bytes, st, launches);
+    case 128: return launch_tc_d<128, kGather>(a, pack_map, n_full, status, (float*)scratch, scratch_bytes, st, launches);
     default: return cudaErrorInvalidConfiguration;
   }
 }

@@ -368,15 +368,16 @@ int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t 
   }
   if (mode != SWAM_REFRESH_FULL && c->sparse_path == SWAM_SPARSE_FUSED && d.dtype == SWAM_BF16 && d.D >= 64 &&
       c->attn_variant == SWAM_ATTN_AUTO) {
-    // packed attention writes each retained row straight to its place in `out`; the omitted rows keep the cached
-    // value they already hold (Eq. 7), so no packed output and no scatter pass exist
-    void* qp = c->ws + c->off_qp;
+    // K and V are packed by the copy kernel (every query tile of a head reads them); the attention kernel fetches
+    // its query rows from the full Q itself and writes each result row straight to its place in `out`.  The omitted
+    // rows keep the cached value they already hold (Eq. 7), so neither a packed Q, nor a packed output, nor a scatter
+    // pass exist.
     void* kp = c->ws + c->off_kp;
     void* vp = c->ws + c->off_vp;
-    if (int r = swam_pack(c, q, k, v, pm, qp, kp, vp, stream)) return r;
-    AttnArgs a{qp, kp, vp, out, nullptr, 0, 0, d.B, d.Lp, d.N_h, d.D, d.scale};
-    cudaError_t e = launch_attn_bf16_tc_scatter(a, pm, d.L, (int*)(c->ws + c->off_status), c->ws + c->off_attn,
-                                                c->attn_scratch, st, &c->launches_i);
+    if (int r = swam_pack(c, nullptr, k, v, pm, nullptr, kp, vp, stream)) return r;
+    AttnArgs a{q, kp, vp, out, nullptr, 0, 0, d.B, d.Lp, d.N_h, d.D, d.scale};
+    cudaError_t e = launch_attn_bf16_tc_gather(a, pm, d.L, (int*)(c->ws + c->off_status), c->ws + c->off_attn,
+                                               c->attn_scratch, st, &c->launches_i);
     count(c);
     if (e != cudaSuccess) return fail_cuda(c, e, "fused sparse attention launch");
   } else if (mode != SWAM_REFRESH_FULL) {

@@ -81,5 +81,9 @@ cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, void* scratch, s
 // pack_map[b, i] of it.  Rows that pack_map does not name are not touched.  a.lse is ignored.
 cudaError_t launch_attn_bf16_tc_scatter(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, void* scratch,
                                         size_t scratch_bytes, cudaStream_t st, int* launches);
+// The same with the query third of Sec. 4.2's pack fused in too: a.q and a.out are FULL tensors [B, n_full, N_h, D],
+// a.k and a.v packed ones; the kernel fetches query row pack_map[b, i] for attended row i itself.
+cudaError_t launch_attn_bf16_tc_gather(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, void* scratch,
+                                       size_t scratch_bytes, cudaStream_t st, int* launches);
 
 }  // namespace swam
