@@ -142,6 +142,24 @@ def per_launch_us(fns, reps):
     return e0.elapsed_time(e1) * 1e3 / (reps * len(fns))
 
 
+def power_profile_us(fns, n_launches=160):
+    """Device time per launch at the start and at the end of one back-to-back run of `n_launches` launches (rotating
+    input sets), after a short idle: the difference shows how much of the steady-state time is the power cap."""
+    torch.cuda.synchronize()
+    time.sleep(0.5)
+    for f in fns:
+        f()                                        # wake the clocks
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_launches + 1)]
+    marks[0].record()
+    for i in range(n_launches):
+        fns[i % len(fns)]()
+        marks[i + 1].record()
+    torch.cuda.synchronize()
+    t = [marks[i].elapsed_time(marks[i + 1]) * 1e3 for i in range(n_launches)]
+    k = max(4, n_launches // 8)
+    return float(np.median(t[2:2 + k])), float(np.median(t[-k:]))
+
+
 def bench_swam(args):
     from paper_2609_38984_b200 import swam
     _, local_rank, _ = sd.env_rank()
@@ -274,6 +292,9 @@ def bench_swam(args):
             "light_refresh_step": stage(lambda i: lambda: lib.swam_step(ctx.ctx, P(rot[i]["q"]), P(rot[i]["k"]),
                                                                         P(rot[i]["v"]), swam.REFRESH_LIGHT, P(outs[i]), S())),
         }
+        dense_fns = [(lambda i: lambda: lib.swam_sparse_attn(ctx.ctx, P(rot[i]["q"]), P(rot[i]["k"]), P(rot[i]["v"]), L,
+                                                             P(outs[i]), None, S()))(i) for i in range(N_ROT)]
+        dense_first_us, dense_late_us = power_profile_us(dense_fns)
         ctx.check()
         algo = {  # algorithmic bytes / flops per launch
             "score": ("hbm", B * (fut * row + wl.n_action * row + wl.n_frames * wl.n_spatial * 4)),
@@ -297,6 +318,9 @@ def bench_swam(args):
                                 "frac": round(ach / peaks["bf16_tflops"], 4)}
         for name in ("full_step", "sparse_step", "light_refresh_step"):
             stages[name] = {"us": round(stage_us[name], 2)}
+        # the dense launch right after an idle gap and after ~0.15 s of back-to-back launches (power cap engaged)
+        stages["attn_dense"]["us_first_launches_after_idle"] = round(dense_first_us, 2)
+        stages["attn_dense"]["us_after_160_back_to_back"] = round(dense_late_us, 2)
         # dominant kernel: the joint-attention kernel (dense launch of the full step + packed launch of the sparse steps)
         att_flops = algo["attn_dense"][1] + (R - 1) * algo["attn_packed"][1]
         att_us = stage_us["attn_dense"] + (R - 1) * stage_us["attn_packed"]
@@ -311,6 +335,11 @@ def bench_swam(args):
                     "achieved": round(achieved, 2), "peak": round(peak, 1), "unit": "TFLOP/s",
                     "frac": round(achieved / peak, 4), "peak_source": src,
                     "traffic": DOMINANT_KERNEL_DRAM_BYTES.get(wl0.name)}
+        if wl.dtype == W.BF16:
+            # the stage loop runs long enough for the power cap to engage, which is the regime the sustained GEMM
+            # figure was measured in; the headline fraction above stays on the (larger) burst figure
+            roofline["frac_of_sustained_peak"] = round(achieved / peaks["bf16_tflops_sustained"], 4)
+            roofline["sustained_peak"] = peaks["bf16_tflops_sustained"]
         cpu = cpu_baseline(wl, host_steps, budget_s=args.cpu_seconds)
         line = {
             "metric": "packed_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,

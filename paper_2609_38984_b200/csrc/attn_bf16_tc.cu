@@ -88,26 +88,37 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// The issuing warp runs its loops converged (so that descriptors and addresses stay in the uniform datapath) and one
+// elected lane issues the tcgen05 instructions: `el` is that lane's flag.  Issuing from inside a divergent
+// `if (lane == 0)` branch costs about twice as many cycles per instruction.
+__device__ __forceinline__ uint32_t elect_one() {
+  uint32_t el;
+  asm volatile("{\n .reg .pred q;\n elect.sync _|q, 0xffffffff;\n selp.u32 %0, 1, 0, q;\n}" : "=r"(el));
+  return el;
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar, uint32_t el) {
+  asm volatile("{\n .reg .pred q;\n setp.ne.b32 q, %1, 0;\n"
+               " @q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}" ::"r"(bar), "r"(el) : "memory");
 }
 // The issuing thread's own instruction count per MMA matters (one MMA of this size executes in 32-64 clk), so the
 // 64-bit shared-memory descriptors are kept as a constant high word and a low word that only needs an add.
 // D[tmem] (+)= A[smem desc] * B[smem desc]
 template <bool kAccum>
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc) {
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                       uint32_t el) {
   asm volatile(
-      "{\n .reg .pred p;\n .reg .b64 da, db;\n setp.ne.b32 p, %5, 0;\n mov.b64 da, {%1, %3};\n mov.b64 db, {%2, %3};\n"
-      " tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n}"
-      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "n"(kAccum ? 1 : 0) : "memory");
+      "{\n .reg .pred p, q;\n .reg .b64 da, db;\n setp.ne.b32 p, %5, 0;\n setp.ne.b32 q, %6, 0;\n"
+      " mov.b64 da, {%1, %3};\n mov.b64 db, {%2, %3};\n"
+      " @q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "n"(kAccum ? 1 : 0), "r"(el) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem desc]
 __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
-                                       uint32_t accum) {
+                                       uint32_t accum, uint32_t el) {
   asm volatile(
-      "{\n .reg .pred p;\n .reg .b64 db;\n setp.ne.b32 p, %5, 0;\n mov.b64 db, {%2, %3};\n"
-      " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n}"
-      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accum) : "memory");
+      "{\n .reg .pred p, q;\n .reg .b64 db;\n setp.ne.b32 p, %5, 0;\n setp.ne.b32 q, %6, 0;\n mov.b64 db, {%2, %3};\n"
+      " @q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accum), "r"(el) : "memory");
 }
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
@@ -227,7 +238,7 @@ struct TcCfg {
   // columns, which leaves room for a third score buffer and lets Q K^T run one tile further ahead of the softmax
   static constexpr int kSBufs = (D == 128) ? 2 : 3;
   static constexpr int kSmemData = 2 * kTileBytes + 2 * kStages * kTileBytes;
-  static constexpr int kSmemBytes = kSmemData + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int kSmemBytes = kSmemData + 1024 /*alignment slack*/ + 512 /*barriers*/;
   static constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
   static constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(D >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
 };
@@ -266,8 +277,10 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   auto bar_s_full = [&](int buf) { return bars + 8 * (1 + 4 * ST + buf); };
   auto bar_p_full = [&](int buf) { return bars + 8 * (4 + 4 * ST + buf); };
   const uint32_t bar_o_final = bars + 8 * (7 + 4 * ST);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + C::kSmemData + 8 * (8 + 4 * ST));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::kSmemData + 8 * (8 + 4 * ST) + 8);
+  // P V of a query tile's item has completed: that tile's output accumulator is up to date
+  auto bar_pv_tile = [&](int s) { return bars + 8 * (8 + 4 * ST + s); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + C::kSmemData + 8 * (10 + 4 * ST));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::kSmemData + 8 * (10 + 4 * ST) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // work item = (sample, head, query tile pair), pair fastest.  Items below n_whole walk over all keys; the few items
@@ -302,6 +315,8 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       mbar_init(bar_s_full(buf), 1);
       mbar_init(bar_p_full(buf), kTile);
     }
+    mbar_init(bar_pv_tile(0), 1);
+    mbar_init(bar_pv_tile(1), 1);
     mbar_init(bar_o_final, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -327,7 +342,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   // 120 x 128 = 15360 registers, and raising the two softmax warpgroups to 224 takes 56 x 256 = 14336 of them.  An
   // increase beyond what was released would wait forever.)
   if (warp >= 8) {
-   asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+   asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
    if (MODE == kGather && warp >= 10) {
     // ------------------------------------------------------------------ gathering producers of Q (64 threads)
     // Tile row rr <- row pack_map[b, prow0 + rr] of the full tensor; 16-byte chunk cc of a row lands where the
@@ -409,71 +424,78 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       }
     }
    } else if (warp == 8) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer (whole warp converged, one lane issues)
+    {
+      const uint32_t el = elect_one();
+      // every lane waits for itself (each then holds the barrier's acquire for what it issues or skips), and the
+      // warp agrees on the outcome so that it stays converged
+      auto wait_all = [&](uint32_t bar, uint32_t parity) {
+        return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag) ? 1 : 0) != 0;
+      };
       // gathered query tiles were written through the generic proxy and are read by the tensor core through the
       // async proxy: the reader fences after the wait
-      bool ok = mbar_wait(bar_q, 0, abort_flag);
+      bool ok = wait_all(bar_q, 0);
       if (MODE == kGather) fence_proxy_async();
       const uint32_t q_lo0 = desc_lo(sQ, 16), k_lo0 = desc_lo(sK, 16), v_lo0 = desc_lo(sV, C::kSubTile);
       auto issue_qk = [&](int s, int buf, int st) {
         // S = Q_s K^T : K dimension = D, 16 elements (32 bytes) per instruction inside the 128-byte swizzle row
         const uint32_t a_lo = q_lo0 + ((uint32_t)(s * C::kTileBytes) >> 4), b_lo = k_lo0 + ((uint32_t)(st * C::kTileBytes) >> 4);
         const uint32_t d = tm_S(buf);
-        mma_ss<false>(d, a_lo, b_lo, kDescHi, C::kIdescQK);
+        mma_ss<false>(d, a_lo, b_lo, kDescHi, C::kIdescQK, el);
 #pragma unroll
         for (int ks = 1; ks < D / 16; ++ks) {
           constexpr int kSub16 = C::kSubTile >> 4;
           const uint32_t off = (uint32_t)((ks >> 2) * kSub16 + (ks & 3) * 2);
-          mma_ss<true>(d, a_lo + off, b_lo + off, kDescHi, C::kIdescQK);
+          mma_ss<true>(d, a_lo + off, b_lo + off, kDescHi, C::kIdescQK, el);
         }
       };
       auto issue_pv = [&](int s, int buf, int st, bool accum) {
         // O_s += P V : K dimension = 128 keys, 16 keys (two 8-row groups) per instruction; V is MN-major
         const uint32_t b_lo = v_lo0 + ((uint32_t)(st * C::kTileBytes) >> 4);
         const uint32_t d = tm_O(s), a = tm_S(buf);
-        mma_ts(d, a, b_lo, kDescHi, C::kIdescPV, accum ? 1u : 0u);
+        mma_ts(d, a, b_lo, kDescHi, C::kIdescPV, accum ? 1u : 0u, el);
 #pragma unroll
-        for (int kk = 1; kk < kTile / 16; ++kk) mma_ts(d, a + kk * 8, b_lo + kk * (2048 >> 4), kDescHi, C::kIdescPV, 1u);
+        for (int kk = 1; kk < kTile / 16; ++kk) mma_ts(d, a + kk * 8, b_lo + kk * (2048 >> 4), kDescHi, C::kIdescPV, 1u, el);
       };
       // Items are issued in order: Q K^T of the first NB items up front, then for each item its P V followed by the
-      // Q K^T of item i + NB into the score buffer that P V has just consumed (the tensor pipe executes in issue
-      // order).  With three buffers the scores of a query tile's next key tile are ready before its softmax
-      // warpgroup has finished the current one.
+      // Q K^T of item i + NB into the score buffer that P V has just consumed (the tensor pipe executes one thread's
+      // instructions in issue order).  With three buffers the scores of a query tile's next key tile are ready before
+      // its softmax warpgroup has finished the current one.
       const int n_items = 2 * n_tiles;
       int k_waited = 0, v_waited = 0;
       auto qk_item = [&](int it) -> bool {
         const int j = it >> 1, sq = it & 1, st = j % ST;
         if (j >= k_waited) {
-          if (!mbar_wait(bar_k_full(st), (j / ST) & 1, abort_flag)) return false;
+          if (!wait_all(bar_k_full(st), (j / ST) & 1)) return false;
           k_waited = j + 1;
           tc_fence_after();
         }
         issue_qk(sq, it % NB, st);
-        tc_commit(bar_s_full(it % NB));
-        if (sq == 1) tc_commit(bar_k_empty(st));   // both query tiles have used this key tile
+        tc_commit(bar_s_full(it % NB), el);
+        if (sq == 1) tc_commit(bar_k_empty(st), el);   // both query tiles have used this key tile
         return true;
       };
       for (int it = 0; it < NB && it < n_items && ok; ++it) ok = qk_item(it);
       for (int it = 0; it < n_items && ok; ++it) {
         const int j = it >> 1, sq = it & 1, st = j % ST, buf = it % NB;
         if (j >= v_waited) {
-          ok = mbar_wait(bar_v_full(st), (j / ST) & 1, abort_flag);
+          ok = wait_all(bar_v_full(st), (j / ST) & 1);
           if (!ok) break;
           v_waited = j + 1;
         }
         TRACE(2, it * 4 + 0);
-        ok = mbar_wait(bar_p_full(buf), (it / NB) & 1, abort_flag);
+        ok = wait_all(bar_p_full(buf), (it / NB) & 1);
         if (!ok) break;
         TRACE(2, it * 4 + 1);
         tc_fence_after();
         issue_pv(sq, buf, st, j > 0);
         TRACE(2, it * 4 + 2);
-        if (sq == 1) tc_commit(bar_v_empty(st));
+        tc_commit(bar_pv_tile(sq), el);
+        if (sq == 1) tc_commit(bar_v_empty(st), el);
         if (it + NB < n_items) ok = qk_item(it + NB);
         TRACE(2, it * 4 + 3);
       }
-      if (ok) tc_commit(bar_o_final);
+      if (ok) tc_commit(bar_o_final, el);
     }
    }
   } else {
@@ -556,6 +578,13 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         m_used += delta;
         l_run *= f;
         tmem_st_wait();
+        // the accumulator must hold every product issued against the old reference before it is rescaled (with three
+        // score buffers the previous P V of this tile may still be waiting behind a Q K^T)
+        if (j > 0) {
+          ok = mbar_wait(bar_pv_tile(s), (j - 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+        }
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
           float ov[32];

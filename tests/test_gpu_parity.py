@@ -219,6 +219,44 @@ def test_attention_matches_oracle(name, kw):
     assert np.abs(lse.cpu().numpy() - wlse).max() <= (1e-4 if wl.dtype == W.F32 else 2e-3)
 
 
+@pytest.mark.parametrize("head_dim", [32, 64, 128])
+@pytest.mark.parametrize("pattern", ["ramp", "late_spike"])
+def test_attention_with_a_growing_row_maximum(head_dim, pattern):
+    """Logits that keep outgrowing the maximum of the first key tile: every later tile (ramp) or one late tile
+    (late_spike) forces the running reference of the online softmax to be raised and the output rescaled."""
+    swam = _swam()
+    n = 1100                                   # nine key tiles, ragged tail
+    wl = W.WORKLOADS["single_view"].with_(n_obs=n - 64 - 32, grid_h=8, grid_w=8, n_frames=1, n_action=32, n_heads=2,
+                                          head_dim=head_dim, keep=1.0)
+    assert wl.seq_len == n
+    rng = np.random.default_rng(5)
+    shape = (1, n, 2, head_dim)
+    u = rng.standard_normal(head_dim)
+    u /= np.linalg.norm(u)
+    # q = noise + sqrt(D) u and k = noise + gain u give a logit of about `gain` (natural-log units)
+    q = 0.3 * rng.standard_normal(shape) + u * np.sqrt(head_dim)
+    pos = np.arange(n)[None, :, None, None]
+    if pattern == "ramp":
+        gain = 12.0 * (pos // 128)             # far beyond the 2^8 slack of the running reference, at every tile
+    else:
+        gain = np.where((pos >= 700) & (pos < 720), 40.0, 0.0)
+    k = 0.3 * rng.standard_normal(shape) + u * gain
+    v = rng.standard_normal(shape)
+    q, k, v = (t.astype(np.float32) for t in (q, k, v))
+    ctx = swam.Swam.from_workload(wl)
+    qd, kd, vd = (dev(t, wl) for t in (q, k, v))
+    qh, kh, vh = (f64(t) for t in (qd, kd, vd))          # the bf16-rounded values the kernel sees
+    out, lse = ctx.sparse_attn(qd, kd, vd, want_lse=True)
+    ctx.check()
+    want, wlse = ora.attention(qh, kh, vh)
+    check_float(f64(out), want, wl.dtype)
+    assert np.abs(lse.cpu().numpy() - wlse).max() <= 5e-3
+    # several passes: the result does not depend on timing between the roles of the kernel
+    for _ in range(5):
+        again = ctx.sparse_attn(qd, kd, vd)
+        assert torch.equal(again, out)
+
+
 def test_attention_short_sequences():
     """seq_len below the full length, down to one token."""
     swam = _swam()
