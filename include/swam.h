@@ -163,6 +163,16 @@ int swam_get_selection(const swam_ctx* ctx, const int32_t** sel_idx, const int32
                        const int32_t** inv_map);
 int swam_get_scores(const swam_ctx* ctx, const float** scores, const float** lse_action, const float** quality);
 
+/* Installs a selection made elsewhere as the state that SWAM_REUSE steps use: sel_idx [B, F, K], pack_map [B, L'] and
+ * inv_map [B, L] (device pointers, int32, the layouts swam_select writes) are copied into the workspace on `stream`.
+ * Uses: the unconditional forward of a guided denoising step reuses the selection of the conditional forward, from
+ * which the scores come (Sec. 4.2; Table 5 lists the guidance scales); the selection ablations of Sec. 5.4 (core only,
+ * anchors only, random) run swam_select on scores of their own and install the result; a saved state is restored.
+ * The maps are not checked here: the kernels that follow them skip and flag entries out of range (swam_check).
+ * Errors: SWAM_ERR_INVALID_ARG (null pointer), SWAM_ERR_WORKSPACE (none bound), SWAM_ERR_CUDA. */
+int swam_set_selection(swam_ctx* ctx, const int32_t* sel_idx, const int32_t* pack_map, const int32_t* inv_map,
+                       void* stream);
+
 /* Synchronises `stream`, reads and clears the device status word; returns SWAM_OK, SWAM_ERR_DEVICE_CHECK,
  * SWAM_ERR_TIMEOUT or SWAM_ERR_CUDA. */
 int swam_check(swam_ctx* ctx, void* stream);

@@ -441,6 +441,22 @@ int swam_get_selection(const swam_ctx* c, const int32_t** sel_idx, const int32_t
   return SWAM_OK;
 }
 
+int swam_set_selection(swam_ctx* c, const int32_t* sel_idx, const int32_t* pack_map, const int32_t* inv_map, void* stream) {
+  if (!c || !sel_idx || !pack_map || !inv_map) return fail(c, SWAM_ERR_INVALID_ARG, "swam_set_selection: null argument");
+  if (int r = need_ws(c)) return r;
+  const Dims& d = c->d;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = cudaMemcpyAsync(c->ws + c->off_sel, sel_idx, (size_t)d.B * d.F * d.K * sizeof(int32_t),
+                                  cudaMemcpyDeviceToDevice, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(c->ws + c->off_pack, pack_map, (size_t)d.B * d.Lp * sizeof(int32_t), cudaMemcpyDeviceToDevice, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(c->ws + c->off_inv, inv_map, (size_t)d.B * d.L * sizeof(int32_t), cudaMemcpyDeviceToDevice, st);
+  if (e != cudaSuccess) return fail_cuda(c, e, "swam_set_selection");
+  c->has_selection = true;
+  return SWAM_OK;
+}
+
 int swam_get_scores(const swam_ctx* c, const float** scores, const float** lse_action, const float** quality) {
   if (!c || !c->ws) return SWAM_ERR_WORKSPACE;
   if (scores) *scores = (const float*)(c->ws + c->off_scores);

@@ -28,7 +28,7 @@ EXPORTS = [
     "swam_create", "swam_destroy", "swam_workspace_bytes", "swam_bind_workspace", "swam_score", "swam_score_noalloc",
     "swam_select", "swam_aggregate", "swam_select_maps",
     "swam_pack", "swam_sparse_attn", "swam_scatter", "swam_step", "swam_host_io_bytes", "swam_bind_host_io",
-    "swam_step_host", "swam_host_join", "swam_get_selection", "swam_get_scores", "swam_check", "swam_set_option", "swam_launch_count",
+    "swam_step_host", "swam_host_join", "swam_get_selection", "swam_get_scores", "swam_set_selection", "swam_check", "swam_set_option", "swam_launch_count",
     "swam_last_error", "swam_version",
 ]
 
@@ -80,6 +80,7 @@ def load_library() -> ctypes.CDLL:
         lib.swam_host_join.argtypes = [vp, vp]
         lib.swam_get_selection.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
         lib.swam_get_scores.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
+        lib.swam_set_selection.argtypes = [vp, vp, vp, vp, vp]
         lib.swam_check.argtypes = [vp, vp]
         lib.swam_set_option.argtypes = [vp, i32, i32]
         lib.swam_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
@@ -274,6 +275,13 @@ class Swam:
         self._chk(self.lib.swam_get_selection(self.ctx, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)))
         return (self._view(a, (self.B, self.F, self.K), torch.int32), self._view(b, (self.B, self.Lp), torch.int32),
                 self._view(c, (self.B, self.L), torch.int32))
+
+    def set_selection(self, sel_idx: torch.Tensor, pack_map: torch.Tensor, inv_map: torch.Tensor):
+        """Install a selection made elsewhere (another context's, or swam_select on other scores) for REUSE steps."""
+        for t, shape in ((sel_idx, (self.B, self.F, self.K)), (pack_map, (self.B, self.Lp)), (inv_map, (self.B, self.L))):
+            if t.dtype != torch.int32 or tuple(t.shape) != shape or not t.is_contiguous() or not t.is_cuda:
+                raise ValueError(f"expected a contiguous int32 CUDA tensor of shape {shape}")
+        self._chk(self.lib.swam_set_selection(self.ctx, _ptr(sel_idx), _ptr(pack_map), _ptr(inv_map), _stream()))
 
     def cached_scores(self):
         a, b, c = ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_void_p()

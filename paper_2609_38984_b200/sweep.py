@@ -1,4 +1,6 @@
-"""Keep-ratio x refresh-interval sweep at the larger-imagination shape (seed 4).
+"""Keep-ratio x refresh-interval sweep at the larger-imagination shape (seed 4), and the paper's ablations on the shapes
+of its Table 5: selection strategy (combined, core only, stable anchors only, random; Sec. 5.4), retained tokens per
+frame (256 / 184 / 112 of 360; Sec. 5.4) and refresh schedule (first step only, or every R-th step; App. C.2).
 
 For each (keep, R) the workload's 10 denoising steps run through swam_step on one GPU; every stage is also timed
 on its own through the individual C-ABI calls.  Reported per configuration: the latency split over score, select,
@@ -8,6 +10,8 @@ score + select at every step), and how far the sparse output is from the dense o
 number, not a pass/fail: the paper gives no figure for it).
 
   python -m paper_2609_38984_b200.sweep [--keeps 0.1,0.3] [--refresh 1,2,4] [--steps 10]
+  python -m paper_2609_38984_b200.sweep --shape cosmos3_nano --variants combined,core_only,stable_only,random \
+         --budgets 256,184,112 --refresh first,1,2
 """
 from __future__ import annotations
 
@@ -52,17 +56,23 @@ def _graph_us(fn, launches=8, reps=3):
     return a.elapsed_time(b) * 1e3 / (launches * reps)
 
 
-def run_config(keep: float, refresh: int, n_steps: int, dev_steps, dense_outs) -> dict:
-    wl = W.sweep_workload(keep, refresh).with_(steps=n_steps)
+def run_config(wl: W.Workload, refresh: int, n_steps: int, dev_steps, dense_outs, variant: str = "combined") -> dict:
+    """`wl` carries the budgets (see workloads.variant_workload); refresh = n_steps runs only the first step in full."""
+    keep = wl.keep
     ctx = swam.Swam.from_workload(wl)
     diag = swam.Swam.from_workload(wl)          # diagnostic scoring/selection at every step
     out = ctx.empty_full().zero_()
     sched = W.refresh_schedule(n_steps, refresh)
+
     step_us, rel_l2, ious, overlaps = [], [], [], []
     prev_sel, prev_scores = None, None
     for t, x in enumerate(dev_steps):
         mode = swam.REFRESH_FULL if sched[t] else swam.REUSE
         step_us.append(_event_us(lambda: ctx.step(x["q"], x["k"], x["v"], mode, out), reps=1))
+        if sched[t] and variant == "random":
+            # random selection: the same budget per frame, ranked by keys that carry no information
+            keys = torch.from_numpy(W.random_scores(wl.seed * 1000 + t, wl.batch, wl.n_frames, wl.n_spatial)).cuda()
+            ctx.set_selection(*ctx.select(keys))
         ctx.check()
         d = dense_outs[t].float()
         rel_l2.append(float((out.float() - d).norm() / d.norm()))
@@ -101,7 +111,7 @@ def run_config(keep: float, refresh: int, n_steps: int, dev_steps, dense_outs) -
     total_us = float(np.sum(step_us))
     tokens = wl.batch * sum(wl.seq_len if f else wl.packed_len for f in sched)
     return {
-        "keep": keep, "refresh": refresh, "k_core": wl.budgets[0], "k_anchor": wl.budgets[1], "packed_len": wl.packed_len,
+        "shape": wl.name, "variant": variant, "keep": round(keep, 4), "refresh": refresh, "k_core": wl.budgets[0], "k_anchor": wl.budgets[1], "packed_len": wl.packed_len,
         "steps": n_steps, "full_steps": len(full), "stage_us": {k: round(v, 2) for k, v in split.items()},
         "full_step_us": round(float(np.median(full)), 1), "sparse_step_us": round(float(np.median(sparse)), 1) if sparse else None,
         "schedule_us": round(total_us, 1), "tokens_per_s": tokens / (total_us * 1e-6),
@@ -112,20 +122,34 @@ def run_config(keep: float, refresh: int, n_steps: int, dev_steps, dense_outs) -
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--keeps", default=",".join(str(k) for k in W.SWEEP_KEEPS))
-    ap.add_argument("--refresh", default=",".join(str(r) for r in W.SWEEP_REFRESH))
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--shape", default="sweep", choices=["sweep"] + sorted(W.PAPER_SHAPES))
+    ap.add_argument("--keeps", default=",".join(str(k) for k in W.SWEEP_KEEPS), help="keep ratios (shape 'sweep')")
+    ap.add_argument("--budgets", default="", help="retained tokens per frame (paper shapes); default: the shape's own")
+    ap.add_argument("--variants", default="combined", help="of " + ",".join(W.SELECT_VARIANTS))
+    ap.add_argument("--refresh", default=",".join(str(r) for r in W.SWEEP_REFRESH),
+                    help="refresh intervals; 'first' = only the first step is a full step")
+    ap.add_argument("--steps", type=int, default=0, help="denoising steps (default: 10, or the paper shape's own)")
     args = ap.parse_args()
-    keeps = [float(k) for k in args.keeps.split(",")]
-    refreshes = [int(r) for r in args.refresh.split(",")]
-    base = W.sweep_workload(1.0, 1).with_(steps=args.steps)
-    host = W.generate_steps(base, args.steps)              # the inputs do not depend on keep or R
+    variants = args.variants.split(",")
+    if args.shape == "sweep":
+        base = W.sweep_workload(1.0, 1)
+        n_steps = args.steps or 10
+        cases = [W.sweep_workload(float(k), 1) for k in args.keeps.split(",")]
+    else:
+        base = W.PAPER_SHAPES[args.shape]
+        n_steps = args.steps or base.steps
+        cases = [base] if not args.budgets else [W.variant_workload(base, "combined", int(k)) for k in args.budgets.split(",")]
+    refreshes = [n_steps if r == "first" else int(r) for r in args.refresh.split(",")]
+    base = base.with_(steps=n_steps)
+    host = W.generate_steps(base, n_steps)                 # the inputs do not depend on budgets, variant or R
     dev_steps = [{n: swam.to_device(x[n], base.dtype) for n in "qkv"} for x in host]
     dense_ctx = swam.Swam.from_workload(base)
     dense_outs = [dense_ctx.sparse_attn(x["q"], x["k"], x["v"]) for x in dev_steps]   # memoised dense results
-    for keep in keeps:
-        for r in refreshes:
-            print(json.dumps(run_config(keep, r, args.steps, dev_steps, dense_outs)), flush=True)
+    for case in cases:
+        for variant in variants:
+            wl = W.variant_workload(case, variant).with_(steps=n_steps, name=f"{base.name}_k{case.k_keep}")
+            for r in refreshes:
+                print(json.dumps(run_config(wl.with_(refresh=r), r, n_steps, dev_steps, dense_outs, variant)), flush=True)
 
 
 if __name__ == "__main__":

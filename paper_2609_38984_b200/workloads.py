@@ -112,6 +112,51 @@ WORKLOADS: Dict[str, Workload] = {
     "multi_view": Workload("multi_view", 8, 1728, 4, 3, 24, 24, 32, 24, 64, BF16, 0.25, 10, 2, 3, blobs=1),
 }
 
+# Shapes of the models the paper evaluates (Table 5): camera views, future latent frames, tokens per future frame,
+# denoising steps, and the integer budgets K_c + K_s; refresh = steps means that only the first step is a full step,
+# the paper's default (Sec. 4.2).  The paper does not print head counts, head sizes, the number of action tokens or the
+# size of the observed frame: those are stand-ins (one observed latent frame of N_s tokens, 8 action tokens per
+# future frame).  Cosmos 3 Edge's three views differ in size (340 tokens per frame do not split into three equal
+# grids), so it is laid out as one 20 x 17 grid.
+PAPER_SHAPES: Dict[str, Workload] = {
+    "cosmos3_nano": Workload("cosmos3_nano", 1, 360, 8, 3, 10, 12, 64, 16, 128, BF16, 184 / 360, 4, 4, 11, blobs=1,
+                             k_core=80, k_anchor=104),
+    "cosmos3_edge": Workload("cosmos3_edge", 1, 340, 8, 1, 20, 17, 64, 16, 128, BF16, 184 / 340, 4, 4, 12, blobs=2,
+                             k_core=80, k_anchor=104),
+    "fastwam_joint": Workload("fastwam_joint", 1, 98, 2, 2, 7, 7, 16, 12, 64, BF16, 31 / 98, 10, 10, 13, blobs=1,
+                              k_core=19, k_anchor=12),
+}
+
+# Retained tokens per frame in the paper's pruning-ratio ablation on 360-token frames (Sec. 5.4: ratios 28.89 %,
+# 48.89 % (the default 184) and 68.89 %)
+PAPER_PRUNING_BUDGETS = (256, 184, 112)
+
+# Selection strategies of the component ablation (Sec. 5.4), all at the same K per frame
+SELECT_VARIANTS = ("combined", "core_only", "stable_only", "random")
+
+
+def variant_workload(wl: Workload, variant: str, k_keep: Optional[int] = None) -> Workload:
+    """The workload with the budgets of a selection variant: `combined` keeps the workload's own split (or the 10:13
+    rule for a new K), `core_only` spends all K on frame-specific core tokens, `stable_only` all K on shared anchors,
+    `random` ranks caller-drawn random keys per frame, which is core_only on those keys."""
+    if variant not in SELECT_VARIANTS:
+        raise ValueError(f"unknown selection variant {variant!r}")
+    k = wl.k_keep if k_keep is None else int(k_keep)
+    if not 0 <= k <= wl.n_spatial:
+        raise ValueError("K must lie in [0, N_s]")
+    if variant == "combined":
+        if k_keep is None:
+            kc, ks = wl.budgets
+        else:
+            kc = int(math.floor(k * 10.0 / 23.0 + 0.5))
+            ks = k - kc
+    elif variant == "stable_only":
+        kc, ks = 0, k
+    else:
+        kc, ks = k, 0
+    return wl.with_(name=f"{wl.name}_{variant}_k{k}", k_core=kc, k_anchor=ks, keep=k / wl.n_spatial)
+
+
 SWEEP_KEEPS = (0.1, 0.2, 0.3, 0.5, 1.0)
 SWEEP_REFRESH = (1, 2, 4)
 

@@ -391,6 +391,107 @@ def test_fused_sparse_step_equals_staged_bit_for_bit(wl, mode):
     assert outs[0][1] < outs[1][1]          # the fused step launches fewer kernels
 
 
+# ------------------------------------------------------------------ ablations and shapes of the paper's evaluation
+def _paper_shape(name, **kw):
+    base = dict(n_heads=2)
+    base.update(kw)
+    return W.PAPER_SHAPES[name].with_(**base)
+
+
+@pytest.mark.parametrize("variant", W.SELECT_VARIANTS)
+@pytest.mark.parametrize("k_keep", W.PAPER_PRUNING_BUDGETS)
+def test_selection_variants_at_the_paper_budgets(variant, k_keep):
+    """Sec. 5.4's strategies (combined, core only, stable anchors only, random) at 256 / 184 / 112 of 360 tokens."""
+    swam = _swam()
+    wl = W.variant_workload(_paper_shape("cosmos3_nano"), variant, k_keep)
+    kc, ks = wl.budgets
+    ctx = swam.Swam.from_workload(wl)
+    if variant == "random":
+        scores = W.random_scores(77 + k_keep, wl.batch, wl.n_frames, wl.n_spatial)
+    else:
+        x = W.generate_steps(wl, 1)[0]
+        scores = ctx.score(dev(x["q"], wl), dev(x["k"], wl)).cpu().numpy()
+    sel, pm, im = ctx.select(torch.from_numpy(scores).cuda())
+    ctx.check()
+    want = ora.select(scores, kc, ks)
+    wpm, wim = ora.maps(want["sel_idx"], wl.n_obs, wl.n_spatial, wl.n_action)
+    assert np.array_equal(sel.cpu().numpy(), want["sel_idx"])
+    assert np.array_equal(pm.cpu().numpy(), wpm) and np.array_equal(im.cpu().numpy(), wim)
+    assert sel.shape[-1] == k_keep
+    if variant == "stable_only":
+        # shared anchors only: every frame keeps the same spatial indices
+        s = sel.cpu().numpy()
+        assert (s == s[:, :1]).all()
+
+
+@pytest.mark.parametrize("name", ["cosmos3_nano", "cosmos3_edge", "fastwam_joint"])
+def test_paper_shapes_with_only_the_first_step_full(name):
+    """The default schedule of Sec. 4.2: one full step, every later step of the action chunk sparse."""
+    swam = _swam()
+    wl = _paper_shape(name)
+    steps = W.generate_steps(wl, min(wl.steps, 4))
+    ctx = swam.Swam.from_workload(wl)
+    refresh = len(steps)
+    assert W.refresh_schedule(len(steps), refresh) == [True] + [False] * (len(steps) - 1)
+    compare_schedule(wl, steps, refresh, run_schedule(ctx, wl, steps, refresh))
+
+
+def test_guided_pair_shares_the_conditional_selection():
+    """Two forwards per step (conditional, unconditional): scores and selection come from the conditional one; the
+    unconditional context installs that selection and runs its sparse steps with it."""
+    swam = _swam()
+    wl = small("larger_imagination", n_obs=40, grid_h=7, grid_w=9, n_heads=2, steps=2)
+    kc, ks = wl.budgets
+    c0, c1 = W.generate_steps(wl, 2)
+    u0, u1 = W.generate_steps(wl.with_(seed=wl.seed + 100), 2)
+    cond, uncond = swam.Swam.from_workload(wl), swam.Swam.from_workload(wl)
+    out_c, out_u = cond.empty_full().zero_(), uncond.empty_full().zero_()
+    cond.step(dev(c0["q"], wl), dev(c0["k"], wl), dev(c0["v"], wl), swam.REFRESH_FULL, out_c)
+    uncond.step(dev(u0["q"], wl), dev(u0["k"], wl), dev(u0["v"], wl), swam.REFRESH_FULL, out_u)
+    own = [t.clone() for t in uncond.selection()]
+    uncond.set_selection(*cond.selection())
+    for a, b in zip(uncond.selection(), cond.selection()):
+        assert torch.equal(a, b)
+    assert not torch.equal(own[0], cond.selection()[0])        # the unconditional forward would have chosen differently
+    cond.step(dev(c1["q"], wl), dev(c1["k"], wl), dev(c1["v"], wl), swam.REUSE, out_c)
+    uncond.step(dev(u1["q"], wl), dev(u1["k"], wl), dev(u1["v"], wl), swam.REUSE, out_u)
+    cond.check()
+    uncond.check()
+    args = (wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, kc, ks)
+    st_c = ora.full_step(ora.StepState(), c0["q"], c0["k"], c0["v"], *args)
+    st_u = ora.full_step(ora.StepState(), u0["q"], u0["k"], u0["v"], *args)
+    assert np.array_equal(cond.selection()[0].cpu().numpy(), st_c.sel["sel_idx"]), st_c.sel["margins"]
+    st_u.pack_map, st_u.inv_map = st_c.pack_map, st_c.inv_map
+    ora.sparse_step(st_c, c1["q"], c1["k"], c1["v"])
+    ora.sparse_step(st_u, u1["q"], u1["k"], u1["v"])
+    check_float(f64(out_c), st_c.out, wl.dtype)
+    check_float(f64(out_u), st_u.out, wl.dtype)
+
+
+def test_corrupt_installed_selection_is_reported_not_followed():
+    swam = _swam()
+    wl = small()
+    x0, x1 = W.generate_steps(wl, 2)
+    ctx = swam.Swam.from_workload(wl)
+    out = ctx.empty_full().zero_()
+    ctx.step(dev(x0["q"], wl), dev(x0["k"], wl), dev(x0["v"], wl), swam.REFRESH_FULL, out)
+    before = out.clone()
+    sel, pm, im = (t.clone() for t in ctx.selection())
+    bad = pm.clone()
+    bad[0, 3] = wl.seq_len + 7
+    bad[0, 4] = -1
+    ctx.set_selection(sel, bad, im)
+    ctx.step(dev(x1["q"], wl), dev(x1["k"], wl), dev(x1["v"], wl), swam.REUSE, out)
+    with pytest.raises(swam.SwamError) as e:
+        ctx.check()
+    assert e.value.code == swam.ERR_DEVICE_CHECK
+    # rows of the bad entries were left alone, the context still works
+    assert torch.equal(out[0, 3], before[0, 3]) and torch.equal(out[0, 4], before[0, 4])
+    ctx.set_selection(sel, pm, im)
+    ctx.step(dev(x1["q"], wl), dev(x1["k"], wl), dev(x1["v"], wl), swam.REUSE, out)
+    ctx.check()
+
+
 def test_reuse_before_refresh_is_a_state_error():
     swam = _swam()
     wl = W.WORKLOADS["tiny"]

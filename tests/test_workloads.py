@@ -54,3 +54,25 @@ def test_hotspot_drift_is_bounded():
 def test_refresh_schedule():
     assert W.refresh_schedule(5, 2) == [True, False, True, False, True]
     assert W.refresh_schedule(3, 1) == [True, True, True]
+
+
+def test_paper_shapes_and_ablation_budgets():
+    """Table 5: tokens per future frame, future frames, denoising steps and K_c + K_s of the evaluated models."""
+    want = {"cosmos3_nano": (360, 8, 4, 80, 104), "cosmos3_edge": (340, 8, 4, 80, 104), "fastwam_joint": (98, 2, 10, 19, 12)}
+    for name, (n_s, frames, steps, kc, ks) in want.items():
+        wl = W.PAPER_SHAPES[name]
+        assert (wl.n_spatial, wl.n_frames, wl.steps, wl.budgets) == (n_s, frames, steps, (kc, ks))
+        assert wl.n_action % wl.n_frames == 0 and wl.group % 4 == 0
+        # the default schedule: only the first step is a full step
+        assert W.refresh_schedule(wl.steps, wl.refresh) == [True] + [False] * (wl.steps - 1)
+    nano = W.PAPER_SHAPES["cosmos3_nano"]
+    # pruning ratios of the ablation: 1 - K / N_s
+    assert [round(100 * (1 - k / nano.n_spatial), 2) for k in W.PAPER_PRUNING_BUDGETS] == [28.89, 48.89, 68.89]
+    assert W.variant_workload(nano, "combined").budgets == (80, 104)
+    assert W.variant_workload(nano, "core_only").budgets == (184, 0)
+    assert W.variant_workload(nano, "stable_only").budgets == (0, 184)
+    assert W.variant_workload(nano, "random").budgets == (184, 0)
+    for k in W.PAPER_PRUNING_BUDGETS:
+        kc, ks = W.variant_workload(nano, "combined", k).budgets
+        assert kc + ks == k and abs(kc / k - 10 / 23) < 0.01
+        assert W.variant_workload(nano, "combined", k).packed_len == nano.n_obs + nano.n_frames * k + nano.n_action
