@@ -35,8 +35,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel's launches in one cycle (dense launch + packed
 # launch), from the ncu captures summarised in profiles/attn_bf16_tc_*.txt
 DOMINANT_KERNEL_DRAM_BYTES = {
-    "larger_imagination": int((228.174336 + 56.776192 + 87.152896 + 10.919168) * 1e6),
-    "multi_view": int((639.898880 + 198.045696 + 257.214464 + 71.534336) * 1e6),   # profiles/attn_bf16_tc_multi_view.txt
+    "larger_imagination": int((228.167680 + 58.832384 + 87.183104 + 10.037504) * 1e6),
+    "multi_view": int((639.497472 + 197.336064 + 257.351168 + 70.517760) * 1e6),   # profiles/attn_bf16_tc_multi_view.txt
 }
 
 
