@@ -246,19 +246,9 @@ __global__ void __launch_bounds__(kQualThreads) quality_kernel(const float* scor
 }
 
 // ---- action-row normalisers over all L keys -----------------------------------------------------------
-// bf16: each CTA takes 128 keys (8 warps x 16), loops over heads, multiplies against all H action queries
-// (NT = H/8 column tiles) and keeps a running (max, sum) per query in the log2 domain; the per-CTA partials
-// go to scratch [B, chunks, N_h, H] and a second kernel merges them.
+// bf16: CTAs take (head, range of keys) pairs and leave a running (max, sum) per query in the log2 domain in scratch
+// [B, ranges, N_h, H]; a second kernel merges the ranges.  The scratch holds one range per 128 keys at most.
 constexpr int kLseKeys = 128;
-constexpr int kLseThreads = 256;
-
-struct LseParams {
-  const __nv_bfloat16* q;
-  const __nv_bfloat16* k;
-  float2* partial;
-  int H, N_h, L, n_chunks, NT;
-  float scale_log2;
-};
 
 __device__ __forceinline__ void merge_ms(float& m, float& s, float m2, float s2) {
   const float mn = fmaxf(m, m2);
@@ -267,109 +257,161 @@ __device__ __forceinline__ void merge_ms(float& m, float& s, float m2, float s2)
   m = mn;
 }
 
-constexpr int kLseHeads = 4;  // heads per CTA
+// ---------------------------------------------------------------------------------------------------------
+// lambda over all L keys, flash style (the first half of an attention step: scores and running row statistics,
+// no values).  A CTA owns up to 64 action queries of one head and a contiguous range of key tiles: the query tile
+// is read once into registers as mma.sync A fragments (ldmatrix), key tiles of 64 rows stream through a two-stage
+// cp.async pipeline into XOR-swizzled shared memory, and every thread keeps the running (max, sum) of its two query
+// rows over the key columns it owns, so the only cross-lane traffic is one quad reduction at the very end.
+// WM warps split the query rows (16 each), the remaining 4 / WM warp groups split each key tile's columns.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kFlashBN = 64, kFlashThreads = 128;
 
+struct LseFlashParams {
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k;
+  float2* partial;          // [B, n_splits, N_h, H] (max, sum) in the log2 domain
+  int H, N_h, L, n_splits, tiles_per_split;
+  float scale_log2;
+};
+
+__device__ __forceinline__ void lse_cp_async16(uint32_t dst, const void* src, int src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void lse_ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+// byte offset of 16-byte chunk c of row r in a tile with CPR chunks per row
+template <int CPR>
+__device__ __forceinline__ uint32_t lse_swz(int r, int c) {
+  const int x = (CPR >= 8) ? (r & 7) : ((r >> 1) & 3);
+  return (uint32_t)((r * CPR + (c ^ x)) << 4);
+}
+// rows [row0, row0 + 64) of one head into a swizzled tile; rows at or beyond row_end are zero-filled
 template <int D>
-__global__ void __launch_bounds__(kLseThreads) lse_partial_bf16_kernel(const LseParams p) {
-  constexpr int KB = D / 32;
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int n_frag = KB * p.NT * 32;
-  uint4* q_frag = reinterpret_cast<uint4*>(smem_raw);                     // [2][KB][NT][32]
-  float2* wpart = reinterpret_cast<float2*>(q_frag + (size_t)2 * n_frag);  // [8 warps][NT*8]
-
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int chunk = blockIdx.x, h0 = blockIdx.y * kLseHeads, b = blockIdx.z;
-  const int64_t tok = (int64_t)p.N_h * D;
-  const int gq = lane >> 2, t = lane & 3;
-  const int r0 = chunk * kLseKeys + warp * 16 + gq, r1 = r0 + 8;
-  const bool v0 = r0 < p.L, v1 = r1 < p.L;
-  const __nv_bfloat16* k0 = p.k + ((int64_t)b * p.L + (v0 ? r0 : 0)) * tok + t * 8;
-  const __nv_bfloat16* k1 = p.k + ((int64_t)b * p.L + (v1 ? r1 : 0)) * tok + t * 8;
-  const int64_t act0 = (int64_t)p.L - p.H;
-  const uint4 zero = make_uint4(0, 0, 0, 0);
-
-  auto stage_q = [&](int h, int buf) {  // this head's H queries as B fragments, asynchronously
-    for (int i = tid; i < n_frag; i += kLseThreads) {
-      const int ln = i & 31;
-      const int nt = (i >> 5) % p.NT;
-      const int kb = (i >> 5) / p.NT;
-      const int n = nt * 8 + (ln >> 2);
-      const bool in = n < p.H;
-      const __nv_bfloat16* src = p.q + ((int64_t)b * p.L + act0 + (in ? n : 0)) * tok + (int64_t)h * D + kb * 32 + (ln & 3) * 8;
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
-                   ::"r"((uint32_t)__cvta_generic_to_shared(q_frag + (size_t)buf * n_frag + i)), "l"(src), "r"(in ? 16 : 0)
-                   : "memory");
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-  };
-  uint4 a0[2][KB], a1[2][KB];
-  auto load_k = [&](int h, int buf) {
+__device__ __forceinline__ void lse_load_tile(uint32_t dst, const __nv_bfloat16* base, int64_t row_stride, int row0,
+                                              int row_end, int tid) {
+  constexpr int CPR = D / 8;
 #pragma unroll
-    for (int kb = 0; kb < KB; ++kb) {
-      a0[buf][kb] = v0 ? ldg_stream(k0 + (int64_t)h * D + kb * 32) : zero;
-      a1[buf][kb] = v1 ? ldg_stream(k1 + (int64_t)h * D + kb * 32) : zero;
-    }
-  };
-
-  stage_q(h0, 0);
-  load_k(h0, 0);
-#pragma unroll
-  for (int hi = 0; hi < kLseHeads; ++hi) {
-    const int h = h0 + hi;
-    if (h >= p.N_h) break;
-    const bool more = (hi + 1 < kLseHeads) && (h + 1 < p.N_h);
-    if (more) {
-      stage_q(h + 1, (hi + 1) & 1);
-      load_k(h + 1, (hi + 1) & 1);
-      asm volatile("cp.async.wait_group 1;" ::: "memory");
-    } else {
-      asm volatile("cp.async.wait_group 0;" ::: "memory");
-    }
-    __syncthreads();
-    const uint4* qf = q_frag + (size_t)(hi & 1) * n_frag;
-    for (int nt = 0; nt < p.NT; ++nt) {
-      float c[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int kb = 0; kb < KB; ++kb) {
-        const uint4 bq = qf[(kb * p.NT + nt) * 32 + lane];
-        mma_bf16_16816(c, a0[hi & 1][kb].x, a1[hi & 1][kb].x, a0[hi & 1][kb].y, a1[hi & 1][kb].y, bq.x, bq.y);
-        mma_bf16_16816(c, a0[hi & 1][kb].z, a1[hi & 1][kb].z, a0[hi & 1][kb].w, a1[hi & 1][kb].w, bq.z, bq.w);
-      }
-      // columns 2t, 2t+1; rows gq (c0, c1) and gq+8 (c2, c3): column max over the warp's 16 keys, then the sum
-      const float x00 = v0 ? c[0] * p.scale_log2 : -INFINITY, x01 = v0 ? c[1] * p.scale_log2 : -INFINITY;
-      const float x10 = v1 ? c[2] * p.scale_log2 : -INFINITY, x11 = v1 ? c[3] * p.scale_log2 : -INFINITY;
-      float m0 = fmaxf(x00, x10), m1 = fmaxf(x01, x11);
-#pragma unroll
-      for (int o = 4; o < 32; o <<= 1) {
-        m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, o));
-        m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o));
-      }
-      float s0 = (m0 == -INFINITY) ? 0.f : exp2f(x00 - m0) + exp2f(x10 - m0);
-      float s1 = (m1 == -INFINITY) ? 0.f : exp2f(x01 - m1) + exp2f(x11 - m1);
-#pragma unroll
-      for (int o = 4; o < 32; o <<= 1) {
-        s0 += __shfl_xor_sync(0xffffffffu, s0, o);
-        s1 += __shfl_xor_sync(0xffffffffu, s1, o);
-      }
-      if (gq == 0) {
-        wpart[warp * p.NT * 8 + nt * 8 + 2 * t] = make_float2(m0, s0);
-        wpart[warp * p.NT * 8 + nt * 8 + 2 * t + 1] = make_float2(m1, s1);
-      }
-    }
-    __syncthreads();
-    for (int n = tid; n < p.H; n += kLseThreads) {
-      float m = -INFINITY, sacc = 0.f;
-      for (int w = 0; w < 8; ++w) {
-        const float2 ws = wpart[w * p.NT * 8 + n];
-        merge_ms(m, sacc, ws.x, ws.y);
-      }
-      p.partial[(((int64_t)b * p.n_chunks + chunk) * p.N_h + h) * p.H + n] = make_float2(m, sacc);
-    }
-    // the next head's barrier (after its wait) orders these reads of wpart before its writes
+  for (int i = tid; i < 64 * CPR; i += kFlashThreads) {
+    const int r = i / CPR, c = i % CPR;
+    const int gr = row0 + r;
+    const bool in = gr < row_end;
+    lse_cp_async16(dst + lse_swz<CPR>(r, c), base + (int64_t)(in ? gr : row0) * row_stride + c * 8, in ? 16 : 0);
   }
 }
 
-// merges the per-chunk partials: lambda = ln2 * (m + log2 s); one warp per (sample, head, query)
+template <int D, int WM>
+__global__ void __launch_bounds__(kFlashThreads) lse_flash_bf16_kernel(const LseFlashParams p) {
+  constexpr int CPR = D / 8, KS = D / 16;
+  constexpr int WN = 4 / WM;                 // warp groups over the key columns
+  constexpr int NPW = kFlashBN / 16 / WN;    // 16-key column pairs per warp and tile
+  extern __shared__ __align__(128) unsigned char smem[];
+  const uint32_t sQ = (uint32_t)__cvta_generic_to_shared(smem);
+  const uint32_t sK = sQ + 64 * D * 2;
+  float2* s_red = reinterpret_cast<float2*>(smem);   // reused after the loop: [WN][64]
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gq = lane >> 2, t = lane & 3;
+  const int wm = warp % WM, wn = warp / WM;
+  const int split = blockIdx.x, h = blockIdx.y;
+  const int q_chunks = (p.H + 63) / 64;
+  const int b = blockIdx.z / q_chunks, qc = blockIdx.z % q_chunks;
+  const int64_t rs = (int64_t)p.N_h * D;
+  const __nv_bfloat16* kb = p.k + (int64_t)b * p.L * rs + (int64_t)h * D;
+  const __nv_bfloat16* qb = p.q + ((int64_t)b * p.L + (p.L - p.H)) * rs + (int64_t)h * D;   // action rows
+  const int n_tiles = (p.L + kFlashBN - 1) / kFlashBN;
+  const int j0 = split * p.tiles_per_split, j1 = min(n_tiles, j0 + p.tiles_per_split);
+
+  lse_load_tile<D>(sQ, qb, rs, qc * 64, p.H, tid);
+  if (j0 < j1) lse_load_tile<D>(sK, kb, rs, j0 * kFlashBN, p.L, tid);
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+
+  uint32_t qf[KS][4];
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks)
+    lse_ldsm_x4(sQ + lse_swz<CPR>(wm * 16 + (lane & 15), ks * 2 + (lane >> 4)), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+  for (int j = j0; j < j1; ++j) {
+    const int buf = (j - j0) & 1;
+    if (j + 1 < j1) {
+      lse_load_tile<D>(sK + (buf ^ 1) * kFlashBN * D * 2, kb, rs, (j + 1) * kFlashBN, p.L, tid);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    const uint32_t kt = sK + buf * kFlashBN * D * 2;
+    float s[2 * NPW][4];
+#pragma unroll
+    for (int i = 0; i < 2 * NPW; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+      for (int np = 0; np < NPW; ++np) {
+        const int key16 = (wn * NPW + np) * 16;
+        uint32_t b0, b1, b2, b3;
+        lse_ldsm_x4(kt + lse_swz<CPR>(key16 + (lane & 7) + ((lane >> 4) << 3), ks * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
+        mma_bf16_16816(s[2 * np], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b0, b1);
+        mma_bf16_16816(s[2 * np + 1], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b2, b3);
+      }
+    }
+    // log2 domain; keys beyond the sequence count as -inf
+    const int c_base = j * kFlashBN + wn * NPW * 16 + 2 * t;
+    const bool tail = (j + 1) * kFlashBN > p.L;
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      float mx = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 2 * NPW; ++i) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int c = c_base + i * 8 + e;
+          float v = s[i][2 * r + e] * p.scale_log2;
+          if (tail && c >= p.L) v = -INFINITY;
+          s[i][2 * r + e] = v;
+          mx = fmaxf(mx, v);
+        }
+      }
+      const float m_new = fmaxf(m_run[r], mx);
+      if (m_new != -INFINITY) {
+        float ps = 0.f;
+#pragma unroll
+        for (int i = 0; i < 2 * NPW; ++i) ps += exp2f(s[i][2 * r] - m_new) + exp2f(s[i][2 * r + 1] - m_new);
+        l_run[r] = l_run[r] * exp2f(m_run[r] - m_new) + ps;
+        m_run[r] = m_new;
+      }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+  }
+  // rows wm * 16 + gq (+ 8): merge the quad's four column subsets, then the WN warp groups through shared memory
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+#pragma unroll
+    for (int o = 1; o <= 2; o <<= 1) {
+      const float om = __shfl_xor_sync(0xffffffffu, m_run[r], o), os = __shfl_xor_sync(0xffffffffu, l_run[r], o);
+      merge_ms(m_run[r], l_run[r], om, os);
+    }
+  }
+  __syncthreads();   // the tiles are no longer read
+  if (t == 0) {
+    s_red[wn * 64 + wm * 16 + gq] = make_float2(m_run[0], l_run[0]);
+    s_red[wn * 64 + wm * 16 + gq + 8] = make_float2(m_run[1], l_run[1]);
+  }
+  __syncthreads();
+  if (tid < WM * 16) {
+    const int i = qc * 64 + tid;
+    if (i < p.H) {
+      float m = -INFINITY, l = 0.f;
+#pragma unroll
+      for (int g = 0; g < WN; ++g) merge_ms(m, l, s_red[g * 64 + tid].x, s_red[g * 64 + tid].y);
+      p.partial[(((int64_t)b * p.n_splits + split) * p.N_h + h) * p.H + i] = make_float2(m, l);
+    }
+  }
+}
+
 __global__ void __launch_bounds__(256) lse_merge_kernel(const float2* partial, float* lse, int n_chunks, int N_h, int H) {
   const int lane = threadIdx.x & 31;
   const int i = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -536,30 +578,45 @@ cudaError_t launch_action_lse(const Dims& d, const void* q, const void* k, float
     lse_f32_kernel<<<grid, 128, 0, st>>>((const float*)q, (const float*)k, lse, d.L, d.H, d.N_h, d.D, d.scale);
     return cudaGetLastError();
   }
-  const int n_chunks = (d.L + kLseKeys - 1) / kLseKeys;
-  const int NT = (d.H + 7) / 8;
-  LseParams p{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (float2*)scratch, d.H, d.N_h, d.L, n_chunks, NT,
-              d.scale * kLog2e};
-  const size_t smem = (size_t)2 * (d.D / 32) * NT * 32 * sizeof(uint4) + (size_t)8 * NT * 8 * sizeof(float2);
-  if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
-  dim3 grid(n_chunks, (d.N_h + kLseHeads - 1) / kLseHeads, d.B);
+  // key ranges per CTA: enough CTAs for about four per SM, never more ranges than the scratch has room for
+  const int n_tiles = (d.L + kFlashBN - 1) / kFlashBN;
+  const int q_chunks = (d.H + 63) / 64;
+  const int max_splits = (d.L + kLseKeys - 1) / kLseKeys;
+  int sms = 148;
+  {
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  }
+  int want = (4 * sms + d.N_h * d.B * q_chunks - 1) / (d.N_h * d.B * q_chunks);
+  want = want < 1 ? 1 : (want > max_splits ? max_splits : want);
+  const int per = (n_tiles + want - 1) / want;
+  const int n_chunks = (n_tiles + per - 1) / per;     // = number of key ranges
+  LseFlashParams p{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (float2*)scratch, d.H, d.N_h, d.L, n_chunks, per,
+                   d.scale * kLog2e};
+  const int wm = d.H >= 64 ? 4 : (d.H > 16 ? 2 : 1);    // warps over the query rows (H <= 16, <= 32, more)
+  dim3 grid(n_chunks, d.N_h, d.B * q_chunks);
   cudaError_t e = cudaSuccess;
   *launches += 2;
+#define SWAM_LSE_LAUNCH(D_, WM_)                                                                                        \
+  do {                                                                                                                  \
+    const size_t smem = (size_t)(64 + 2 * kFlashBN) * D_ * 2;                                                           \
+    e = cudaFuncSetAttribute(lse_flash_bf16_kernel<D_, WM_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);   \
+    if (e == cudaSuccess) lse_flash_bf16_kernel<D_, WM_><<<grid, kFlashThreads, smem, st>>>(p);                         \
+  } while (0)
+#define SWAM_LSE_DISPATCH(D_)                                                                                           \
+  do {                                                                                                                  \
+    if (wm == 4) SWAM_LSE_LAUNCH(D_, 4);                                                                                \
+    else if (wm == 2) SWAM_LSE_LAUNCH(D_, 2);                                                                           \
+    else SWAM_LSE_LAUNCH(D_, 1);                                                                                        \
+  } while (0)
   switch (d.D) {
-    case 32:
-      e = cudaFuncSetAttribute(lse_partial_bf16_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e == cudaSuccess) lse_partial_bf16_kernel<32><<<grid, kLseThreads, smem, st>>>(p);
-      break;
-    case 64:
-      e = cudaFuncSetAttribute(lse_partial_bf16_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e == cudaSuccess) lse_partial_bf16_kernel<64><<<grid, kLseThreads, smem, st>>>(p);
-      break;
-    case 128:
-      e = cudaFuncSetAttribute(lse_partial_bf16_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e == cudaSuccess) lse_partial_bf16_kernel<128><<<grid, kLseThreads, smem, st>>>(p);
-      break;
+    case 32: SWAM_LSE_DISPATCH(32); break;
+    case 64: SWAM_LSE_DISPATCH(64); break;
+    case 128: SWAM_LSE_DISPATCH(128); break;
     default: return cudaErrorInvalidConfiguration;
   }
+#undef SWAM_LSE_DISPATCH
+#undef SWAM_LSE_LAUNCH
   if (e != cudaSuccess) return e;
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
