@@ -1,5 +1,6 @@
 """The C-ABI library loads without a GPU, exports every symbol the header declares, and rejects bad shapes
 before touching the device."""
+import numpy as np
 import ctypes
 import os
 import re
@@ -77,3 +78,12 @@ def test_shapes_beyond_the_selection_kernels_shared_memory_are_rejected(lib):
     # F * N_s scores (two maps) + keys + flags must fit one SM's shared memory
     assert _create(lib, n_frames=8, n_spatial=8192, n_action=32, k_core=10, k_anchor=10) == swam.ERR_UNSUPPORTED
     assert _create(lib, n_obs=1 << 25) == swam.ERR_UNSUPPORTED            # sequence length limit
+
+
+def test_degree4_exp2_polynomial_bound():
+    """The softmax pass of the head-dim-64 attention kernel evaluates one exponential in eight as
+    2^round(x) * p(x - round(x)); this pins the coefficients' error bound against the library exp2."""
+    c = [0.9999992847442627, 0.6931217908859253, 0.240247443318367, 0.05591785907745361, 0.009570102207362652]
+    f = np.linspace(-0.5, 0.5, 200001)
+    p = ((((c[4] * f + c[3]) * f + c[2]) * f + c[1]) * f + c[0])
+    assert np.abs(p / np.exp2(f) - 1).max() < 3e-6

@@ -422,3 +422,4 @@ def test_select2_uses_core_map_for_cores_and_all_map_for_anchors():
     v_all[0, :, 3] = 0.95                      # core position: must not become an anchor
     sel = ora.select2(v_core, v_all, kc, ks)
     assert sel[0, 0].tolist() == [2, 3, 7, 10, 11] and sel[0, 1].tolist() == [1, 2, 5, 10, 11]
+
