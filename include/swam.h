@@ -56,7 +56,13 @@ typedef struct {
   float softmax_scale;        /* 0 => 1/sqrt(head_dim) */
   float cv_beta;              /* coefficient of the cross-frame variation penalty; the paper uses 1.0 */
   const float* query_weights; /* host, [H/F], non-negative, sums to 1; NULL => central half 2x outer quarters */
+  int32_t n_kv_heads;         /* key/value heads (grouped-query attention); 0 => n_heads; must divide n_heads */
 } swam_shape;
+
+/* Tensor layouts.  Q and every output are [B, L, n_heads, head_dim]; K and V are [B, L, n_kv_heads, head_dim]
+ * (packed tensors likewise with L' rows).  Query head h reads key/value head h / (n_heads / n_kv_heads): the backbone's
+ * head mapping, which the scoring follows (App. A.2).  With n_kv_heads = n_heads (the default) all four tensors have the
+ * same shape. */
 
 /* Context: validates the shape (H divisible by F, Eq. 8; K_c + K_s <= N_s; head_dim in {32, 64, 128};
  * NULL weights need H/F divisible by 4) and fixes the workspace layout.  The shape (and the weights) are

@@ -60,14 +60,25 @@ def query_weights(g: int) -> np.ndarray:
     return w / w.sum()
 
 
+def expand_kv(x: np.ndarray, n_heads: int) -> np.ndarray:
+    """Grouped-query attention written out: a key/value tensor with fewer heads than the queries is the tensor in
+    which query head h finds key/value head h // (N_h / N_kv); repeating each head N_h / N_kv times gives the plain
+    multi-head problem every function below is defined on."""
+    n_kv = x.shape[2]
+    if n_kv == n_heads:
+        return x
+    assert n_heads % n_kv == 0, "the number of query heads must be a multiple of the key/value heads"
+    return np.repeat(x, n_heads // n_kv, axis=2)
+
+
 def attention_rows(q: np.ndarray, k: np.ndarray, v: np.ndarray, rows: np.ndarray,
                    scale: Optional[float] = None) -> Tuple[np.ndarray, np.ndarray]:
     """Softmax attention (Sec. 3.1) for the listed (b, r) query rows, all heads.
-    q, k, v: [B, n, N_h, D] float32.  Returns out [n_rows, N_h, D], lse [n_rows, N_h] (float64)."""
+    q: [B, n, N_h, D], k, v: [B, n, N_h or N_kv, D] float32.  Returns out [n_rows, N_h, D], lse [n_rows, N_h] (float64)."""
     lib = _load()
     q = np.ascontiguousarray(q, dtype=np.float32)
-    k = np.ascontiguousarray(k, dtype=np.float32)
-    v = np.ascontiguousarray(v, dtype=np.float32)
+    k = np.ascontiguousarray(expand_kv(k, q.shape[2]), dtype=np.float32)
+    v = np.ascontiguousarray(expand_kv(v, q.shape[2]), dtype=np.float32)
     _, n, nh, d = q.shape
     rows = np.ascontiguousarray(rows, dtype=np.int32).reshape(-1, 2)
     scale = 1.0 / np.sqrt(d) if scale is None else float(scale)
@@ -103,7 +114,7 @@ def score(q: np.ndarray, k: np.ndarray, n_obs: int, n_frames: int, n_spatial: in
     """Spatial score S [B, F, N_s] (Eq. 12), float64."""
     lib = _load()
     q = np.ascontiguousarray(q, dtype=np.float32)
-    k = np.ascontiguousarray(k, dtype=np.float32)
+    k = np.ascontiguousarray(expand_kv(k, q.shape[2]), dtype=np.float32)
     b, n, nh, d = q.shape
     assert n == n_obs + n_frames * n_spatial + n_action and n_action % n_frames == 0
     scale = 1.0 / np.sqrt(d) if scale is None else float(scale)

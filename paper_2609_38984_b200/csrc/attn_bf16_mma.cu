@@ -71,16 +71,17 @@ __global__ void __launch_bounds__(kThreads) attn_bf16_mma_kernel(const AttnArgs 
   const int gq = lane >> 2, t = lane & 3;
   const int h = blockIdx.y, b = blockIdx.z;
   const int m0 = blockIdx.x * BM;
-  const int64_t rs = (int64_t)a.N_h * D;
+  const int64_t rs = (int64_t)a.N_h * D, rs_kv = (int64_t)a.N_kv * D;
+  const int h_kv = h / (a.N_h / a.N_kv);
   const __nv_bfloat16* qb = (const __nv_bfloat16*)a.q + (int64_t)b * a.n * rs + (int64_t)h * D;
-  const __nv_bfloat16* kb = (const __nv_bfloat16*)a.k + (int64_t)b * a.n * rs + (int64_t)h * D;
-  const __nv_bfloat16* vb = (const __nv_bfloat16*)a.v + (int64_t)b * a.n * rs + (int64_t)h * D;
+  const __nv_bfloat16* kb = (const __nv_bfloat16*)a.k + (int64_t)b * a.n * rs_kv + (int64_t)h_kv * D;
+  const __nv_bfloat16* vb = (const __nv_bfloat16*)a.v + (int64_t)b * a.n * rs_kv + (int64_t)h_kv * D;
   const int n_tiles = (a.n + BN - 1) / BN;
   const float sl2 = a.scale * kLog2e;
 
   load_tile<D>(sQ, qb, rs, m0, a.n, tid);
-  load_tile<D>(sK, kb, rs, 0, a.n, tid);
-  load_tile<D>(sV, vb, rs, 0, a.n, tid);
+  load_tile<D>(sK, kb, rs_kv, 0, a.n, tid);
+  load_tile<D>(sV, vb, rs_kv, 0, a.n, tid);
   cp_async_commit();
   cp_async_wait_all();
   __syncthreads();
@@ -98,8 +99,8 @@ __global__ void __launch_bounds__(kThreads) attn_bf16_mma_kernel(const AttnArgs 
   for (int j = 0; j < n_tiles; ++j) {
     const int buf = j & 1;
     if (j + 1 < n_tiles) {
-      load_tile<D>(sK + (buf ^ 1) * BN * D * 2, kb, rs, (j + 1) * BN, a.n, tid);
-      load_tile<D>(sV + (buf ^ 1) * BN * D * 2, vb, rs, (j + 1) * BN, a.n, tid);
+      load_tile<D>(sK + (buf ^ 1) * BN * D * 2, kb, rs_kv, (j + 1) * BN, a.n, tid);
+      load_tile<D>(sV + (buf ^ 1) * BN * D * 2, vb, rs_kv, (j + 1) * BN, a.n, tid);
       cp_async_commit();
     }
     const uint32_t kt = sK + buf * BN * D * 2, vt = sV + buf * BN * D * 2;

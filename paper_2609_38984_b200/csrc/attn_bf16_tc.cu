@@ -246,6 +246,7 @@ struct TcParams {
   const __nv_bfloat16* q_full;  // gather mode: the full [B, n_full, N_h, D] query tensor
   int lse_row0, lse_rows;
   int n, N_h;
+  int kv_group;        // query heads per key/value head
   int pairs;           // query tile pairs per (sample, head)
   int n_whole;         // work items that run over all keys and write the output themselves
   int splits;          // pieces per split item (0 when nothing is split)
@@ -443,12 +444,12 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (!ok) break;
         mbar_expect_tx(bar_k_full(st), C::kTileBytes);
         for (int db = 0; db < C::DB; ++db)
-          tma_load_4d(sK + st * C::kTileBytes + db * C::kSubTile, &map_k, bar_k_full(st), db * 64, (kv_begin + j) * kTile, h, b);
+          tma_load_4d(sK + st * C::kTileBytes + db * C::kSubTile, &map_k, bar_k_full(st), db * 64, (kv_begin + j) * kTile, h / p.kv_group, b);
         ok = mbar_wait(bar_v_empty(st), par, abort_flag);
         if (!ok) break;
         mbar_expect_tx(bar_v_full(st), C::kTileBytes);
         for (int db = 0; db < C::DB; ++db)
-          tma_load_4d(sV + st * C::kTileBytes + db * C::kSubTile, &map_v, bar_v_full(st), db * 64, (kv_begin + j) * kTile, h, b);
+          tma_load_4d(sV + st * C::kTileBytes + db * C::kSubTile, &map_v, bar_v_full(st), db * 64, (kv_begin + j) * kTile, h / p.kv_group, b);
       }
     }
    } else if (warp == 8) {
@@ -863,7 +864,7 @@ cudaError_t launch_tc_d(const AttnArgs& a, const int32_t* pack_map, int n_full, 
   CUtensorMap mq, mk, mv, mo;
   if (!(MODE != kDirect ? make_map(&mo, a.out, a.B, n_full, a.N_h, D, 1) : make_map(&mo, a.out, a.B, a.n, a.N_h, D)))
     return cudaErrorInvalidValue;
-  if (!make_map(&mk, a.k, a.B, a.n, a.N_h, D) || !make_map(&mv, a.v, a.B, a.n, a.N_h, D)) return cudaErrorInvalidValue;
+  if (!make_map(&mk, a.k, a.B, a.n, a.N_kv, D) || !make_map(&mv, a.v, a.B, a.n, a.N_kv, D)) return cudaErrorInvalidValue;
   if (MODE == kGather) {
     mq = mo;   // not used by the kernel
   } else if (!make_map(&mq, a.q, a.B, a.n, a.N_h, D)) {
@@ -891,7 +892,7 @@ cudaError_t launch_tc_d(const AttnArgs& a, const int32_t* pack_map, int n_full, 
 #ifdef SWAM_TC_TRACE
       (long long*)partial_trace_buffer(),
 #endif
-      a.lse, status, partial, pack_map, n_full, (const __nv_bfloat16*)a.q, a.lse_row0, a.lse_rows, a.n, a.N_h, pairs, n_whole, splits, per,
+      a.lse, status, partial, pack_map, n_full, (const __nv_bfloat16*)a.q, a.lse_row0, a.lse_rows, a.n, a.N_h, a.N_h / a.N_kv, pairs, n_whole, splits, per,
       a.scale * kLog2e};
   const int grid = n_whole + (splits ? rem * splits : 0);
   ++*launches;

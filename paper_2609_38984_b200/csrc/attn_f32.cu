@@ -19,8 +19,10 @@ __global__ void __launch_bounds__(kRows * 32) attn_f32_kernel(const AttnArgs a) 
   const bool active = row < a.n;
   const int64_t tok = (int64_t)a.N_h * D;
   const float* q = (const float*)a.q + ((int64_t)b * a.n) * tok + (int64_t)h * D;
-  const float* k = (const float*)a.k + ((int64_t)b * a.n) * tok + (int64_t)h * D;
-  const float* v = (const float*)a.v + ((int64_t)b * a.n) * tok + (int64_t)h * D;
+  const int64_t tok_kv = (int64_t)a.N_kv * D;
+  const int h_kv = h / (a.N_h / a.N_kv);
+  const float* k = (const float*)a.k + ((int64_t)b * a.n) * tok_kv + (int64_t)h_kv * D;
+  const float* v = (const float*)a.v + ((int64_t)b * a.n) * tok_kv + (int64_t)h_kv * D;
   if (active)
     for (int d = lane; d < D; d += 32) Qs[warp][d] = q[(int64_t)row * tok + d];
 
@@ -35,8 +37,8 @@ __global__ void __launch_bounds__(kRows * 32) attn_f32_kernel(const AttnArgs a) 
     for (int i = threadIdx.x; i < kKeys * D; i += kRows * 32) {
       const int kk = i / D, d = i % D;
       const bool in = c0 + kk < a.n;
-      Ks[kk][d] = in ? k[(int64_t)(c0 + kk) * tok + d] : 0.f;
-      Vs[kk][d] = in ? v[(int64_t)(c0 + kk) * tok + d] : 0.f;
+      Ks[kk][d] = in ? k[(int64_t)(c0 + kk) * tok_kv + d] : 0.f;
+      Vs[kk][d] = in ? v[(int64_t)(c0 + kk) * tok_kv + d] : 0.f;
     }
     __syncthreads();
     if (!active) continue;

@@ -219,16 +219,30 @@ cudaError_t launch_row_copy(RowCopyParams& p, int batch, cudaStream_t st) {
 
 cudaError_t launch_pack(const Dims& d, const void* const src[3], void* const dst[3], const int32_t* pack_map,
                         int* status, cudaStream_t st, int* launches) {
-  RowCopyParams p{};
-  int n = 0;
-  for (int i = 0; i < 3; ++i)
-    if (src[i] && dst[i]) { p.src[n] = (const unsigned char*)src[i]; p.dst[n] = (unsigned char*)dst[i]; ++n; }
-  if (n == 0 || d.Lp == 0) return cudaSuccess;
-  p.src_idx = pack_map; p.dst_idx = nullptr; p.status = status;
-  p.n_tensors = n; p.n_rows = d.Lp; p.src_rows = d.L; p.dst_rows = d.Lp;
-  p.row_bytes = d.N_h * d.D * (d.dtype == 0 ? 4 : 2);
-  ++*launches;
-  return launch_row_copy(p, d.B, st);
+  if (d.Lp == 0) return cudaSuccess;
+  const int eb = d.dtype == 0 ? 4 : 2;
+  // tensors with the same row size share a launch: Q has N_h heads per row, K and V have N_kv
+  const int rows_of[3] = {d.N_h * d.D * eb, d.N_kv * d.D * eb, d.N_kv * d.D * eb};
+  bool done[3] = {false, false, false};
+  for (int first = 0; first < 3; ++first) {
+    if (done[first] || !src[first] || !dst[first]) continue;
+    RowCopyParams p{};
+    int n = 0;
+    for (int i = first; i < 3; ++i)
+      if (!done[i] && src[i] && dst[i] && rows_of[i] == rows_of[first]) {
+        p.src[n] = (const unsigned char*)src[i];
+        p.dst[n] = (unsigned char*)dst[i];
+        ++n;
+        done[i] = true;
+      }
+    p.src_idx = pack_map; p.dst_idx = nullptr; p.status = status;
+    p.n_tensors = n; p.n_rows = d.Lp; p.src_rows = d.L; p.dst_rows = d.Lp;
+    p.row_bytes = rows_of[first];
+    ++*launches;
+    cudaError_t e = launch_row_copy(p, d.B, st);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 cudaError_t launch_scatter(const Dims& d, const void* out_p, const int32_t* pack_map, const int32_t* inv_map,

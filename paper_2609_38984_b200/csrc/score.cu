@@ -45,6 +45,7 @@ struct ScoreParams {
   int n_obs, F, N_s, H, N_h, L, g;
   float scale_log2, inv_nh;
   Alpha alpha;
+  int N_kv;          // heads of k; query head h reads key head h / (N_h / N_kv)
 };
 
 
@@ -90,9 +91,11 @@ __global__ void __launch_bounds__(32 * MT * kHeadGroups, 16 / (MT * kHeadGroups)
   const int gq = lane >> 2, t = lane & 3;
   const int r0 = key0 + mt * 16 + gq, r1 = r0 + 8;
   const bool v0 = r0 < p.N_s, v1 = r1 < p.N_s;
-  const __nv_bfloat16* kbase = p.k + ((int64_t)b * p.L + p.n_obs + (int64_t)f * p.N_s) * tok + t * 8;
-  const __nv_bfloat16* k0 = kbase + (int64_t)(v0 ? r0 : 0) * tok;
-  const __nv_bfloat16* k1 = kbase + (int64_t)(v1 ? r1 : 0) * tok;
+  const int64_t tok_k = (int64_t)p.N_kv * D;
+  const int kv_group = p.N_h / p.N_kv;
+  const __nv_bfloat16* kbase = p.k + ((int64_t)b * p.L + p.n_obs + (int64_t)f * p.N_s) * tok_k + t * 8;
+  const __nv_bfloat16* k0 = kbase + (int64_t)(v0 ? r0 : 0) * tok_k;
+  const __nv_bfloat16* k1 = kbase + (int64_t)(v1 ? r1 : 0) * tok_k;
 
   float w[NT][2];
 #pragma unroll
@@ -107,8 +110,8 @@ __global__ void __launch_bounds__(32 * MT * kHeadGroups, 16 / (MT * kHeadGroups)
   auto load = [&](int h, int buf) {
 #pragma unroll
     for (int kb = 0; kb < KB; ++kb) {
-      a0[buf][kb] = v0 ? ldg_stream(k0 + (int64_t)h * D + kb * 32) : zero;
-      a1[buf][kb] = v1 ? ldg_stream(k1 + (int64_t)h * D + kb * 32) : zero;
+      a0[buf][kb] = v0 ? ldg_stream(k0 + (int64_t)(h / kv_group) * D + kb * 32) : zero;
+      a1[buf][kb] = v1 ? ldg_stream(k1 + (int64_t)(h / kv_group) * D + kb * 32) : zero;
     }
   };
   auto compute = [&](int h, int buf) {
@@ -176,6 +179,7 @@ struct ScoreParamsF32 {
   int n_obs, F, N_s, H, N_h, D, L, g;
   float scale, inv_nh;
   Alpha alpha;
+  int N_kv;
 };
 
 __global__ void __launch_bounds__(256) score_f32_kernel(const ScoreParamsF32 p) {
@@ -185,14 +189,15 @@ __global__ void __launch_bounds__(256) score_f32_kernel(const ScoreParamsF32 p) 
   if (j >= p.N_s) return;
   const int64_t tok = (int64_t)p.N_h * p.D;
   const int64_t act0 = (int64_t)p.n_obs + (int64_t)p.F * p.N_s;
-  const float* kt = p.k + ((int64_t)b * p.L + p.n_obs + (int64_t)f * p.N_s + j) * tok;
+  const int kv_group = p.N_h / p.N_kv;
+  const float* kt = p.k + ((int64_t)b * p.L + p.n_obs + (int64_t)f * p.N_s + j) * ((int64_t)p.N_kv * p.D);
   float acc = 0.f;
   for (int a = 0; a < p.g; ++a) {
     const int i = f * p.g + a;
     const float* qt = p.q + ((int64_t)b * p.L + act0 + i) * tok;
     for (int h = 0; h < p.N_h; ++h) {
       float dot = 0.f;
-      for (int d = lane; d < p.D; d += 32) dot = fmaf(qt[h * p.D + d], kt[h * p.D + d], dot);
+      for (int d = lane; d < p.D; d += 32) dot = fmaf(qt[h * p.D + d], kt[(h / kv_group) * p.D + d], dot);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
       acc += p.alpha.w[a] * expf(p.scale * dot - p.lse[((int64_t)b * p.N_h + h) * p.H + i]);
@@ -273,6 +278,7 @@ struct LseFlashParams {
   float2* partial;          // [B, n_splits, N_h, H] (max, sum) in the log2 domain
   int H, N_h, L, n_splits, tiles_per_split;
   float scale_log2;
+  int N_kv;
 };
 
 __device__ __forceinline__ void lse_cp_async16(uint32_t dst, const void* src, int src_bytes) {
@@ -318,14 +324,14 @@ __global__ void __launch_bounds__(kFlashThreads) lse_flash_bf16_kernel(const Lse
   const int split = blockIdx.x, h = blockIdx.y;
   const int q_chunks = (p.H + 63) / 64;
   const int b = blockIdx.z / q_chunks, qc = blockIdx.z % q_chunks;
-  const int64_t rs = (int64_t)p.N_h * D;
-  const __nv_bfloat16* kb = p.k + (int64_t)b * p.L * rs + (int64_t)h * D;
+  const int64_t rs = (int64_t)p.N_h * D, rs_k = (int64_t)p.N_kv * D;
+  const __nv_bfloat16* kb = p.k + (int64_t)b * p.L * rs_k + (int64_t)(h / (p.N_h / p.N_kv)) * D;
   const __nv_bfloat16* qb = p.q + ((int64_t)b * p.L + (p.L - p.H)) * rs + (int64_t)h * D;   // action rows
   const int n_tiles = (p.L + kFlashBN - 1) / kFlashBN;
   const int j0 = split * p.tiles_per_split, j1 = min(n_tiles, j0 + p.tiles_per_split);
 
   lse_load_tile<D>(sQ, qb, rs, qc * 64, p.H, tid);
-  if (j0 < j1) lse_load_tile<D>(sK, kb, rs, j0 * kFlashBN, p.L, tid);
+  if (j0 < j1) lse_load_tile<D>(sK, kb, rs_k, j0 * kFlashBN, p.L, tid);
   asm volatile("cp.async.commit_group;" ::: "memory");
   asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
@@ -339,7 +345,7 @@ __global__ void __launch_bounds__(kFlashThreads) lse_flash_bf16_kernel(const Lse
   for (int j = j0; j < j1; ++j) {
     const int buf = (j - j0) & 1;
     if (j + 1 < j1) {
-      lse_load_tile<D>(sK + (buf ^ 1) * kFlashBN * D * 2, kb, rs, (j + 1) * kFlashBN, p.L, tid);
+      lse_load_tile<D>(sK + (buf ^ 1) * kFlashBN * D * 2, kb, rs_k, (j + 1) * kFlashBN, p.L, tid);
       asm volatile("cp.async.commit_group;" ::: "memory");
     }
     const uint32_t kt = sK + buf * kFlashBN * D * 2;
@@ -432,14 +438,14 @@ __global__ void __launch_bounds__(256) lse_merge_kernel(const float2* partial, f
 
 // fp32: one CTA per (b, h, i); threads stride over keys with a running (max, sum) in natural-log units
 __global__ void __launch_bounds__(128) lse_f32_kernel(const float* q, const float* k, float* lse, int L, int H,
-                                                      int N_h, int D, float scale) {
+                                                      int N_h, int N_kv, int D, float scale) {
   __shared__ float sm[4], ss[4];
   const int i = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int64_t tok = (int64_t)N_h * D;
   const float* qt = q + ((int64_t)b * L + (L - H) + i) * tok + (int64_t)h * D;
   float m = -INFINITY, s = 0.f;
   for (int c = threadIdx.x; c < L; c += blockDim.x) {
-    const float* kt = k + ((int64_t)b * L + c) * tok + (int64_t)h * D;
+    const float* kt = k + ((int64_t)b * L + c) * ((int64_t)N_kv * D) + (int64_t)(h / (N_h / N_kv)) * D;
     float dot = 0.f;
     for (int d = 0; d < D; ++d) dot = fmaf(qt[d], kt[d], dot);
     const float x = dot * scale;
@@ -513,13 +519,13 @@ cudaError_t launch_score(const Dims& d, const Alpha& alpha, const void* q, const
   ++*launches;
   if (d.dtype == 0) {
     ScoreParamsF32 p{(const float*)q, (const float*)k, lse, scores, d.n_obs, d.F, d.N_s, d.H,
-                     d.N_h, d.D, d.L, d.g, d.scale, 1.0f / (float)d.N_h, alpha};
+                     d.N_h, d.D, d.L, d.g, d.scale, 1.0f / (float)d.N_h, alpha, d.N_kv};
     dim3 grid((d.N_s + 7) / 8, d.F, d.B);
     score_f32_kernel<<<grid, 256, 0, st>>>(p);
     return cudaGetLastError();
   }
   ScoreParams p{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, lse, scores, d.n_obs, d.F, d.N_s, d.H,
-                d.N_h, d.L, d.g, d.scale * kLog2e, 1.0f / (float)d.N_h, alpha};
+                d.N_h, d.L, d.g, d.scale * kLog2e, 1.0f / (float)d.N_h, alpha, d.N_kv};
   switch (d.D) {
     case 32: return launch_score_bf16_d<32>(d, p, st);
     case 64: return launch_score_bf16_d<64>(d, p, st);
@@ -575,7 +581,7 @@ cudaError_t launch_action_lse(const Dims& d, const void* q, const void* k, float
   if (d.dtype == 0) {
     ++*launches;
     dim3 grid(d.H, d.N_h, d.B);
-    lse_f32_kernel<<<grid, 128, 0, st>>>((const float*)q, (const float*)k, lse, d.L, d.H, d.N_h, d.D, d.scale);
+    lse_f32_kernel<<<grid, 128, 0, st>>>((const float*)q, (const float*)k, lse, d.L, d.H, d.N_h, d.N_kv, d.D, d.scale);
     return cudaGetLastError();
   }
   // key ranges per CTA: enough CTAs for about four per SM, never more ranges than the scratch has room for
@@ -592,7 +598,7 @@ cudaError_t launch_action_lse(const Dims& d, const void* q, const void* k, float
   const int per = (n_tiles + want - 1) / want;
   const int n_chunks = (n_tiles + per - 1) / per;     // = number of key ranges
   LseFlashParams p{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (float2*)scratch, d.H, d.N_h, d.L, n_chunks, per,
-                   d.scale * kLog2e};
+                   d.scale * kLog2e, d.N_kv};
   const int wm = d.H >= 64 ? 4 : (d.H > 16 ? 2 : 1);    // warps over the query rows (H <= 16, <= 32, more)
   dim3 grid(n_chunks, d.N_h, d.B * q_chunks);
   cudaError_t e = cudaSuccess;

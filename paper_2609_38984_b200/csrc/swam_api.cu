@@ -51,6 +51,8 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 size_t elem_bytes(const Dims& d) { return d.dtype == SWAM_F32 ? 4 : 2; }
 size_t full_bytes(const Dims& d) { return (size_t)d.B * d.L * d.N_h * d.D * elem_bytes(d); }
 size_t packed_bytes(const Dims& d) { return (size_t)d.B * d.Lp * d.N_h * d.D * elem_bytes(d); }
+size_t kv_full_bytes(const Dims& d) { return (size_t)d.B * d.L * d.N_kv * d.D * elem_bytes(d); }
+size_t kv_packed_bytes(const Dims& d) { return (size_t)d.B * d.Lp * d.N_kv * d.D * elem_bytes(d); }
 
 void count(swam_ctx* c) {
   c->launches += c->launches_i;
@@ -59,7 +61,7 @@ void count(swam_ctx* c) {
 
 int run_attention(swam_ctx* c, const void* q, const void* k, const void* v, int n, void* out, float* lse, int lse_row0,
                   int lse_rows, cudaStream_t st) {
-  AttnArgs a{q, k, v, out, lse, lse_row0, lse_rows, c->d.B, n, c->d.N_h, c->d.D, c->d.scale};
+  AttnArgs a{q, k, v, out, lse, lse_row0, lse_rows, c->d.B, n, c->d.N_h, c->d.D, c->d.scale, c->d.N_kv};
   cudaError_t e;
   if (c->d.dtype == SWAM_F32) {
     e = launch_attn_f32(a, st, &c->launches_i);
@@ -106,6 +108,7 @@ int swam_create(const swam_shape* s, swam_ctx** out_ctx) {
   if (s->dtype != SWAM_F32 && s->dtype != SWAM_BF16) return SWAM_ERR_INVALID_ARG;
   if (!(s->softmax_scale >= 0.f) || !(s->cv_beta >= 0.f)) return SWAM_ERR_INVALID_ARG;
   if (s->head_dim != 32 && s->head_dim != 64 && s->head_dim != 128) return SWAM_ERR_UNSUPPORTED;
+  if (s->n_kv_heads < 0 || (s->n_kv_heads > 0 && s->n_heads % s->n_kv_heads != 0)) return SWAM_ERR_INVALID_ARG;
   const int g = s->n_action / s->n_frames;
   if (g > kMaxGroup) return SWAM_ERR_UNSUPPORTED;
   if (!s->query_weights && (g % 4) != 0) return SWAM_ERR_INVALID_ARG;
@@ -117,7 +120,7 @@ int swam_create(const swam_shape* s, swam_ctx** out_ctx) {
   memset(c, 0, sizeof(*c));
   Dims& d = c->d;
   d.B = s->batch; d.n_obs = s->n_obs; d.F = s->n_frames; d.N_s = s->n_spatial; d.H = s->n_action;
-  d.N_h = s->n_heads; d.D = s->head_dim; d.Kc = s->k_core; d.Ks = s->k_anchor; d.K = d.Kc + d.Ks;
+  d.N_h = s->n_heads; d.N_kv = s->n_kv_heads > 0 ? s->n_kv_heads : s->n_heads; d.D = s->head_dim; d.Kc = s->k_core; d.Ks = s->k_anchor; d.K = d.Kc + d.Ks;
   d.L = (int)L; d.Lp = d.n_obs + d.F * d.K + d.H; d.g = g; d.dtype = s->dtype;
   d.scale = s->softmax_scale > 0.f ? s->softmax_scale : 1.0f / sqrtf((float)d.D);
   d.beta = s->cv_beta;
@@ -149,8 +152,8 @@ int swam_create(const swam_shape* s, swam_ctx** out_ctx) {
   c->off_inv = put((size_t)d.B * d.L * 4);
   c->off_scratch = put(lse_scratch_bytes(d));
   c->off_qp = put(packed_bytes(d));
-  c->off_kp = put(packed_bytes(d));
-  c->off_vp = put(packed_bytes(d));
+  c->off_kp = put(kv_packed_bytes(d));
+  c->off_vp = put(kv_packed_bytes(d));
   c->off_op = put(packed_bytes(d));
   c->attn_scratch = (d.dtype == SWAM_BF16 && d.D >= 64) ? attn_tc_scratch_bytes(d.D) : 0;
   c->off_attn = put(c->attn_scratch);
@@ -375,7 +378,7 @@ int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t 
     void* kp = c->ws + c->off_kp;
     void* vp = c->ws + c->off_vp;
     if (int r = swam_pack(c, nullptr, k, v, pm, nullptr, kp, vp, stream)) return r;
-    AttnArgs a{q, kp, vp, out, nullptr, 0, 0, d.B, d.Lp, d.N_h, d.D, d.scale};
+    AttnArgs a{q, kp, vp, out, nullptr, 0, 0, d.B, d.Lp, d.N_h, d.D, d.scale, d.N_kv};
     cudaError_t e = launch_attn_bf16_tc_gather(a, pm, d.L, (int*)(c->ws + c->off_status), c->ws + c->off_attn,
                                                c->attn_scratch, st, &c->launches_i);
     count(c);
@@ -397,7 +400,7 @@ int swam_step_host(swam_ctx* c, const void* q_host, const void* k_host, const vo
   if (!c || !q_host || !k_host || !v_host || !out_host) return fail(c, SWAM_ERR_INVALID_ARG, "swam_step_host: null argument");
   if (!c->io) return fail(c, SWAM_ERR_WORKSPACE, "swam_step_host: no staging area bound");
   cudaStream_t st = (cudaStream_t)stream;
-  const size_t fb = full_bytes(c->d), stride = align_up(fb, 256);
+  const size_t fb = full_bytes(c->d), kvb = kv_full_bytes(c->d), stride = align_up(fb, 256);
   // Three-stage pipeline over two input slots: this step's inputs travel on the copy-in stream while the previous
   // step still computes, the step runs on the caller's stream, and the result leaves on the copy-out stream while
   // the next inputs arrive (PCIe is full duplex).
@@ -409,8 +412,8 @@ int swam_step_host(swam_ctx* c, const void* q_host, const void* k_host, const vo
   void* dout = c->io + 6 * stride;
   cudaError_t e = cudaStreamWaitEvent(c->s_in, c->ev_done[slot], 0);   // the step two calls ago has read this slot
   if (e == cudaSuccess) e = cudaMemcpyAsync(dq, q_host, fb, cudaMemcpyHostToDevice, c->s_in);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(dk, k_host, fb, cudaMemcpyHostToDevice, c->s_in);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v_host, fb, cudaMemcpyHostToDevice, c->s_in);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dk, k_host, kvb, cudaMemcpyHostToDevice, c->s_in);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v_host, kvb, cudaMemcpyHostToDevice, c->s_in);
   if (e == cudaSuccess) e = cudaEventRecord(c->ev_h2d[slot], c->s_in);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_h2d[slot], 0);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_d2h, 0);     // the previous result has been copied out

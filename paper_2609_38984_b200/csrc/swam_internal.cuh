@@ -13,6 +13,7 @@ constexpr int kMaxGroup = 32;  // largest frame-aligned query group the tensor-c
 
 struct Dims {
   int B, n_obs, F, N_s, H, N_h, D, Kc, Ks, K, L, Lp, g, dtype;
+  int N_kv;   // key/value heads; query head h reads key/value head h / (N_h / N_kv)
   float scale, beta;
 };
 
@@ -67,6 +68,7 @@ struct AttnArgs {
   int lse_rows;      // number of rows written from lse_row0
   int B, n, N_h, D;  // n = sequence length of this call
   float scale;
+  int N_kv;          // heads of k and v (q and out have N_h); query head h reads head h / (N_h / N_kv)
 };
 cudaError_t attn_prepare(int D, int dtype);
 cudaError_t launch_attn_f32(const AttnArgs& a, cudaStream_t st, int* launches);

@@ -39,7 +39,7 @@ class SwamShape(ctypes.Structure):
         ("n_spatial", ctypes.c_int32), ("n_action", ctypes.c_int32), ("n_heads", ctypes.c_int32),
         ("head_dim", ctypes.c_int32), ("k_core", ctypes.c_int32), ("k_anchor", ctypes.c_int32),
         ("dtype", ctypes.c_int32), ("softmax_scale", ctypes.c_float), ("cv_beta", ctypes.c_float),
-        ("query_weights", ctypes.POINTER(ctypes.c_float)),
+        ("query_weights", ctypes.POINTER(ctypes.c_float)), ("n_kv_heads", ctypes.c_int32),
     ]
 
 
@@ -108,18 +108,19 @@ def torch_dtype(dtype: int) -> torch.dtype:
 
 class Swam:
     """One context = one shape.  Methods mirror the C entry points and take CUDA tensors laid out
-    [B, L, N_h, D] (or [B, L', N_h, D] for packed tensors)."""
+    [B, L, N_h, D] (or [B, L', N_h, D] for packed tensors); K and V have n_kv_heads heads instead of N_h."""
 
     def __init__(self, batch, n_obs, n_frames, n_spatial, n_action, n_heads, head_dim, k_core, k_anchor,
                  dtype=BF16, softmax_scale: float = 0.0, cv_beta: float = 1.0, query_weights=None,
-                 device: Optional[torch.device] = None, bind: bool = True):
+                 device: Optional[torch.device] = None, bind: bool = True, n_kv_heads: int = 0):
         self.lib = load_library()
         self._weights = None
         if query_weights is not None:
             self._weights = (ctypes.c_float * len(query_weights))(*[float(x) for x in query_weights])
         self.shape = SwamShape(batch, n_obs, n_frames, n_spatial, n_action, n_heads, head_dim, k_core, k_anchor,
                                dtype, softmax_scale, cv_beta,
-                               ctypes.cast(self._weights, ctypes.POINTER(ctypes.c_float)) if self._weights else None)
+                               ctypes.cast(self._weights, ctypes.POINTER(ctypes.c_float)) if self._weights else None,
+                               n_kv_heads)
         self.ctx = ctypes.c_void_p()
         if device is None:
             if not torch.cuda.is_available():
@@ -132,6 +133,7 @@ class Swam:
             raise SwamError(rc, "swam_create rejected the shape")
         self.B, self.F, self.N_s, self.H = batch, n_frames, n_spatial, n_action
         self.n_obs, self.N_h, self.D = n_obs, n_heads, head_dim
+        self.N_kv = n_kv_heads if n_kv_heads > 0 else n_heads
         self.K = k_core + k_anchor
         self.L = n_obs + n_frames * n_spatial + n_action
         self.Lp = n_obs + n_frames * self.K + n_action
@@ -145,7 +147,7 @@ class Swam:
     def from_workload(cls, wl: W.Workload, **kw) -> "Swam":
         kc, ks = wl.budgets
         return cls(wl.batch, wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, wl.n_heads, wl.head_dim, kc, ks,
-                   dtype=wl.dtype, **kw)
+                   dtype=wl.dtype, n_kv_heads=wl.kv_heads, **kw)
 
     def __del__(self):
         try:
@@ -185,8 +187,9 @@ class Swam:
     def empty_full(self) -> torch.Tensor:
         return torch.empty((self.B, self.L, self.N_h, self.D), dtype=torch_dtype(self.dtype), device=self.device)
 
-    def empty_packed(self) -> torch.Tensor:
-        return torch.empty((self.B, self.Lp, self.N_h, self.D), dtype=torch_dtype(self.dtype), device=self.device)
+    def empty_packed(self, kv: bool = False) -> torch.Tensor:
+        return torch.empty((self.B, self.Lp, self.N_kv if kv else self.N_h, self.D), dtype=torch_dtype(self.dtype),
+                           device=self.device)
 
     # -- the calls ---------------------------------------------------------
     def score(self, q, k, lse_action=None, quality: bool = False):
@@ -227,7 +230,7 @@ class Swam:
         return sel, pack, inv
 
     def pack(self, q, k, v, pack_map):
-        outs = [self.empty_packed() if x is not None else None for x in (q, k, v)]
+        outs = [self.empty_packed(kv=i > 0) if x is not None else None for i, x in enumerate((q, k, v))]
         self._chk(self.lib.swam_pack(self.ctx, _ptr(q), _ptr(k), _ptr(v), _ptr(pack_map), _ptr(outs[0]),
                                      _ptr(outs[1]), _ptr(outs[2]), _stream()))
         return outs

@@ -62,6 +62,11 @@ class Workload:
     blob_sigma: float = 3.0  # hotspot width in patches
     k_core: Optional[int] = None
     k_anchor: Optional[int] = None
+    n_kv_heads: Optional[int] = None   # key/value heads (grouped-query attention); None = n_heads
+
+    @property
+    def kv_heads(self) -> int:
+        return self.n_heads if self.n_kv_heads is None else self.n_kv_heads
 
     @property
     def n_spatial(self) -> int:
@@ -260,7 +265,7 @@ class Generator:
 
     # -- stepping ---------------------------------------------------------
     def next_step(self) -> Dict[str, np.ndarray]:
-        """Advance one denoising step; returns float32 arrays q, k, v of shape [B, L, N_h, D] whose values
+        """Advance one denoising step; returns float32 arrays q [B, L, N_h, D] and k, v [B, L, N_kv, D] whose values
         are already rounded to the workload's storage type (bf16 workloads: bf16-representable)."""
         wl = self.wl
         self._t += 1
@@ -294,10 +299,15 @@ class Generator:
                 fut = x[:, wl.n_obs:wl.n_obs + n_fut].reshape(
                     wl.batch, wl.n_frames, wl.n_spatial, wl.n_heads, wl.head_dim)
                 fut += np.float32(amp) * bump[:, :, :, None, None] * self._u[None, :, None, :, :]
+            grp = wl.n_heads // wl.kv_heads
             if bump is not None and name == "q":
                 act = x[:, wl.n_obs + n_fut:].reshape(
                     wl.batch, wl.n_frames, wl.group, wl.n_heads, wl.head_dim)
-                act += np.float32(amp) * self._u[None, :, None, :, :]
+                # every query head points along the direction of the key head it reads
+                u_q = self._u if grp == 1 else np.repeat(self._u[:, ::grp], grp, axis=1)
+                act += np.float32(amp) * u_q[None, :, None, :, :]
+            if grp > 1 and name in ("k", "v"):
+                x = np.ascontiguousarray(x[:, :, ::grp])      # grouped-query attention: one K/V head per group
             if wl.dtype == BF16:
                 x = bf16_bits_to_f32(f32_to_bf16_bits(x)).reshape(x.shape)
             out[name] = x

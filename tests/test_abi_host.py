@@ -38,12 +38,12 @@ def test_header_symbols_are_exported(lib):
 def _create(lib, **kw):
     from paper_2609_38984_b200 import swam
     base = dict(batch=1, n_obs=16, n_frames=2, n_spatial=64, n_action=8, n_heads=2, head_dim=32, k_core=14,
-                k_anchor=18, dtype=0, softmax_scale=0.0, cv_beta=1.0)
+                k_anchor=18, dtype=0, softmax_scale=0.0, cv_beta=1.0, n_kv_heads=0)
     base.update(kw)
     weights = base.pop("weights", None)
     arr = (ctypes.c_float * len(weights))(*weights) if weights else None
-    sh = swam.SwamShape(*[base[f] for f, _ in swam.SwamShape._fields_[:-1]],
-                        ctypes.cast(arr, ctypes.POINTER(ctypes.c_float)) if arr else None)
+    base["query_weights"] = ctypes.cast(arr, ctypes.POINTER(ctypes.c_float)) if arr else None
+    sh = swam.SwamShape(*[base[f] for f, _ in swam.SwamShape._fields_])
     ctx = ctypes.c_void_p()
     rc = lib.swam_create(ctypes.byref(sh), ctypes.byref(ctx))
     if rc == 0:
@@ -61,6 +61,9 @@ def test_shape_validation_happens_on_the_host(lib):
     assert _create(lib, batch=0) == swam.ERR_INVALID_ARG
     assert _create(lib, n_action=12, weights=[0.5] * 6) == swam.ERR_INVALID_ARG   # weights must sum to one
     assert _create(lib, n_action=128) == swam.ERR_UNSUPPORTED             # group of 64 exceeds the scorer's limit
+    assert _create(lib, n_heads=6, n_kv_heads=4) == swam.ERR_INVALID_ARG  # key/value heads must divide the heads
+    assert _create(lib, n_heads=6, n_kv_heads=-1) == swam.ERR_INVALID_ARG
+    assert _create(lib, n_heads=6, n_kv_heads=2) in (0, swam.ERR_CUDA)   # a valid shape; no device on a CPU-only host
     assert lib.swam_create(None, None) == swam.ERR_INVALID_ARG
 
 

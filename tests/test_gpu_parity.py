@@ -492,6 +492,71 @@ def test_corrupt_installed_selection_is_reported_not_followed():
     ctx.check()
 
 
+# ------------------------------------------------------------------ grouped-query attention (fewer key/value heads)
+GQA_CASES = [
+    ("tiny", dict(n_heads=4, n_kv_heads=2)),                                                           # fp32 kernels
+    ("single_view", dict(n_obs=70, grid_h=10, grid_w=9, n_heads=6, n_kv_heads=2)),                        # D = 64, tcgen05
+    ("larger_imagination", dict(n_obs=40, grid_h=7, grid_w=9, n_heads=4, n_kv_heads=1, batch=2)),         # D = 128, one K/V head
+    ("single_view", dict(n_obs=9, grid_h=6, grid_w=6, n_heads=4, n_kv_heads=2, head_dim=32)),             # D = 32, mma.sync
+]
+
+
+@pytest.mark.parametrize("name,kw", GQA_CASES, ids=["f32", "d64", "d128_mqa", "d32"])
+def test_grouped_query_stages_match_oracle(name, kw):
+    """Score (both normaliser sources), pack and attention with K and V holding fewer heads than Q."""
+    swam = _swam()
+    wl = W.WORKLOADS[name].with_(**kw)
+    x = W.generate_steps(wl, 1)[0]
+    assert x["k"].shape[2] == wl.kv_heads and x["q"].shape[2] == wl.n_heads
+    ctx = swam.Swam.from_workload(wl)
+    q, k, v = (dev(x[n], wl) for n in "qkv")
+    out, lse = ctx.sparse_attn(q, k, v, want_lse=True)
+    want, wlse = ora.attention(x["q"], x["k"], x["v"])
+    check_float(f64(out), want, wl.dtype)
+    assert np.abs(lse.cpu().numpy() - wlse).max() <= (1e-4 if wl.dtype == W.F32 else 2e-3)
+    lse_act = np.ascontiguousarray(wlse[:, :, wl.seq_len - wl.n_action:]).astype(np.float32)
+    s64 = ora.score(x["q"], x["k"], wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, lse=lse_act.astype(np.float64))
+    for given in (torch.from_numpy(lse_act).cuda(), None):
+        got = ctx.score(q, k, given).cpu().numpy()
+        rel = np.abs(got - s64) / np.maximum(s64, 1e-30)
+        assert rel.max() <= (2e-5 if given is not None else 5e-5), rel.max()
+    sel, pm, im = ctx.select(ctx.score(q, k))
+    qp, kp, vp = ctx.pack(q, k, v, pm)
+    assert kp.shape[2] == wl.kv_heads and qp.shape[2] == wl.n_heads
+    pm_np = pm.cpu().numpy()
+    for src, gotp in ((x["q"], qp), (x["k"], kp), (x["v"], vp)):
+        assert np.array_equal(gotp.float().cpu().numpy(), ora.pack(src, pm_np))
+    outp = ctx.sparse_attn(qp, kp, vp)
+    wantp, _ = ora.attention(ora.pack(x["q"], pm_np), ora.pack(x["k"], pm_np), ora.pack(x["v"], pm_np))
+    check_float(f64(outp), wantp, wl.dtype)
+    ctx.check()
+
+
+@pytest.mark.parametrize("name,kw", GQA_CASES[1:3], ids=["d64", "d128_mqa"])
+def test_grouped_query_schedule_matches_oracle(name, kw):
+    swam = _swam()
+    wl = W.WORKLOADS[name].with_(steps=3, **kw)
+    steps = W.generate_steps(wl)
+    ctx = swam.Swam.from_workload(wl)
+    compare_schedule(wl, steps, wl.refresh, run_schedule(ctx, wl, steps, wl.refresh))
+    # light refresh and the host-buffer path see the narrower K and V as well
+    out = ctx.empty_full().zero_()
+    x0, x1 = steps[0], steps[1]
+    ctx.step(dev(x0["q"], wl), dev(x0["k"], wl), dev(x0["v"], wl), swam.REFRESH_FULL, out)
+    ctx.step(dev(x1["q"], wl), dev(x1["k"], wl), dev(x1["v"], wl), swam.REFRESH_LIGHT, out)
+    ctx.check()
+    tdt = swam.torch_dtype(wl.dtype)
+    pinned = [{n: torch.from_numpy(x[n]).to(tdt).pin_memory() for n in "qkv"} for x in (x0, x1)]
+    out_h = torch.empty(out.shape, dtype=tdt).pin_memory()
+    host_ctx = swam.Swam.from_workload(wl)
+    host_ctx.step_host(pinned[0]["q"], pinned[0]["k"], pinned[0]["v"], swam.REFRESH_FULL, out_h)
+    host_ctx.step_host(pinned[1]["q"], pinned[1]["k"], pinned[1]["v"], swam.REFRESH_LIGHT, out_h)
+    host_ctx.host_join()
+    torch.cuda.synchronize()
+    host_ctx.check()
+    assert torch.equal(out_h.cuda(), out)
+
+
 def test_reuse_before_refresh_is_a_state_error():
     swam = _swam()
     wl = W.WORKLOADS["tiny"]
