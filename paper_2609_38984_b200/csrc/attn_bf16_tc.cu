@@ -431,6 +431,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       bool ok = true;
+      const int h_kv = h / p.kv_group;
       if (MODE != kGather) {
         mbar_expect_tx(bar_q, 2 * C::kTileBytes);
         for (int s = 0; s < 2; ++s)
@@ -444,12 +445,12 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (!ok) break;
         mbar_expect_tx(bar_k_full(st), C::kTileBytes);
         for (int db = 0; db < C::DB; ++db)
-          tma_load_4d(sK + st * C::kTileBytes + db * C::kSubTile, &map_k, bar_k_full(st), db * 64, (kv_begin + j) * kTile, h / p.kv_group, b);
+          tma_load_4d(sK + st * C::kTileBytes + db * C::kSubTile, &map_k, bar_k_full(st), db * 64, (kv_begin + j) * kTile, h_kv, b);
         ok = mbar_wait(bar_v_empty(st), par, abort_flag);
         if (!ok) break;
         mbar_expect_tx(bar_v_full(st), C::kTileBytes);
         for (int db = 0; db < C::DB; ++db)
-          tma_load_4d(sV + st * C::kTileBytes + db * C::kSubTile, &map_v, bar_v_full(st), db * 64, (kv_begin + j) * kTile, h / p.kv_group, b);
+          tma_load_4d(sV + st * C::kTileBytes + db * C::kSubTile, &map_v, bar_v_full(st), db * 64, (kv_begin + j) * kTile, h_kv, b);
       }
     }
    } else if (warp == 8) {

@@ -108,10 +108,11 @@ __global__ void __launch_bounds__(32 * MT * kHeadGroups, 16 / (MT * kHeadGroups)
   uint4 a0[2][KB], a1[2][KB];
   const uint4 zero = make_uint4(0, 0, 0, 0);
   auto load = [&](int h, int buf) {
+    const int hk = (kv_group == 1) ? h : h / kv_group;   // the division only runs for grouped-query shapes
 #pragma unroll
     for (int kb = 0; kb < KB; ++kb) {
-      a0[buf][kb] = v0 ? ldg_stream(k0 + (int64_t)(h / kv_group) * D + kb * 32) : zero;
-      a1[buf][kb] = v1 ? ldg_stream(k1 + (int64_t)(h / kv_group) * D + kb * 32) : zero;
+      a0[buf][kb] = v0 ? ldg_stream(k0 + hk * D + kb * 32) : zero;
+      a1[buf][kb] = v1 ? ldg_stream(k1 + hk * D + kb * 32) : zero;
     }
   };
   auto compute = [&](int h, int buf) {
