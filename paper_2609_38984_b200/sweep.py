@@ -4,7 +4,8 @@ frame (256 / 184 / 112 of 360; Sec. 5.4) and refresh schedule (first step only, 
 
 For each (keep, R) the workload's 10 denoising steps run through swam_step on one GPU; every stage is also timed
 on its own through the individual C-ABI calls.  Reported per configuration: the latency split over score, select,
-pack, attention (dense and packed) and scatter, the step latencies, packed tokens/s, the overlap of consecutive
+pack, attention (dense and packed) and scatter, the step latencies (eager, one launch sequence per step) and the device
+time of the whole schedule replayed from a CUDA graph, packed tokens/s, the overlap of consecutive
 steps' selections (IoU of retained sets and the Eq. 13 overlap of the normalised score maps, from a diagnostic
 score + select at every step), and how far the sparse output is from the dense one (relative L2; a reported
 number, not a pass/fail: the paper gives no figure for it).
@@ -63,6 +64,17 @@ def run_config(wl: W.Workload, refresh: int, n_steps: int, dev_steps, dense_outs
     diag = swam.Swam.from_workload(wl)          # diagnostic scoring/selection at every step
     out = ctx.empty_full().zero_()
     sched = W.refresh_schedule(n_steps, refresh)
+    # untimed first use (module load, lazily created descriptors), then the whole schedule replayed from a CUDA graph:
+    # the device time of the action chunk without host launch overhead, which dominates eager timing of small shapes
+    ctx.step(dev_steps[0]["q"], dev_steps[0]["k"], dev_steps[0]["v"], swam.REFRESH_FULL, out)
+    ctx.step(dev_steps[0]["q"], dev_steps[0]["k"], dev_steps[0]["v"], swam.REUSE, out)
+    ctx.check()
+    graph_us = None
+    if variant != "random":                      # the random variant installs its keys from the host between steps
+        def whole_schedule():
+            for t, x in enumerate(dev_steps):
+                ctx.step(x["q"], x["k"], x["v"], swam.REFRESH_FULL if sched[t] else swam.REUSE, out)
+        graph_us = _graph_us(whole_schedule, launches=1, reps=5)
 
     step_us, rel_l2, ious, overlaps = [], [], [], []
     prev_sel, prev_scores = None, None
@@ -114,8 +126,11 @@ def run_config(wl: W.Workload, refresh: int, n_steps: int, dev_steps, dense_outs
         "shape": wl.name, "variant": variant, "keep": round(keep, 4), "refresh": refresh, "k_core": wl.budgets[0], "k_anchor": wl.budgets[1], "packed_len": wl.packed_len,
         "steps": n_steps, "full_steps": len(full), "stage_us": {k: round(v, 2) for k, v in split.items()},
         "full_step_us": round(float(np.median(full)), 1), "sparse_step_us": round(float(np.median(sparse)), 1) if sparse else None,
-        "schedule_us": round(total_us, 1), "tokens_per_s": tokens / (total_us * 1e-6),
-        "iou_consecutive_steps": round(float(np.mean(ious)), 4), "overlap_eq13_consecutive_steps": round(float(np.mean(overlaps)), 4),
+        "schedule_us": round(total_us, 1),
+        "schedule_graph_us": None if graph_us is None else round(graph_us, 1),
+        "tokens_per_s": tokens / ((graph_us if graph_us is not None else total_us) * 1e-6),
+        "iou_consecutive_steps": None if variant == "random" else round(float(np.mean(ious)), 4),
+        "overlap_eq13_consecutive_steps": round(float(np.mean(overlaps)), 4),
         "rel_l2_vs_dense_per_step": [round(v, 4) for v in rel_l2],
     }
 
