@@ -248,6 +248,7 @@ struct TcParams {
   int n, N_h;
   int kv_group;        // query heads per key/value head
   int pairs;           // query tile pairs per (sample, head)
+  int total_work;      // n_whole + (items of the last, partly filled wave) * splits: what the CTAs share out
   int n_whole;         // work items that run over all keys and write the output themselves
   int splits;          // pieces per split item (0 when nothing is split)
   int tiles_per_split; // key tiles per piece
@@ -308,27 +309,41 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const uint32_t bar_o_final = bars + 8 * (7 + 4 * ST);
   // P V of a query tile's item has completed: that tile's output accumulator is up to date
   auto bar_pv_tile = [&](int s) { return bars + 8 * (8 + 4 * ST + s); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + C::kSmemData + 8 * (10 + 4 * ST));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::kSmemData + 8 * (10 + 4 * ST) + 8);
+  // a CTA works through several items: the output accumulators have been read (the next item's first P V may
+  // overwrite them), and the output staging in the query tiles has been read by the copy engine (the next item's
+  // queries may be loaded)
+  const uint32_t bar_o_free = bars + 8 * (10 + 4 * ST);
+  const uint32_t bar_q_free = bars + 8 * (11 + 4 * ST);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + C::kSmemData + 8 * (12 + 4 * ST));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::kSmemData + 8 * (12 + 4 * ST) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // work item = (sample, head, query tile pair), pair fastest.  Items below n_whole walk over all keys; the few items
+  // Work item = (sample, head, query tile pair), pair fastest.  Items below n_whole walk over all keys; the few items
   // of the last, partly filled wave are cut into `splits` pieces over the keys so that they spread over idle SMs,
-  // each piece leaving an unnormalised partial result for the combine kernel.
-  int item = blockIdx.x, kv_begin = 0;
+  // each piece leaving an unnormalised partial result for the combine kernel.  The grid has one CTA per SM (or per
+  // work item if there are fewer); CTA c takes work c, c + gridDim.x, ...  Every role walks through the same
+  // sequence on its own, and all barrier phases simply keep counting across items (running tile and item counters),
+  // so that the next item's key/value tiles stream in while this item's epilogue runs and nothing is set up twice.
+  struct Work { int h, b, row0, kv_begin, n_tiles, slot; };
   const int all_tiles = (p.n + kTile - 1) / kTile;
-  int kv_end = all_tiles;
-  int slot = -1;
-  if (item >= p.n_whole) {
-    slot = item - p.n_whole;
-    item = p.n_whole + slot / p.splits;
-    kv_begin = (slot % p.splits) * p.tiles_per_split;
-    kv_end = min(all_tiles, kv_begin + p.tiles_per_split);
-  }
-  const int pair = item % p.pairs;
-  const int h = (item / p.pairs) % p.N_h, b = item / (p.pairs * p.N_h);
-  const int row0 = pair * 2 * kTile;
-  const int n_tiles = kv_end - kv_begin;  // >= 1 by construction
+  auto decode = [&](int w) {
+    Work k;
+    int item = w, kv_end = all_tiles;
+    k.kv_begin = 0;
+    k.slot = -1;
+    if (item >= p.n_whole) {
+      k.slot = item - p.n_whole;
+      item = p.n_whole + k.slot / p.splits;
+      k.kv_begin = (k.slot % p.splits) * p.tiles_per_split;
+      kv_end = min(all_tiles, k.kv_begin + p.tiles_per_split);
+    }
+    const int pair = item % p.pairs;
+    k.h = (item / p.pairs) % p.N_h;
+    k.b = item / (p.pairs * p.N_h);
+    k.row0 = pair * 2 * kTile;
+    k.n_tiles = kv_end - k.kv_begin;  // >= 1 by construction
+    return k;
+  };
 
   if (threadIdx.x == 0) CTA_T(0);
   if (threadIdx.x == 0) {
@@ -347,6 +362,8 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     mbar_init(bar_pv_tile(0), 1);
     mbar_init(bar_pv_tile(1), 1);
     mbar_init(bar_o_final, 1);
+    mbar_init(bar_o_free, 2 * kTile);
+    mbar_init(bar_q_free, (MODE == kDirect) ? 2 : 2 * kTile);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -383,10 +400,10 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     constexpr int RPI = 32 / CPR;              // rows per warp instruction
     const int pw = warp - 10;
     const int cc = lane % CPR, sub = lane / CPR;
-    const int32_t* pm = p.pack_map + (int64_t)b * p.n;
     const int64_t row_stride = (int64_t)p.N_h * D;
-    const int64_t base_off = ((int64_t)b * p.n_full * p.N_h + h) * D + cc * 8;
     const uint32_t dst_cc = (uint32_t)((cc >> 3) * C::kSubTile);
+    const int32_t* pm = nullptr;     // map of the current work item's sample
+    int64_t base_off = 0;            // first element of (sample, head), this lane's chunk
     // map entries of row block rb of the tile starting at packed row prow0: -1 = fill with zeros
     auto block_rows = [&](int prow0, int rb) {
       const int pr = prow0 + rb * 32 + lane;
@@ -418,39 +435,64 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     src_lane + (orow < 0 ? 0 : orow) * row_stride, orow < 0 ? 0u : 16u);
       }
     };
-    // warp pw copies row blocks pw and pw + 2 of both query tiles
-    for (int s = 0; s < 2; ++s) {
-      const int prow0 = row0 + s * kTile;
-      const int r0 = block_rows(prow0, pw), r1 = block_rows(prow0, pw + 2);
-      gather_block(sQ + s * C::kTileBytes, p.q_full, pw, r0);
-      gather_block(sQ + s * C::kTileBytes, p.q_full, pw + 2, r1);
+    int iter = 0;
+    for (int work = blockIdx.x; work < p.total_work; work += gridDim.x, ++iter) {
+      const Work wk = decode(work);
+      pm = p.pack_map + (int64_t)wk.b * p.n;
+      base_off = ((int64_t)wk.b * p.n_full * p.N_h + wk.h) * D + cc * 8;
+      if (iter > 0) {
+        // the previous item's output has left the query tiles
+        int go = 1;
+        if (lane == 0) go = mbar_wait(bar_q_free, (iter - 1) & 1, abort_flag) ? 1 : 0;
+        if (__shfl_sync(0xffffffffu, go, 0) == 0) break;
+      }
+      // warp pw copies row blocks pw and pw + 2 of both query tiles
+      for (int s = 0; s < 2; ++s) {
+        const int prow0 = wk.row0 + s * kTile;
+        const int r0 = block_rows(prow0, pw), r1 = block_rows(prow0, pw + 2);
+        gather_block(sQ + s * C::kTileBytes, p.q_full, pw, r0);
+        gather_block(sQ + s * C::kTileBytes, p.q_full, pw + 2, r1);
+      }
+      cp_async_arrive(bar_q);
     }
-    cp_async_arrive(bar_q);
     cp_async_wait_all();   // nothing of this thread is still on its way into shared memory at exit
    } else if (warp == 9) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       bool ok = true;
-      const int h_kv = h / p.kv_group;
-      if (MODE != kGather) {
-        mbar_expect_tx(bar_q, 2 * C::kTileBytes);
-        for (int s = 0; s < 2; ++s)
+      int kt = 0;      // key/value tiles loaded so far by this CTA: ring slot kt % ST, pass kt / ST
+      int iter = 0;
+      for (int work = blockIdx.x; work < p.total_work && ok; work += gridDim.x, ++iter) {
+        const Work wk = decode(work);
+        const int h_kv = wk.h / p.kv_group;
+        // The first item's queries go first.  A later item's queries have to wait until the previous item's output has
+        // left the query tiles, so that item's first key/value tiles (as many as the ring holds) are requested before.
+        auto load_q = [&]() {
+          if (MODE == kGather) return true;
+          if (iter > 0 && !mbar_wait(bar_q_free, (iter - 1) & 1, abort_flag)) return false;
+          mbar_expect_tx(bar_q, 2 * C::kTileBytes);
+          for (int s = 0; s < 2; ++s)
+            for (int db = 0; db < C::DB; ++db)
+              tma_load_4d(sQ + s * C::kTileBytes + db * C::kSubTile, &map_q, bar_q, db * 64, wk.row0 + s * kTile, wk.h, wk.b);
+          return true;
+        };
+        const int q_after = (iter == 0) ? -1 : min(ST, wk.n_tiles) - 1;   // tile after which the queries are requested
+        if (q_after < 0) ok = load_q();
+        for (int j = 0; j < wk.n_tiles && ok; ++j, ++kt) {
+          const int st = kt % ST;
+          const uint32_t par = ((kt / ST) & 1) ^ 1;  // first pass over the ring: slots start empty
+          ok = mbar_wait(bar_k_empty(st), par, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(bar_k_full(st), C::kTileBytes);
           for (int db = 0; db < C::DB; ++db)
-            tma_load_4d(sQ + s * C::kTileBytes + db * C::kSubTile, &map_q, bar_q, db * 64, row0 + s * kTile, h, b);
-      }
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int st = j % ST;
-        const uint32_t par = ((j / ST) & 1) ^ 1;  // first pass over the ring: slots start empty
-        ok = mbar_wait(bar_k_empty(st), par, abort_flag);
-        if (!ok) break;
-        mbar_expect_tx(bar_k_full(st), C::kTileBytes);
-        for (int db = 0; db < C::DB; ++db)
-          tma_load_4d(sK + st * C::kTileBytes + db * C::kSubTile, &map_k, bar_k_full(st), db * 64, (kv_begin + j) * kTile, h_kv, b);
-        ok = mbar_wait(bar_v_empty(st), par, abort_flag);
-        if (!ok) break;
-        mbar_expect_tx(bar_v_full(st), C::kTileBytes);
-        for (int db = 0; db < C::DB; ++db)
-          tma_load_4d(sV + st * C::kTileBytes + db * C::kSubTile, &map_v, bar_v_full(st), db * 64, (kv_begin + j) * kTile, h_kv, b);
+            tma_load_4d(sK + st * C::kTileBytes + db * C::kSubTile, &map_k, bar_k_full(st), db * 64, (wk.kv_begin + j) * kTile, h_kv, wk.b);
+          ok = mbar_wait(bar_v_empty(st), par, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(bar_v_full(st), C::kTileBytes);
+          for (int db = 0; db < C::DB; ++db)
+            tma_load_4d(sV + st * C::kTileBytes + db * C::kSubTile, &map_v, bar_v_full(st), db * 64, (wk.kv_begin + j) * kTile, h_kv, wk.b);
+          if (j == q_after) ok = load_q();
+        }
       }
     }
    } else if (warp == 8) {
@@ -462,10 +504,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       auto wait_all = [&](uint32_t bar, uint32_t parity) {
         return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag) ? 1 : 0) != 0;
       };
-      // gathered query tiles were written through the generic proxy and are read by the tensor core through the
-      // async proxy: the reader fences after the wait
-      bool ok = wait_all(bar_q, 0);
-      if (MODE == kGather) fence_proxy_async();
+      bool ok = true;
       const uint32_t q_lo0 = desc_lo(sQ, 16), k_lo0 = desc_lo(sK, 16), v_lo0 = desc_lo(sV, C::kSubTile);
       auto issue_qk = [&](int s, int buf, int st) {
         // S = Q_s K^T : K dimension = D, 16 elements (32 bytes) per instruction inside the 128-byte swizzle row
@@ -491,41 +530,60 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       // Q K^T of item i + NB into the score buffer that P V has just consumed (the tensor pipe executes one thread's
       // instructions in issue order).  With three buffers the scores of a query tile's next key tile are ready before
       // its softmax warpgroup has finished the current one.
-      const int n_items = 2 * n_tiles;
-      int k_waited = 0, v_waited = 0;
-      auto qk_item = [&](int it) -> bool {
-        const int j = it >> 1, sq = it & 1, st = j % ST;
-        if (j >= k_waited) {
-          if (!wait_all(bar_k_full(st), (j / ST) & 1)) return false;
-          k_waited = j + 1;
-          tc_fence_after();
-        }
-        issue_qk(sq, it % NB, st);
-        tc_commit(bar_s_full(it % NB), el);
-        if (sq == 1) tc_commit(bar_k_empty(st), el);   // both query tiles have used this key tile
-        return true;
-      };
-      for (int it = 0; it < NB && it < n_items && ok; ++it) ok = qk_item(it);
-      for (int it = 0; it < n_items && ok; ++it) {
-        const int j = it >> 1, sq = it & 1, st = j % ST, buf = it % NB;
-        if (j >= v_waited) {
-          ok = wait_all(bar_v_full(st), (j / ST) & 1);
-          if (!ok) break;
-          v_waited = j + 1;
-        }
-        TRACE(2, it * 4 + 0);
-        ok = wait_all(bar_p_full(buf), (it / NB) & 1);
+      int kt0 = 0;     // key tiles of the items this CTA has finished (ring position of the current item's tile 0)
+      int it0 = 0;     // (key tile, query tile) items finished: score buffer (it0 + i) % NB for the current item's i
+      int iter = 0;
+      for (int work = blockIdx.x; work < p.total_work && ok; work += gridDim.x, ++iter) {
+        const Work wk = decode(work);
+        // gathered query tiles were written through the generic proxy and are read by the tensor core through the
+        // async proxy: the reader fences after the wait
+        ok = wait_all(bar_q, iter & 1);
         if (!ok) break;
-        TRACE(2, it * 4 + 1);
-        tc_fence_after();
-        issue_pv(sq, buf, st, j > 0);
-        TRACE(2, it * 4 + 2);
-        tc_commit(bar_pv_tile(sq), el);
-        if (sq == 1) tc_commit(bar_v_empty(st), el);
-        if (it + NB < n_items) ok = qk_item(it + NB);
-        TRACE(2, it * 4 + 3);
+        if (MODE == kGather) fence_proxy_async();
+        const int n_items = 2 * wk.n_tiles;
+        int k_waited = 0, v_waited = 0;
+        auto qk_item = [&](int it) -> bool {
+          const int j = it >> 1, sq = it & 1, st = (kt0 + j) % ST, g = it0 + it;
+          if (j >= k_waited) {
+            if (!wait_all(bar_k_full(st), ((kt0 + j) / ST) & 1)) return false;
+            k_waited = j + 1;
+            tc_fence_after();
+          }
+          issue_qk(sq, g % NB, st);
+          tc_commit(bar_s_full(g % NB), el);
+          if (sq == 1) tc_commit(bar_k_empty(st), el);   // both query tiles have used this key tile
+          return true;
+        };
+        for (int it = 0; it < NB && it < n_items && ok; ++it) ok = qk_item(it);
+        for (int it = 0; it < n_items && ok; ++it) {
+          const int j = it >> 1, sq = it & 1, st = (kt0 + j) % ST, g = it0 + it, buf = g % NB;
+          if (j >= v_waited) {
+            ok = wait_all(bar_v_full(st), ((kt0 + j) / ST) & 1);
+            if (!ok) break;
+            v_waited = j + 1;
+          }
+          if (iter == 0) TRACE(2, it * 4 + 0);
+          ok = wait_all(bar_p_full(buf), (g / NB) & 1);
+          if (!ok) break;
+          if (it == 0 && iter > 0) {
+            // the first product of an item overwrites the output accumulators: the previous item's epilogue must
+            // have read them
+            ok = wait_all(bar_o_free, (iter - 1) & 1);
+            if (!ok) break;
+          }
+          if (iter == 0) TRACE(2, it * 4 + 1);
+          tc_fence_after();
+          issue_pv(sq, buf, st, j > 0);
+          if (iter == 0) TRACE(2, it * 4 + 2);
+          tc_commit(bar_pv_tile(sq), el);
+          if (sq == 1) tc_commit(bar_v_empty(st), el);
+          if (it + NB < n_items) ok = qk_item(it + NB);
+          if (iter == 0) TRACE(2, it * 4 + 3);
+        }
+        if (ok) tc_commit(bar_o_final, el);
+        kt0 += wk.n_tiles;
+        it0 += n_items;
       }
-      if (ok) tc_commit(bar_o_final, el);
     }
    }
   } else {
@@ -535,22 +593,26 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const int r = (warp & 3) * 32 + lane;    // row inside the tile == TMEM lane
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tO = tm_O(s) + lane_off;
-    float m_used = -INFINITY, l_run = 0.f;
     bool ok = true;
+    int kt0 = 0, it0 = 0, iter = 0;   // the same running counters as in the issuing warp
+    for (int work = blockIdx.x; work < p.total_work && ok; work += gridDim.x, ++iter) {
+    const Work wk = decode(work);
+    const int h = wk.h, b = wk.b, row0 = wk.row0, kv_begin = wk.kv_begin, n_tiles = wk.n_tiles, slot = wk.slot;
+    float m_used = -INFINITY, l_run = 0.f;
     for (int j = 0; j < n_tiles; ++j) {
-      const int item = 2 * j + s, buf = item % NB;
+      const int item = it0 + 2 * j + s, buf = item % NB;
       const uint32_t tS = tm_S(buf) + lane_off;
-      if (r == 0) TRACE(s, j * 8 + 0);
+      if (r == 0 && iter == 0) TRACE(s, j * 8 + 0);
       ok = mbar_wait(bar_s_full(buf), (item / NB) & 1, abort_flag);
       if (!ok) break;
-      if (r == 0) TRACE(s, j * 8 + 1);
-      if (r == 0 && s == 0 && j == 0) CTA_T(1);
+      if (r == 0 && iter == 0) TRACE(s, j * 8 + 1);
+      if (r == 0 && s == 0 && j == 0 && iter == 0) CTA_T(1);
       tc_fence_after();
       float sv[kTile];
 #pragma unroll
       for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<float(*)[32]>(&sv[c * 32]));
       tmem_ld_wait();
-      if (r == 0) TRACE(s, j * 8 + 2);
+      if (r == 0 && iter == 0) TRACE(s, j * 8 + 2);
       const int valid = p.n - (kv_begin + j) * kTile;  // keys of this tile inside the sequence
       if (valid < kTile) {
 #pragma unroll
@@ -618,7 +680,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         // the accumulator must hold every product issued against the old reference before it is rescaled (with three
         // score buffers the previous P V of this tile may still be waiting behind a Q K^T)
         if (j > 0) {
-          ok = mbar_wait(bar_pv_tile(s), (j - 1) & 1, abort_flag);
+          ok = mbar_wait(bar_pv_tile(s), (kt0 + j - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
         }
@@ -647,15 +709,15 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
       }
       l_run += sum;
-      if (r == 0) TRACE(s, j * 8 + 3);
+      if (r == 0 && iter == 0) TRACE(s, j * 8 + 3);
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(bar_p_full(buf));
-      if (r == 0) TRACE(s, j * 8 + 4);
+      if (r == 0 && iter == 0) TRACE(s, j * 8 + 4);
     }
     // epilogue
-    if (ok) ok = mbar_wait(bar_o_final, 0, abort_flag);
-    if (r == 0 && s == 0) CTA_T(2);
+    if (ok) ok = mbar_wait(bar_o_final, iter & 1, abort_flag);
+    if (r == 0 && s == 0 && iter == 0) CTA_T(2);
     if (slot >= 0) {
       // a piece of a split item: unnormalised O, reference max and sum go to scratch; the combine kernel finishes
       if (ok) {
@@ -672,6 +734,10 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
         dst[D] = m_used;
         dst[D + 1] = l_run;
+        tc_fence_before();
+        mbar_arrive(bar_o_free);          // the accumulator row has been read
+        // nothing was staged in the query tiles: they are free as far as this thread is concerned
+        if (MODE != kDirect || ((warp & 3) == 0 && lane == 0)) mbar_arrive(bar_q_free);
       }
     } else {
     // O / l -> bf16 -> swizzled staging in the (finished) Q tile -> TMA store; rows beyond n are clipped
@@ -700,6 +766,8 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       if (p.lse && row < p.n && row >= p.lse_row0 && row < p.lse_row0 + p.lse_rows)
         p.lse[((int64_t)b * p.N_h + h) * p.lse_rows + (row - p.lse_row0)] = (m_used + log2f(l_run)) * 0.6931471805599453f;
       fence_proxy_async();
+      tc_fence_before();
+      mbar_arrive(bar_o_free);            // the accumulator row has been read
     }
     if (MODE != kDirect) {
       // each thread sends the row it has just staged (it reads only its own writes, so its own proxy fence is all the
@@ -716,15 +784,22 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           atomicOr(p.status, ST_BAD_MAP);
         }
       }
+      if (ok) mbar_arrive(bar_q_free);    // this thread's staged row has been read (or was never sent)
     } else {
       asm volatile("bar.sync %0, 128;" ::"r"(1 + s) : "memory");  // the four warps of this query tile
-      if (ok && (warp & 3) == 0 && lane == 0 && row0 + s * kTile < p.n) {
-        for (int db = 0; db < C::DB; ++db)
-          tma_store_4d(&map_o, sQ + s * C::kTileBytes + db * C::kSubTile, db * 64, row0 + s * kTile, h, b);
-        tma_store_commit_wait();
+      if (ok && (warp & 3) == 0 && lane == 0) {
+        if (row0 + s * kTile < p.n) {
+          for (int db = 0; db < C::DB; ++db)
+            tma_store_4d(&map_o, sQ + s * C::kTileBytes + db * C::kSubTile, db * 64, row0 + s * kTile, h, b);
+          tma_store_commit_wait();
+        }
+        mbar_arrive(bar_q_free);          // this tile's staging has been read (or was never sent)
       }
     }
     }
+    kt0 += n_tiles;
+    it0 += 2 * n_tiles;
+    }   // work items of this CTA
   }
 
   tc_fence_before();
@@ -893,9 +968,9 @@ cudaError_t launch_tc_d(const AttnArgs& a, const int32_t* pack_map, int n_full, 
 #ifdef SWAM_TC_TRACE
       (long long*)partial_trace_buffer(),
 #endif
-      a.lse, status, partial, pack_map, n_full, (const __nv_bfloat16*)a.q, a.lse_row0, a.lse_rows, a.n, a.N_h, a.N_h / a.N_kv, pairs, n_whole, splits, per,
+      a.lse, status, partial, pack_map, n_full, (const __nv_bfloat16*)a.q, a.lse_row0, a.lse_rows, a.n, a.N_h, a.N_h / a.N_kv, pairs, n_whole + (splits ? rem * splits : 0), n_whole, splits, per,
       a.scale * kLog2e};
-  const int grid = n_whole + (splits ? rem * splits : 0);
+  const int grid = p.total_work < sms ? p.total_work : sms;   // one CTA per SM; each walks through its share of the work
   ++*launches;
   attn_bf16_tc_kernel<D, MODE><<<grid, kThreadsTc, TcCfg<D>::kSmemBytes, st>>>(mq, mk, mv, mo, p);
   e = cudaGetLastError();
