@@ -215,40 +215,8 @@ constexpr int kQualThreads = 1024;
 __global__ void __launch_bounds__(kQualThreads) quality_kernel(const float* scores, float* quality, int F, int N_s,
                                                                int parts) {
   extern __shared__ double2 part_sums[];  // [F * parts]
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, b = blockIdx.x;
-  const float* s = scores + (int64_t)b * F * N_s;
-  const int per = (N_s + parts - 1) / parts;
-  for (int u = warp; u < F * parts; u += kQualThreads / 32) {
-    const int f = u / parts, part = u % parts;
-    const int j1 = min(N_s, (part + 1) * per);
-    double a = 0.0, bq = 0.0;
-    for (int j = part * per + lane; j < j1; j += 32) {
-      const float v = s[f * N_s + j];
-      a += (double)v;
-      if (v > 0.f) bq += (double)(v * logf(v));
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      a += __shfl_xor_sync(0xffffffffu, a, o);
-      bq += __shfl_xor_sync(0xffffffffu, bq, o);
-    }
-    if (lane == 0) part_sums[u] = make_double2(a, bq);
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    double total = 0.0, ent = 0.0;
-    for (int f = 0; f < F; ++f) {
-      double a = 0.0, bq = 0.0;
-      for (int q = 0; q < parts; ++q) { a += part_sums[f * parts + q].x; bq += part_sums[f * parts + q].y; }
-      total += a;
-      if (a > 0.0) ent += log(a) - bq / a;
-    }
-    const double R = total / (double)F;
-    const double E = ent / ((double)F * log((double)N_s));
-    quality[b * 3 + 0] = (float)R;
-    quality[b * 3 + 1] = (float)E;
-    quality[b * 3 + 2] = (float)(R * (1.0 - E));
-  }
+  const int b = blockIdx.x;
+  quality_of_scores(scores + (int64_t)b * F * N_s, F, N_s, parts, part_sums, quality + b * 3, kQualThreads);
 }
 
 // ---- action-row normalisers over all L keys -----------------------------------------------------------
@@ -537,8 +505,7 @@ cudaError_t launch_score(const Dims& d, const Alpha& alpha, const void* q, const
 
 cudaError_t launch_quality(const Dims& d, const float* scores, float* quality, cudaStream_t st, int* launches) {
   ++*launches;
-  int parts = 32 / d.F;
-  if (parts < 1) parts = 1;
+  const int parts = quality_parts(d.F);
   quality_kernel<<<d.B, kQualThreads, (size_t)d.F * parts * sizeof(double2), st>>>(scores, quality, d.F, d.N_s, parts);
   return cudaGetLastError();
 }

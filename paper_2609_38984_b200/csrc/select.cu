@@ -191,6 +191,7 @@ struct SelectParams {
   int* status;
   int n_obs, F, N_s, H, Kc, Ks, L, Lp;
   double beta;
+  float* quality;           // [B, 3] (R, E, Q) of Eq. 9 for `scores`, or nullptr
 };
 
 // shared-memory layout (bytes), identical in every CTA of the cluster
@@ -332,6 +333,13 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
     if (im) im[p.n_obs + F * N + t] = p.n_obs + F * K + t;
   }
   if (bad && tid == 0) atomicOr(p.status, ST_BAD_COUNT);
+  // the layer-quality diagnostics of the scores this CTA already holds: the last CTA of the cluster computes them
+  // once its selection work is done (the anchor-key area is free by then and serves as scratch)
+  if (p.quality && rank == C - 1) {
+    __syncthreads();
+    quality_of_scores(S, F, N, quality_parts(F), reinterpret_cast<double2*>(smem_raw + lay.keyA), p.quality + b * 3,
+                      kSelThreads);
+  }
 }
 
 // Multi-layer aggregation (Eq. 3, Eq. 11): V = sum over the k_layer best layers of Q_l S_l / sum Q_l and V_all the
@@ -410,10 +418,14 @@ cudaError_t select_prepare(const Dims& d) {
   return cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
 
+// the anchor-key area (8 bytes per spatial position) must hold the F * parts partial sums (16 bytes each)
+bool select_can_fold_quality(const Dims& d) { return (size_t)d.N_s * 8 >= (size_t)d.F * quality_parts(d.F) * sizeof(double2); }
+
 cudaError_t launch_select(const Dims& d, const float* scores, const float* scores_all, int32_t* sel_idx,
-                          int32_t* pack_map, int32_t* inv_map, int* status, cudaStream_t st, int* launches) {
+                          int32_t* pack_map, int32_t* inv_map, int* status, cudaStream_t st, int* launches,
+                          float* quality) {
   SelectParams p{scores, scores_all ? scores_all : scores, sel_idx, pack_map, inv_map, status, d.n_obs, d.F, d.N_s, d.H,
-                 d.Kc, d.Ks, d.L, d.Lp, (double)d.beta};
+                 d.Kc, d.Ks, d.L, d.Lp, (double)d.beta, select_can_fold_quality(d) ? quality : nullptr};
   const int C = cluster_size(d);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(C, d.B, 1);

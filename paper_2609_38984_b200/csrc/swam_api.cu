@@ -365,8 +365,13 @@ int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t 
   }
   if (mode != SWAM_REUSE) {
     const float* lse_in = (mode == SWAM_REFRESH_FULL) ? lse : nullptr;
-    if (int r = swam_score(c, q, k, lse_in, scores, quality, stream)) return r;
-    if (int r = swam_select(c, scores, sel, pm, im, stream)) return r;
+    // the Eq. 9 diagnostics ride along with the selection kernel, which holds the scores in shared memory anyway
+    const bool fold = select_can_fold_quality(d);
+    if (int r = swam_score(c, q, k, lse_in, scores, fold ? nullptr : quality, stream)) return r;
+    cudaError_t e = launch_select(d, scores, nullptr, sel, pm, im, (int*)(c->ws + c->off_status), st, &c->launches_i,
+                                  quality);
+    count(c);
+    if (e != cudaSuccess) return fail_cuda(c, e, "select launch");
     c->has_selection = true;
   }
   if (mode != SWAM_REFRESH_FULL && c->sparse_path == SWAM_SPARSE_FUSED && d.dtype == SWAM_BF16 && d.D >= 64 &&

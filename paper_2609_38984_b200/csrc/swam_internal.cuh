@@ -21,6 +21,49 @@ struct Alpha {
   float w[kMaxGroup];
 };
 
+// Layer quality (Eq. 9) of one sample's scores S [F, N_s] (global or shared memory): R = sum S / F, E = mean normalised
+// spatial entropy, Q = R (1 - E), written to out3[0..2].  Called by every thread of a CTA of `n_threads` threads
+// (a multiple of 32); part_sums: shared memory, F * parts entries.  With a_f = sum_j s and b_f = sum_j s ln s the
+// entropy of frame f is ln a_f - b_f / a_f.  Warps take (frame, part) units; partial sums are combined in a fixed
+// order, so the result does not depend on which kernel calls it.
+__device__ __forceinline__ void quality_of_scores(const float* s, int F, int N_s, int parts, double2* part_sums,
+                                                  float* out3, int n_threads) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int per = (N_s + parts - 1) / parts;
+  for (int u = warp; u < F * parts; u += n_threads / 32) {
+    const int f = u / parts, part = u % parts;
+    const int j1 = min(N_s, (part + 1) * per);
+    double a = 0.0, bq = 0.0;
+    for (int j = part * per + lane; j < j1; j += 32) {
+      const float v = s[f * N_s + j];
+      a += (double)v;
+      if (v > 0.f) bq += (double)(v * logf(v));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      a += __shfl_xor_sync(0xffffffffu, a, o);
+      bq += __shfl_xor_sync(0xffffffffu, bq, o);
+    }
+    if (lane == 0) part_sums[u] = make_double2(a, bq);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double total = 0.0, ent = 0.0;
+    for (int f = 0; f < F; ++f) {
+      double a = 0.0, bq = 0.0;
+      for (int q = 0; q < parts; ++q) { a += part_sums[f * parts + q].x; bq += part_sums[f * parts + q].y; }
+      total += a;
+      if (a > 0.0) ent += log(a) - bq / a;
+    }
+    const double R = total / (double)F;
+    const double E = ent / ((double)F * log((double)N_s));
+    out3[0] = (float)R;
+    out3[1] = (float)E;
+    out3[2] = (float)(R * (1.0 - E));
+  }
+}
+__host__ __device__ inline int quality_parts(int F) { return F >= 32 ? 1 : 32 / F; }
+
 // ---- score.cu -------------------------------------------------------------
 // S[b,f,j] (Eq. 12) from the action rows of q, the future rows of k and lambda [B,N_h,H].
 cudaError_t launch_score(const Dims& d, const Alpha& alpha, const void* q, const void* k, const float* lse,
@@ -42,8 +85,12 @@ cudaError_t static_scratch(const Dims& d, float** lse, void** partial);
 size_t select_smem_bytes(const Dims& d);
 cudaError_t select_prepare(const Dims& d);  // opt in to the dynamic shared memory the kernel needs
 // scores: core map (pool, cores); scores_all: anchor map, nullptr => same as scores
+// quality: [B, 3] or nullptr; when given (and select_can_fold_quality(d)) the kernel also writes the Eq. 9 diagnostics
+// of `scores`, which saves the separate launch of launch_quality
+bool select_can_fold_quality(const Dims& d);
 cudaError_t launch_select(const Dims& d, const float* scores, const float* scores_all, int32_t* sel_idx,
-                          int32_t* pack_map, int32_t* inv_map, int* status, cudaStream_t st, int* launches);
+                          int32_t* pack_map, int32_t* inv_map, int* status, cudaStream_t st, int* launches,
+                          float* quality = nullptr);
 int max_layers();
 // V and V_all from per-layer scores [n_layers, B, F, N_s] and qualities [n_layers, B, 3]
 cudaError_t launch_aggregate(const Dims& d, const float* layer_scores, const float* layer_quality, int n_layers, int k_layer,

@@ -557,6 +557,26 @@ def test_grouped_query_schedule_matches_oracle(name, kw):
     assert torch.equal(out_h.cuda(), out)
 
 
+@pytest.mark.parametrize("wl", [W.WORKLOADS["tiny"], small(batch=2), small("multi_view", batch=2, n_obs=33, grid_h=5, grid_w=4, n_heads=2)],
+                         ids=["f32", "d64", "multiview"])
+def test_step_leaves_the_layer_quality_of_its_scores(wl):
+    """The (R, E, Q) diagnostics of Eq. 9 that a refresh step caches equal those of the stand-alone scoring call on the
+    same scores (the selection kernel computes them in passing) and match the oracle."""
+    swam = _swam()
+    x = W.generate_steps(wl, 1)[0]
+    ctx = swam.Swam.from_workload(wl)
+    out = ctx.empty_full().zero_()
+    q, k, v = (dev(x[n], wl) for n in "qkv")
+    for mode in (swam.REFRESH_FULL, swam.REFRESH_LIGHT):
+        ctx.step(q, k, v, mode, out)
+        ctx.check()
+        scores, lse, qual = (t.clone() for t in ctx.cached_scores())
+        _, qual_alone = ctx.score(q, k, lse if mode == swam.REFRESH_FULL else None, quality=True)
+        assert torch.equal(qual, qual_alone)
+        want = ora.quality(scores.cpu().numpy())
+        assert np.abs(qual.cpu().numpy() - want).max() <= 1e-5 * max(1.0, np.abs(want).max())
+
+
 def test_reuse_before_refresh_is_a_state_error():
     swam = _swam()
     wl = W.WORKLOADS["tiny"]
