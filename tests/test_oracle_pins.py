@@ -32,6 +32,25 @@ def test_attention_matches_library_fp64():
     assert np.abs(lse - torch.logsumexp(logits, -1).numpy()).max() < 1e-12
 
 
+def test_grouped_query_attention_matches_library_head_mapping():
+    """K and V with fewer heads: query head h reads head h // (N_h / N_kv), as the library's own grouped-query
+    attention does; a head order of "h % N_kv" (the plausible mistake) gives a different answer."""
+    rng = np.random.default_rng(11)
+    q = rng.standard_normal((2, 23, 6, 8)).astype(np.float32)
+    k = rng.standard_normal((2, 23, 2, 8)).astype(np.float32)
+    v = rng.standard_normal((2, 23, 2, 8)).astype(np.float32)
+    out, _ = ora.attention(q, k, v)
+    tq, tk, tv = [torch.from_numpy(x).double().permute(0, 2, 1, 3) for x in (q, k, v)]
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, enable_gqa=True).permute(0, 2, 1, 3).numpy()
+    assert np.abs(out - ref).max() < 1e-12
+    wrong = torch.nn.functional.scaled_dot_product_attention(tq, tk.repeat(1, 3, 1, 1), tv.repeat(1, 3, 1, 1))
+    assert np.abs(out - wrong.permute(0, 2, 1, 3).numpy()).max() > 1e-3
+    # the score sees the same mapping: expanding the key heads by hand changes nothing
+    s1 = ora.score(q, k, 3, 2, 6, 8)
+    s2 = ora.score(q, np.repeat(k, 3, axis=2), 3, 2, 6, 8)
+    assert np.array_equal(s1, s2)
+
+
 def test_attention_scale_and_transpose_sensitivity():
     # non-square: queries from one tensor, keys from another with different statistics; a swapped
     # operand or a missing scale changes the answer
