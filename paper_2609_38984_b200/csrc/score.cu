@@ -214,7 +214,7 @@ constexpr int kQualThreads = 1024;
 
 __global__ void __launch_bounds__(kQualThreads) quality_kernel(const float* scores, float* quality, int F, int N_s,
                                                                int parts) {
-  extern __shared__ double2 part_sums[];  // [F * parts]
+  extern __shared__ double2 part_sums[];  // [F * (parts + 1)]
   const int b = blockIdx.x;
   quality_of_scores(scores + (int64_t)b * F * N_s, F, N_s, parts, part_sums, quality + b * 3, kQualThreads);
 }
@@ -506,7 +506,7 @@ cudaError_t launch_score(const Dims& d, const Alpha& alpha, const void* q, const
 cudaError_t launch_quality(const Dims& d, const float* scores, float* quality, cudaStream_t st, int* launches) {
   ++*launches;
   const int parts = quality_parts(d.F);
-  quality_kernel<<<d.B, kQualThreads, (size_t)d.F * parts * sizeof(double2), st>>>(scores, quality, d.F, d.N_s, parts);
+  quality_kernel<<<d.B, kQualThreads, (size_t)d.F * (parts + 1) * sizeof(double2), st>>>(scores, quality, d.F, d.N_s, parts);
   return cudaGetLastError();
 }
 

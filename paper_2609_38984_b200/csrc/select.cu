@@ -418,8 +418,10 @@ cudaError_t select_prepare(const Dims& d) {
   return cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
 
-// the anchor-key area (8 bytes per spatial position) must hold the F * parts partial sums (16 bytes each)
-bool select_can_fold_quality(const Dims& d) { return (size_t)d.N_s * 8 >= (size_t)d.F * quality_parts(d.F) * sizeof(double2); }
+// the anchor-key area (8 bytes per spatial position) must hold the F * (parts + 1) partial sums (16 bytes each)
+bool select_can_fold_quality(const Dims& d) {
+  return (size_t)d.N_s * 8 >= (size_t)d.F * (quality_parts(d.F) + 1) * sizeof(double2);
+}
 
 cudaError_t launch_select(const Dims& d, const float* scores, const float* scores_all, int32_t* sel_idx,
                           int32_t* pack_map, int32_t* inv_map, int* status, cudaStream_t st, int* launches,

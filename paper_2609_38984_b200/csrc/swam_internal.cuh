@@ -23,9 +23,10 @@ struct Alpha {
 
 // Layer quality (Eq. 9) of one sample's scores S [F, N_s] (global or shared memory): R = sum S / F, E = mean normalised
 // spatial entropy, Q = R (1 - E), written to out3[0..2].  Called by every thread of a CTA of `n_threads` threads
-// (a multiple of 32); part_sums: shared memory, F * parts entries.  With a_f = sum_j s and b_f = sum_j s ln s the
-// entropy of frame f is ln a_f - b_f / a_f.  Warps take (frame, part) units; partial sums are combined in a fixed
-// order, so the result does not depend on which kernel calls it.
+// (a multiple of 32); part_sums: shared memory, F * (parts + 1) entries.  With a_f = sum_j s and b_f = sum_j s ln s the
+// entropy of frame f is ln a_f - b_f / a_f.  Warps take (frame, part) units, one thread per frame then forms the
+// frame's sum and entropy term (the double-precision logarithm is the expensive part), and one thread adds the frames
+// up in ascending order: the result does not depend on which kernel calls it.
 __device__ __forceinline__ void quality_of_scores(const float* s, int F, int N_s, int parts, double2* part_sums,
                                                   float* out3, int n_threads) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -47,13 +48,18 @@ __device__ __forceinline__ void quality_of_scores(const float* s, int F, int N_s
     if (lane == 0) part_sums[u] = make_double2(a, bq);
   }
   __syncthreads();
+  double2* frame_terms = part_sums + F * parts;   // (a_f, entropy term of frame f)
+  for (int f = threadIdx.x; f < F; f += n_threads) {
+    double a = 0.0, bq = 0.0;
+    for (int q = 0; q < parts; ++q) { a += part_sums[f * parts + q].x; bq += part_sums[f * parts + q].y; }
+    frame_terms[f] = make_double2(a, (a > 0.0) ? log(a) - bq / a : 0.0);
+  }
+  __syncthreads();
   if (threadIdx.x == 0) {
     double total = 0.0, ent = 0.0;
     for (int f = 0; f < F; ++f) {
-      double a = 0.0, bq = 0.0;
-      for (int q = 0; q < parts; ++q) { a += part_sums[f * parts + q].x; bq += part_sums[f * parts + q].y; }
-      total += a;
-      if (a > 0.0) ent += log(a) - bq / a;
+      total += frame_terms[f].x;
+      if (frame_terms[f].x > 0.0) ent += frame_terms[f].y;
     }
     const double R = total / (double)F;
     const double E = ent / ((double)F * log((double)N_s));
