@@ -179,6 +179,16 @@ int swam_get_scores(const swam_ctx* ctx, const float** scores, const float** lse
 int swam_set_selection(swam_ctx* ctx, const int32_t* sel_idx, const int32_t* pack_map, const int32_t* inv_map,
                        void* stream);
 
+/* The whole cross-step state of swam_step (scores, Eq. 9 diagnostics, action-row normalisers, selection, maps) as one
+ * opaque device buffer: swam_state_bytes gives its size, swam_state_export copies the state into dev_buf and
+ * swam_state_import installs a buffer written by a context of the same shape, after which SWAM_REUSE steps continue
+ * where the exporting context stood (the cached output tensor `out` belongs to the caller and travels separately).
+ * Both copies are asynchronous on `stream`.  Errors: SWAM_ERR_STATE (export before any refresh), SWAM_ERR_WORKSPACE,
+ * SWAM_ERR_INVALID_ARG, SWAM_ERR_CUDA. */
+int swam_state_bytes(const swam_ctx* ctx, size_t* bytes);
+int swam_state_export(swam_ctx* ctx, void* dev_buf, void* stream);
+int swam_state_import(swam_ctx* ctx, const void* dev_buf, void* stream);
+
 /* Synchronises `stream`, reads and clears the device status word; returns SWAM_OK, SWAM_ERR_DEVICE_CHECK,
  * SWAM_ERR_TIMEOUT or SWAM_ERR_CUDA. */
 int swam_check(swam_ctx* ctx, void* stream);

@@ -465,6 +465,33 @@ int swam_set_selection(swam_ctx* c, const int32_t* sel_idx, const int32_t* pack_
   return SWAM_OK;
 }
 
+// the state blocks are laid out back to back in the workspace: scores, quality, normalisers, selection, maps
+int swam_state_bytes(const swam_ctx* c, size_t* bytes) {
+  if (!c || !bytes) return SWAM_ERR_INVALID_ARG;
+  *bytes = c->off_scratch - c->off_scores;
+  return SWAM_OK;
+}
+
+int swam_state_export(swam_ctx* c, void* dev_buf, void* stream) {
+  if (!c || !dev_buf) return fail(c, SWAM_ERR_INVALID_ARG, "swam_state_export: null argument");
+  if (int r = need_ws(c)) return r;
+  if (!c->has_selection) return fail(c, SWAM_ERR_STATE, "swam_state_export: no refresh step has run yet");
+  cudaError_t e = cudaMemcpyAsync(dev_buf, c->ws + c->off_scores, c->off_scratch - c->off_scores, cudaMemcpyDeviceToDevice,
+                                  (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail_cuda(c, e, "swam_state_export");
+  return SWAM_OK;
+}
+
+int swam_state_import(swam_ctx* c, const void* dev_buf, void* stream) {
+  if (!c || !dev_buf) return fail(c, SWAM_ERR_INVALID_ARG, "swam_state_import: null argument");
+  if (int r = need_ws(c)) return r;
+  cudaError_t e = cudaMemcpyAsync(c->ws + c->off_scores, dev_buf, c->off_scratch - c->off_scores, cudaMemcpyDeviceToDevice,
+                                  (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail_cuda(c, e, "swam_state_import");
+  c->has_selection = true;
+  return SWAM_OK;
+}
+
 int swam_get_scores(const swam_ctx* c, const float** scores, const float** lse_action, const float** quality) {
   if (!c || !c->ws) return SWAM_ERR_WORKSPACE;
   if (scores) *scores = (const float*)(c->ws + c->off_scores);

@@ -28,7 +28,8 @@ EXPORTS = [
     "swam_create", "swam_destroy", "swam_workspace_bytes", "swam_bind_workspace", "swam_score", "swam_score_noalloc",
     "swam_select", "swam_aggregate", "swam_select_maps",
     "swam_pack", "swam_sparse_attn", "swam_scatter", "swam_step", "swam_host_io_bytes", "swam_bind_host_io",
-    "swam_step_host", "swam_host_join", "swam_get_selection", "swam_get_scores", "swam_set_selection", "swam_check", "swam_set_option", "swam_launch_count",
+    "swam_step_host", "swam_host_join", "swam_get_selection", "swam_get_scores", "swam_set_selection", "swam_state_bytes",
+    "swam_state_export", "swam_state_import", "swam_check", "swam_set_option", "swam_launch_count",
     "swam_last_error", "swam_version",
 ]
 
@@ -81,6 +82,9 @@ def load_library() -> ctypes.CDLL:
         lib.swam_get_selection.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
         lib.swam_get_scores.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
         lib.swam_set_selection.argtypes = [vp, vp, vp, vp, vp]
+        lib.swam_state_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t)]
+        lib.swam_state_export.argtypes = [vp, vp, vp]
+        lib.swam_state_import.argtypes = [vp, vp, vp]
         lib.swam_check.argtypes = [vp, vp]
         lib.swam_set_option.argtypes = [vp, i32, i32]
         lib.swam_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
@@ -285,6 +289,21 @@ class Swam:
             if t.dtype != torch.int32 or tuple(t.shape) != shape or not t.is_contiguous() or not t.is_cuda:
                 raise ValueError(f"expected a contiguous int32 CUDA tensor of shape {shape}")
         self._chk(self.lib.swam_set_selection(self.ctx, _ptr(sel_idx), _ptr(pack_map), _ptr(inv_map), _stream()))
+
+    def export_state(self) -> torch.Tensor:
+        """The cross-step state (scores, diagnostics, normalisers, selection, maps) as one opaque byte tensor."""
+        n = ctypes.c_size_t()
+        self._chk(self.lib.swam_state_bytes(self.ctx, ctypes.byref(n)))
+        buf = torch.empty(n.value, dtype=torch.uint8, device=self.device)
+        self._chk(self.lib.swam_state_export(self.ctx, _ptr(buf), _stream()))
+        return buf
+
+    def import_state(self, buf: torch.Tensor):
+        n = ctypes.c_size_t()
+        self._chk(self.lib.swam_state_bytes(self.ctx, ctypes.byref(n)))
+        if buf.dtype != torch.uint8 or buf.numel() != n.value or not buf.is_cuda or not buf.is_contiguous():
+            raise ValueError(f"expected a contiguous uint8 CUDA tensor of {n.value} bytes")
+        self._chk(self.lib.swam_state_import(self.ctx, _ptr(buf), _stream()))
 
     def cached_scores(self):
         a, b, c = ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_void_p()

@@ -468,6 +468,31 @@ def test_guided_pair_shares_the_conditional_selection():
     check_float(f64(out_u), st_u.out, wl.dtype)
 
 
+def test_exported_state_continues_in_another_context():
+    swam = _swam()
+    wl = small("larger_imagination", n_obs=40, grid_h=7, grid_w=9, n_heads=2, steps=3)
+    x0, x1, x2 = W.generate_steps(wl, 3)
+    a = swam.Swam.from_workload(wl)
+    out_a = a.empty_full().zero_()
+    with pytest.raises(swam.SwamError) as e:
+        a.export_state()
+    assert e.value.code == swam.ERR_STATE                      # nothing to export before a refresh
+    a.step(dev(x0["q"], wl), dev(x0["k"], wl), dev(x0["v"], wl), swam.REFRESH_FULL, out_a)
+    state, out_b = a.export_state(), out_a.clone()
+    b = swam.Swam.from_workload(wl)
+    b.import_state(state)
+    for x in (x1, x2):
+        a.step(dev(x["q"], wl), dev(x["k"], wl), dev(x["v"], wl), swam.REUSE, out_a)
+        b.step(dev(x["q"], wl), dev(x["k"], wl), dev(x["v"], wl), swam.REUSE, out_b)
+    a.check()
+    b.check()
+    assert torch.equal(out_a, out_b)
+    for ta, tb in zip(a.selection() + a.cached_scores(), b.selection() + b.cached_scores()):
+        assert torch.equal(ta, tb)
+    with pytest.raises(ValueError):
+        b.import_state(state[:-1])
+
+
 def test_corrupt_installed_selection_is_reported_not_followed():
     swam = _swam()
     wl = small()
