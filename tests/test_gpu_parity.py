@@ -257,6 +257,40 @@ def test_attention_with_a_growing_row_maximum(head_dim, pattern):
         assert torch.equal(again, out)
 
 
+@pytest.mark.parametrize("head_dim,n_heads,n", [
+    (64, 50, 768),       # 150 work items on 148 SMs: two left over, cut over the keys
+    (64, 37, 2048),      # 296 items: exactly two per CTA
+    (128, 38, 2148),     # 342 items: two per CTA and 46 left over (split), ragged last tile
+    (128, 5, 4000),      # 80 items: fewer than SMs
+])
+def test_attention_work_distribution_over_persistent_ctas(head_dim, n_heads, n):
+    """Item counts below, at and just above multiples of the SM count: the CTAs walk through several items each and
+    the leftover items are cut over the keys and merged; every element is compared with the mma.sync kernel, sampled
+    rows with the oracle."""
+    swam = _swam()
+    wl = W.WORKLOADS["single_view"].with_(n_obs=n - 64 - 32, grid_h=8, grid_w=8, n_frames=1, n_action=32,
+                                          n_heads=n_heads, head_dim=head_dim, keep=1.0, seed=21)
+    assert wl.seq_len == n
+    x = W.generate_steps(wl, 1)[0]
+    q, k, v = (dev(x[m], wl) for m in "qkv")
+    tc = swam.Swam.from_workload(wl)
+    ref = swam.Swam.from_workload(wl)
+    ref.set_option(swam.OPT_ATTN_VARIANT, swam.ATTN_WARP_MMA)
+    out, lse = tc.sparse_attn(q, k, v, want_lse=True)
+    out_r, lse_r = ref.sparse_attn(q, k, v, want_lse=True)
+    tc.check()
+    diff = (out.float() - out_r.float()).abs()
+    assert float(diff.max()) <= 2e-2 and float(diff.norm() / out_r.float().norm()) <= 5e-3
+    assert float((lse - lse_r).abs().max()) <= 1e-3
+    rng = np.random.default_rng(3)
+    rows = np.stack([np.zeros(24, np.int32), rng.integers(0, n, 24).astype(np.int32)], axis=1)
+    rows[0, 1], rows[1, 1], rows[2, 1] = 0, n - 1, min((n // 256) * 256, n - 1)
+    assert rows[:, 1].min() >= 0 and rows[:, 1].max() < n
+    want, _ = ora.attention_rows(x["q"], x["k"], x["v"], rows)
+    check_float(f64(out[rows[:, 0], rows[:, 1]]), want, wl.dtype)
+    assert torch.equal(out, tc.sparse_attn(q, k, v))          # and the same bits again
+
+
 def test_attention_short_sequences():
     """seq_len below the full length, down to one token."""
     swam = _swam()
