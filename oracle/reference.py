@@ -71,10 +71,24 @@ def expand_kv(x: np.ndarray, n_heads: int) -> np.ndarray:
     return np.repeat(x, n_heads // n_kv, axis=2)
 
 
+SEES_OBSERVED, SEES_FUTURE, SEES_ALL = 0, 1, 2
+
+
+def key_limits(rows: np.ndarray, obs_end: int, fut_end: int, n: int, sees: Sequence[int]) -> np.ndarray:
+    """Visible-key count of each listed (b, r) row under segment-prefix visibility: the sequence is
+    [observed | future | action] with the observed tokens ending at obs_end and the future tokens at fut_end; a row of
+    segment s sees the keys up to the end of the segment sees[s] names (observed, future, or everything)."""
+    ends = np.array([obs_end, fut_end, n], dtype=np.int32)
+    r = np.asarray(rows).reshape(-1, 2)[:, 1]
+    seg = (r >= obs_end).astype(np.int32) + (r >= fut_end).astype(np.int32)
+    return ends[np.asarray(sees, dtype=np.int32)[seg]].astype(np.int32)
+
+
 def attention_rows(q: np.ndarray, k: np.ndarray, v: np.ndarray, rows: np.ndarray,
-                   scale: Optional[float] = None) -> Tuple[np.ndarray, np.ndarray]:
+                   scale: Optional[float] = None, key_limit: Optional[np.ndarray] = None) -> Tuple[np.ndarray, np.ndarray]:
     """Softmax attention (Sec. 3.1) for the listed (b, r) query rows, all heads.
-    q: [B, n, N_h, D], k, v: [B, n, N_h or N_kv, D] float32.  Returns out [n_rows, N_h, D], lse [n_rows, N_h] (float64)."""
+    q: [B, n, N_h, D], k, v: [B, n, N_h or N_kv, D] float32.  key_limit: per listed row, the number of leading keys it
+    sees (None = all).  Returns out [n_rows, N_h, D], lse [n_rows, N_h] (float64)."""
     lib = _load()
     q = np.ascontiguousarray(q, dtype=np.float32)
     k = np.ascontiguousarray(expand_kv(k, q.shape[2]), dtype=np.float32)
@@ -87,24 +101,30 @@ def attention_rows(q: np.ndarray, k: np.ndarray, v: np.ndarray, rows: np.ndarray
     lib.oracle_attention_rows(_p(q, ctypes.c_float), _p(k, ctypes.c_float), _p(v, ctypes.c_float),
                               ctypes.c_int(n), ctypes.c_int(nh), ctypes.c_int(d), ctypes.c_double(scale),
                               _p(rows, ctypes.c_int32), ctypes.c_int64(rows.shape[0]),
-                              _p(out, ctypes.c_double), _p(lse, ctypes.c_double))
+                              _p(out, ctypes.c_double), _p(lse, ctypes.c_double),
+                              None if key_limit is None else _p(np.ascontiguousarray(key_limit, dtype=np.int32), ctypes.c_int32))
     return out, lse
 
 
-def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray,
-              scale: Optional[float] = None) -> Tuple[np.ndarray, np.ndarray]:
-    """All rows: out [B, n, N_h, D], lse [B, N_h, n]."""
+def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, scale: Optional[float] = None,
+              visibility: Optional[Tuple[int, int, Sequence[int]]] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """All rows: out [B, n, N_h, D], lse [B, N_h, n].  visibility = (obs_end, fut_end, sees) restricts each row to
+    the key prefix its segment sees (see key_limits); None = every row sees every key."""
     b, n, nh, d = q.shape
     rows = np.stack(np.meshgrid(np.arange(b), np.arange(n), indexing="ij"), axis=-1).reshape(-1, 2)
-    out, lse = attention_rows(q, k, v, rows, scale)
+    lim = None if visibility is None else key_limits(rows, visibility[0], visibility[1], n, visibility[2])
+    out, lse = attention_rows(q, k, v, rows, scale, lim)
     return out.reshape(b, n, nh, d), np.ascontiguousarray(lse.reshape(b, n, nh).transpose(0, 2, 1))
 
 
-def action_lse(q: np.ndarray, k: np.ndarray, n_action: int, scale: Optional[float] = None) -> np.ndarray:
-    """lambda_h(i): log-sum-exp of the action queries over all keys of the full sequence.  [B, N_h, H]."""
+def action_lse(q: np.ndarray, k: np.ndarray, n_action: int, scale: Optional[float] = None,
+               n_visible: Optional[int] = None) -> np.ndarray:
+    """lambda_h(i): log-sum-exp of the action queries over the keys they see: all keys of the full sequence, or its
+    first n_visible keys (App. A.2: "over all visible keys").  [B, N_h, H]."""
     b, n, nh, d = q.shape
     rows = np.stack(np.meshgrid(np.arange(b), np.arange(n - n_action, n), indexing="ij"), axis=-1).reshape(-1, 2)
-    _, lse = attention_rows(q, k, np.zeros_like(k, dtype=np.float32), rows, scale)
+    lim = None if n_visible is None else np.full(rows.shape[0], n_visible, dtype=np.int32)
+    _, lse = attention_rows(q, k, np.zeros_like(k, dtype=np.float32), rows, scale, lim)
     return np.ascontiguousarray(lse.reshape(b, n_action, nh).transpose(0, 2, 1))
 
 
@@ -241,28 +261,43 @@ class StepState:
         self.sel: Optional[Dict[str, np.ndarray]] = None
         self.pack_map: Optional[np.ndarray] = None
         self.inv_map: Optional[np.ndarray] = None
+        self.sees: Optional[Sequence[int]] = None    # segment-prefix visibility of the backbone, None = full
+        self.n_obs = 0
+        self.n_action = 0
 
 
 def full_step(st: StepState, q, k, v, n_obs, n_frames, n_spatial, n_action, k_core, k_anchor,
-              beta: float = 1.0, rows: Optional[np.ndarray] = None, scale: Optional[float] = None) -> StepState:
+              beta: float = 1.0, rows: Optional[np.ndarray] = None, scale: Optional[float] = None,
+              sees: Optional[Sequence[int]] = None) -> StepState:
     """Dense joint attention over all L tokens, then score, select and build the maps.
     With `rows` given only those (b, r) rows of the dense output are computed (sampled parity at full size);
-    st.out then holds NaN elsewhere."""
+    st.out then holds NaN elsewhere.  sees: segment-prefix visibility (see key_limits), None = full."""
     b, n, nh, d = q.shape
+    obs_end, fut_end = n_obs, n_obs + n_frames * n_spatial
+    vis = None if sees is None else (obs_end, fut_end, sees)
+    st.sees, st.n_obs, st.n_action = sees, n_obs, n_action
     if rows is None:
-        out, lse = attention(q, k, v, scale)
+        out, lse = attention(q, k, v, scale, vis)
         lse_act = np.ascontiguousarray(lse[:, :, n - n_action:])
         st.out = out
     else:
-        o, _ = attention_rows(q, k, v, rows, scale)
+        lim = None if sees is None else key_limits(rows, obs_end, fut_end, n, sees)
+        o, _ = attention_rows(q, k, v, rows, scale, lim)
         st.out = np.full((b, n, nh, d), np.nan)
         st.out[rows[:, 0], rows[:, 1]] = o
-        lse_act = action_lse(q, k, n_action, scale)
+        lse_act = action_lse(q, k, n_action, scale, None if sees is None else [obs_end, fut_end, n][sees[2]])
     s64 = score(q, k, n_obs, n_frames, n_spatial, n_action, lse=lse_act, scale=scale)
     st.scores = s64.astype(np.float32)
     st.sel = select(st.scores, k_core, k_anchor, beta)
     st.pack_map, st.inv_map = maps(st.sel["sel_idx"], n_obs, n_spatial, n_action)
     return st
+
+
+def _packed_visibility(st: "StepState", n_p: int):
+    """(obs_end, fut_end, sees) of the packed sequence [observed | F * K retained | action], or None."""
+    if st.sees is None:
+        return None
+    return (st.n_obs, n_p - st.n_action, st.sees)
 
 
 def sparse_step(st: StepState, q, k, v, rows_packed: Optional[np.ndarray] = None,
@@ -271,25 +306,28 @@ def sparse_step(st: StepState, q, k, v, rows_packed: Optional[np.ndarray] = None
     attention output ([B, L', N_h, D], or the listed packed rows when `rows_packed` is given)."""
     assert st.pack_map is not None, "a full step must come first"
     qp, kp, vp = pack(q, st.pack_map), pack(k, st.pack_map), pack(v, st.pack_map)
+    n_p = qp.shape[1]
     if rows_packed is None:
-        op, _ = attention(qp, kp, vp, scale)
+        op, _ = attention(qp, kp, vp, scale, _packed_visibility(st, n_p))
         st.out = scatter(op, st.pack_map, st.out)
         return op
-    o, _ = attention_rows(qp, kp, vp, rows_packed, scale)
+    vis = _packed_visibility(st, n_p)
+    lim = None if vis is None else key_limits(rows_packed, vis[0], vis[1], n_p, vis[2])
+    o, _ = attention_rows(qp, kp, vp, rows_packed, scale, lim)
     orig = st.pack_map[rows_packed[:, 0], rows_packed[:, 1]]
     st.out[rows_packed[:, 0], orig] = o
     return o
 
 
 def run_steps(steps: Sequence[Dict[str, np.ndarray]], refresh: int, n_obs, n_frames, n_spatial, n_action,
-              k_core, k_anchor, beta: float = 1.0) -> List[Dict[str, np.ndarray]]:
+              k_core, k_anchor, beta: float = 1.0, sees: Optional[Sequence[int]] = None) -> List[Dict[str, np.ndarray]]:
     """All denoising steps of one action chunk; step t is a full step when t % refresh == 0."""
     st = StepState()
     log = []
     for t, x in enumerate(steps):
         is_full = (t % refresh) == 0
         if is_full:
-            full_step(st, x["q"], x["k"], x["v"], n_obs, n_frames, n_spatial, n_action, k_core, k_anchor, beta)
+            full_step(st, x["q"], x["k"], x["v"], n_obs, n_frames, n_spatial, n_action, k_core, k_anchor, beta, sees=sees)
         else:
             sparse_step(st, x["q"], x["k"], x["v"])
         log.append(dict(full=is_full, out=st.out.copy(), scores=st.scores.copy(),

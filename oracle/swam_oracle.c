@@ -27,16 +27,20 @@
 
 /* ------------------------------------------------------------------------
  * Softmax attention, plain definition (Sec. 3.1; the compact sequence of
- * Sec. 4.2 is the same operation on fewer tokens).  Full visibility.
+ * Sec. 4.2 is the same operation on fewer tokens).
  *   x_c = scale * sum_d Q[r,d] K[c,d];  lambda_r = log sum_c exp(x_c)
  *   O[r,:] = sum_c exp(x_c - lambda_r) V[c,:]
+ * The sums run over the keys visible to the row: all n of them when
+ * key_limit is NULL (full visibility), else the first key_limit[i] keys of
+ * the sequence for the i-th listed row (the backbone's visibility
+ * constraints of App. A.2, read as: a token sees a prefix of the sequence).
  * rows: [n_rows, 2] pairs (b, r).  out_rows: [n_rows, N_h, D];
  * lse_rows: [n_rows, N_h] (may be NULL).
  * ------------------------------------------------------------------------ */
 void oracle_attention_rows(const float* q, const float* k, const float* v,
                            int n, int n_heads, int head_dim, double scale,
                            const int32_t* rows, int64_t n_rows,
-                           double* out_rows, double* lse_rows)
+                           double* out_rows, double* lse_rows, const int32_t* key_limit)
 {
     const int64_t tok = (int64_t)n_heads * head_dim;
     const int64_t work = n_rows * n_heads;
@@ -51,8 +55,9 @@ void oracle_attention_rows(const float* q, const float* k, const float* v,
             const float* qr = q + (b * n + r) * tok + (int64_t)h * head_dim;
             const float* kb = k + b * n * tok + (int64_t)h * head_dim;
             const float* vb = v + b * n * tok + (int64_t)h * head_dim;
+            const int nv = key_limit ? key_limit[ri] : n;   /* visible keys of this row */
             double m = -INFINITY;
-            for (int c = 0; c < n; ++c) {
+            for (int c = 0; c < nv; ++c) {
                 const float* kc = kb + (int64_t)c * tok;
                 double dot = 0.0;
                 for (int d = 0; d < head_dim; ++d) dot += (double)qr[d] * (double)kc[d];
@@ -60,11 +65,11 @@ void oracle_attention_rows(const float* q, const float* k, const float* v,
                 if (x[c] > m) m = x[c];
             }
             double sum = 0.0;
-            for (int c = 0; c < n; ++c) sum += exp(x[c] - m);
+            for (int c = 0; c < nv; ++c) sum += exp(x[c] - m);
             const double lambda = m + log(sum);
             double* o = out_rows + (ri * n_heads + h) * head_dim;
             for (int d = 0; d < head_dim; ++d) o[d] = 0.0;
-            for (int c = 0; c < n; ++c) {
+            for (int c = 0; c < nv; ++c) {
                 const double p = exp(x[c] - lambda);
                 const float* vc = vb + (int64_t)c * tok;
                 for (int d = 0; d < head_dim; ++d) o[d] += p * (double)vc[d];

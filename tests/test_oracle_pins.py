@@ -442,3 +442,28 @@ def test_select2_uses_core_map_for_cores_and_all_map_for_anchors():
     sel = ora.select2(v_core, v_all, kc, ks)
     assert sel[0, 0].tolist() == [2, 3, 7, 10, 11] and sel[0, 1].tolist() == [1, 2, 5, 10, 11]
 
+
+
+def test_segment_prefix_visibility_matches_library_mask():
+    """Rows restricted to a key prefix per segment equal the library's attention under the corresponding boolean mask;
+    a mask transposed (keys restricted by their own segment instead of the query's) gives a different answer."""
+    q, k, v = _rand_qkv(5, 2, 29, 2, 8)
+    obs_end, fut_end, n = 7, 21, 29
+    for sees in ((0, 1, 2), (2, 1, 2), (0, 2, 1), (2, 2, 2)):
+        out, lse = ora.attention(q, k, v, visibility=(obs_end, fut_end, sees))
+        ends = np.array([obs_end, fut_end, n])
+        seg = (np.arange(n) >= obs_end).astype(int) + (np.arange(n) >= fut_end).astype(int)
+        mask = np.arange(n)[None, :] < ends[np.array(sees)[seg]][:, None]            # [query, key]
+        tq, tk, tv = [torch.from_numpy(x).double().permute(0, 2, 1, 3) for x in (q, k, v)]
+        ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, attn_mask=torch.from_numpy(mask))
+        assert np.abs(out - ref.permute(0, 2, 1, 3).numpy()).max() < 1e-12
+        logits = torch.einsum("bhqd,bhkd->bhqk", tq, tk) / np.sqrt(8)
+        logits = logits.masked_fill(~torch.from_numpy(mask), -np.inf)
+        assert np.abs(lse - torch.logsumexp(logits, -1).numpy()).max() < 1e-12
+        if sees != (2, 2, 2):
+            wrong = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, attn_mask=torch.from_numpy(mask.T.copy() | np.eye(n, dtype=bool)))
+            assert np.abs(out - wrong.permute(0, 2, 1, 3).numpy()).max() > 1e-3
+    # the action-row normaliser over a key prefix is the masked log-sum-exp of those rows
+    lam = ora.action_lse(q, k, 8, n_visible=fut_end)
+    _, lse_vis = ora.attention(q, k, v, visibility=(obs_end, fut_end, (2, 2, 1)))
+    assert np.abs(lam - lse_vis[:, :, n - 8:]).max() < 1e-12
