@@ -202,10 +202,23 @@ int swam_check(swam_ctx* ctx, void* stream);
  * Q through pack_map and writes each retained row straight to its original position in `out`, so that the packed Q,
  * the packed output and the scatter pass do not exist; SWAM_SPARSE_STAGED runs swam_pack, swam_sparse_attn and
  * swam_scatter one after the other.  The fused path needs bf16, head_dim 64 or 128 and SWAM_ATTN_AUTO; every other
- * configuration runs staged.  Both paths produce the same bits. */
-enum { SWAM_OPT_ATTN_VARIANT = 1, SWAM_OPT_SPARSE_PATH = 2 };
+ * configuration runs staged.  Both paths produce the same bits.
+ *
+ * SWAM_OPT_VISIBILITY sets the backbone's visibility constraints (App. A.2) in the form this library supports: the
+ * joint sequence is [observed | future | action], and the rows of each of the three segments see a prefix of it, up to
+ * the end of the observed tokens (SWAM_SEES_OBSERVED), of the future tokens (SWAM_SEES_FUTURE) or of the whole
+ * sequence (SWAM_SEES_ALL).  value = SWAM_VISIBILITY(observed_rows_see, future_rows_see, action_rows_see); the default
+ * is SWAM_SEES_ALL for all three (full visibility).  Future rows must see at least the future tokens and action rows
+ * at least the future tokens (they score them).  The setting applies to swam_step, to swam_sparse_attn at the full
+ * and the packed length (segment boundaries N_o and N_o + F*N_s, or N_o and N_o + F*K; other lengths return
+ * SWAM_ERR_UNSUPPORTED unless visibility is full) and to the normalisers swam_score computes, which then run over the
+ * keys the action rows see. */
+enum { SWAM_OPT_ATTN_VARIANT = 1, SWAM_OPT_SPARSE_PATH = 2, SWAM_OPT_VISIBILITY = 3 };
 enum { SWAM_ATTN_AUTO = 0, SWAM_ATTN_WARP_MMA = 1 };
 enum { SWAM_SPARSE_FUSED = 0, SWAM_SPARSE_STAGED = 1 };
+enum { SWAM_SEES_OBSERVED = 0, SWAM_SEES_FUTURE = 1, SWAM_SEES_ALL = 2 };
+#define SWAM_VISIBILITY(observed_rows_see, future_rows_see, action_rows_see) \
+  ((observed_rows_see) | ((future_rows_see) << 2) | ((action_rows_see) << 4))
 int swam_set_option(swam_ctx* ctx, int32_t option, int32_t value);
 
 /* Number of kernels this context has launched so far (host-side counter). */

@@ -76,7 +76,12 @@ __global__ void __launch_bounds__(kThreads) attn_bf16_mma_kernel(const AttnArgs 
   const __nv_bfloat16* qb = (const __nv_bfloat16*)a.q + (int64_t)b * a.n * rs + (int64_t)h * D;
   const __nv_bfloat16* kb = (const __nv_bfloat16*)a.k + (int64_t)b * a.n * rs_kv + (int64_t)h_kv * D;
   const __nv_bfloat16* vb = (const __nv_bfloat16*)a.v + (int64_t)b * a.n * rs_kv + (int64_t)h_kv * D;
-  const int n_tiles = (a.n + BN - 1) / BN;
+  // key tiles up to what some row of this block sees; each thread's two rows (gq and gq + 8 of the warp's 16) see
+  // the first lim_r[0], lim_r[1] keys
+  const int block_lim = a.max_limit(m0, min(m0 + BM, a.n) > m0 ? min(m0 + BM, a.n) : m0 + 1);
+  const int n_tiles = (block_lim + BN - 1) / BN;
+  const int lim_r[2] = {a.row_limit(m0 + warp * 16 + gq), a.row_limit(m0 + warp * 16 + gq + 8)};
+  const int lim_min = min(a.lim[0], min(a.lim[1], a.lim[2]));
   const float sl2 = a.scale * kLog2e;
 
   load_tile<D>(sQ, qb, rs, m0, a.n, tid);
@@ -120,13 +125,13 @@ __global__ void __launch_bounds__(kThreads) attn_bf16_mma_kernel(const AttnArgs 
     }
     // scale into the log2 domain; keys beyond the sequence get -inf
     const int c_base = j * BN + 2 * t;
-    const bool tail = (j + 1) * BN > a.n;
+    const bool tail = (j + 1) * BN > lim_min;     // some row of some block may not see all keys of this tile
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const int c = c_base + i * 8 + (e & 1);
-        s[i][e] = (tail && c >= a.n) ? -INFINITY : s[i][e] * sl2;
+        s[i][e] = (tail && c >= lim_r[e >> 1]) ? -INFINITY : s[i][e] * sl2;
       }
     }
     // online softmax: rows gq (elements 0,1) and gq+8 (elements 2,3)

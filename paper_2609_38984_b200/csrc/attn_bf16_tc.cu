@@ -253,6 +253,9 @@ struct TcParams {
   int splits;          // pieces per split item (0 when nothing is split)
   int tiles_per_split; // key tiles per piece
   float scale_log2;
+  // segment-prefix visibility: rows [0, obs_end) see the first lim0 keys, rows [obs_end, fut_end) the first lim1, the
+  // rest the first lim2 (all equal to n: full visibility)
+  int obs_end, fut_end, lim0, lim1, lim2;
 };
 
 template <int D>
@@ -284,7 +287,8 @@ struct TcCfg {
 enum { kDirect = 0, kScatter = 1, kGather = 2 };
 constexpr int kGatherThreads = 64;   // warps 10 and 11
 
-template <int D, int MODE>
+// VIS: visibility is restricted (per-row key limits); false = every row sees all n keys and none of that code exists
+template <int D, int MODE, bool VIS>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o, const TcParams p) {
@@ -326,6 +330,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   // so that the next item's key/value tiles stream in while this item's epilogue runs and nothing is set up twice.
   struct Work { int h, b, row0, kv_begin, n_tiles, slot; };
   const int all_tiles = (p.n + kTile - 1) / kTile;
+  auto row_limit = [&](int row) { return row < p.obs_end ? p.lim0 : (row < p.fut_end ? p.lim1 : p.lim2); };
   auto decode = [&](int w) {
     Work k;
     int item = w, kv_end = all_tiles;
@@ -341,6 +346,15 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     k.h = (item / p.pairs) % p.N_h;
     k.b = item / (p.pairs * p.N_h);
     k.row0 = pair * 2 * kTile;
+    // key tiles beyond what any row of the pair sees are not visited (items are not cut over the keys when visibility
+    // is restricted, so kv_begin is 0 then)
+    if (VIS) {
+      const int r_last = min(k.row0 + 2 * kTile, p.n) - 1;
+      int lim = row_limit(k.row0);
+      if (r_last >= p.obs_end && k.row0 < p.fut_end) lim = max(lim, p.lim1);
+      if (r_last >= p.fut_end) lim = max(lim, p.lim2);
+      kv_end = min(kv_end, (lim + kTile - 1) / kTile);
+    }
     k.n_tiles = kv_end - k.kv_begin;  // >= 1 by construction
     return k;
   };
@@ -599,6 +613,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const Work wk = decode(work);
     const int h = wk.h, b = wk.b, row0 = wk.row0, kv_begin = wk.kv_begin, n_tiles = wk.n_tiles, slot = wk.slot;
     float m_used = -INFINITY, l_run = 0.f;
+    const int row_keys = VIS ? row_limit(row0 + s * kTile + r) : p.n;   // leading keys of the sequence this row sees
     for (int j = 0; j < n_tiles; ++j) {
       const int item = it0 + 2 * j + s, buf = item % NB;
       const uint32_t tS = tm_S(buf) + lane_off;
@@ -613,7 +628,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<float(*)[32]>(&sv[c * 32]));
       tmem_ld_wait();
       if (r == 0 && iter == 0) TRACE(s, j * 8 + 2);
-      const int valid = p.n - (kv_begin + j) * kTile;  // keys of this tile inside the sequence
+      const int valid = row_keys - (kv_begin + j) * kTile;  // keys of this tile that this row sees (<= 0: none)
       if (valid < kTile) {
 #pragma unroll
         for (int c = 0; c < kTile; ++c)
@@ -934,8 +949,8 @@ int sm_count_tc() {
 
 // kScatter: a.out is the full [B, n_full, N_h, D] tensor and pack_map [B, a.n] names the row each attended row goes
 // to.  kGather: a.q is the full tensor as well and pack_map also names the query rows.
-template <int D, int MODE>
-cudaError_t launch_tc_d(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, float* partial,
+template <int D, int MODE, bool VIS>
+cudaError_t launch_tc_v(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, float* partial,
                         size_t partial_bytes, cudaStream_t st, int* launches) {
   CUtensorMap mq, mk, mv, mo;
   if (!(MODE != kDirect ? make_map(&mo, a.out, a.B, n_full, a.N_h, D, 1) : make_map(&mo, a.out, a.B, a.n, a.N_h, D)))
@@ -946,7 +961,7 @@ cudaError_t launch_tc_d(const AttnArgs& a, const int32_t* pack_map, int n_full, 
   } else if (!make_map(&mq, a.q, a.B, a.n, a.N_h, D)) {
     return cudaErrorInvalidValue;
   }
-  cudaError_t e = cudaFuncSetAttribute(attn_bf16_tc_kernel<D, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<D>::kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(attn_bf16_tc_kernel<D, MODE, VIS>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<D>::kSmemBytes);
   if (e != cudaSuccess) return e;
   const int pairs = (a.n + 2 * kTile - 1) / (2 * kTile);
   const int items = pairs * a.N_h * a.B;
@@ -954,7 +969,7 @@ cudaError_t launch_tc_d(const AttnArgs& a, const int32_t* pack_map, int n_full, 
   const int sms = sm_count_tc();
   // one CTA per SM: the items beyond the last full wave are cut over the keys into pieces that fill the idle SMs
   int rem = items % sms, splits = 0, per = n_tiles;
-  if (items > sms && rem > 0 && rem <= sms / 2 && n_tiles >= 4) {
+  if (items > sms && rem > 0 && rem <= sms / 2 && n_tiles >= 4 && a.full_visibility()) {
     int want = sms / rem;
     if (want > 16) want = 16;
     if (want > n_tiles / 2) want = n_tiles / 2;
@@ -969,10 +984,10 @@ cudaError_t launch_tc_d(const AttnArgs& a, const int32_t* pack_map, int n_full, 
       (long long*)partial_trace_buffer(),
 #endif
       a.lse, status, partial, pack_map, n_full, (const __nv_bfloat16*)a.q, a.lse_row0, a.lse_rows, a.n, a.N_h, a.N_h / a.N_kv, pairs, n_whole + (splits ? rem * splits : 0), n_whole, splits, per,
-      a.scale * kLog2e};
+      a.scale * kLog2e, a.obs_end, a.fut_end, a.lim[0], a.lim[1], a.lim[2]};
   const int grid = p.total_work < sms ? p.total_work : sms;   // one CTA per SM; each walks through its share of the work
   ++*launches;
-  attn_bf16_tc_kernel<D, MODE><<<grid, kThreadsTc, TcCfg<D>::kSmemBytes, st>>>(mq, mk, mv, mo, p);
+  attn_bf16_tc_kernel<D, MODE, VIS><<<grid, kThreadsTc, TcCfg<D>::kSmemBytes, st>>>(mq, mk, mv, mo, p);
   e = cudaGetLastError();
   if (e != cudaSuccess || !splits) return e;
   CombineParams c{partial, MODE != kDirect ? pack_map : nullptr, n_full, status, (__nv_bfloat16*)a.out, a.lse, a.lse_row0, a.lse_rows,
@@ -980,6 +995,13 @@ cudaError_t launch_tc_d(const AttnArgs& a, const int32_t* pack_map, int n_full, 
   ++*launches;
   attn_combine_kernel<D><<<(rem * 2 * kTile + 7) / 8, 256, 0, st>>>(c);
   return cudaGetLastError();
+}
+
+template <int D, int MODE>
+cudaError_t launch_tc_d(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, float* partial,
+                        size_t partial_bytes, cudaStream_t st, int* launches) {
+  return a.full_visibility() ? launch_tc_v<D, MODE, false>(a, pack_map, n_full, status, partial, partial_bytes, st, launches)
+                             : launch_tc_v<D, MODE, true>(a, pack_map, n_full, status, partial, partial_bytes, st, launches);
 }
 
 }  // namespace

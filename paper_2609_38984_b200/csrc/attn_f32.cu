@@ -17,6 +17,7 @@ __global__ void __launch_bounds__(kRows * 32) attn_f32_kernel(const AttnArgs a) 
   const int h = blockIdx.y, b = blockIdx.z;
   const int row = blockIdx.x * kRows + warp;
   const bool active = row < a.n;
+  const int row_keys = a.row_limit(row);   // leading keys of the sequence this row sees
   const int64_t tok = (int64_t)a.N_h * D;
   const float* q = (const float*)a.q + ((int64_t)b * a.n) * tok + (int64_t)h * D;
   const int64_t tok_kv = (int64_t)a.N_kv * D;
@@ -45,7 +46,7 @@ __global__ void __launch_bounds__(kRows * 32) attn_f32_kernel(const AttnArgs a) 
     float dot = 0.f;
 #pragma unroll 8
     for (int d = 0; d < D; ++d) dot = fmaf(Qs[warp][d], Ks[lane][d], dot);
-    const float x = (c0 + lane < a.n) ? dot * a.scale : -INFINITY;
+    const float x = (c0 + lane < row_keys) ? dot * a.scale : -INFINITY;
     float mx = x;
 #pragma unroll
     for (int s = 16; s > 0; s >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));

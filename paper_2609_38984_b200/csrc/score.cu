@@ -248,6 +248,7 @@ struct LseFlashParams {
   int H, N_h, L, n_splits, tiles_per_split;
   float scale_log2;
   int N_kv;
+  int Lk;                   // leading keys the action rows see (<= L)
 };
 
 __device__ __forceinline__ void lse_cp_async16(uint32_t dst, const void* src, int src_bytes) {
@@ -296,11 +297,11 @@ __global__ void __launch_bounds__(kFlashThreads) lse_flash_bf16_kernel(const Lse
   const int64_t rs = (int64_t)p.N_h * D, rs_k = (int64_t)p.N_kv * D;
   const __nv_bfloat16* kb = p.k + (int64_t)b * p.L * rs_k + (int64_t)(h / (p.N_h / p.N_kv)) * D;
   const __nv_bfloat16* qb = p.q + ((int64_t)b * p.L + (p.L - p.H)) * rs + (int64_t)h * D;   // action rows
-  const int n_tiles = (p.L + kFlashBN - 1) / kFlashBN;
+  const int n_tiles = (p.Lk + kFlashBN - 1) / kFlashBN;
   const int j0 = split * p.tiles_per_split, j1 = min(n_tiles, j0 + p.tiles_per_split);
 
   lse_load_tile<D>(sQ, qb, rs, qc * 64, p.H, tid);
-  if (j0 < j1) lse_load_tile<D>(sK, kb, rs_k, j0 * kFlashBN, p.L, tid);
+  if (j0 < j1) lse_load_tile<D>(sK, kb, rs_k, j0 * kFlashBN, p.Lk, tid);
   asm volatile("cp.async.commit_group;" ::: "memory");
   asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
@@ -314,7 +315,7 @@ __global__ void __launch_bounds__(kFlashThreads) lse_flash_bf16_kernel(const Lse
   for (int j = j0; j < j1; ++j) {
     const int buf = (j - j0) & 1;
     if (j + 1 < j1) {
-      lse_load_tile<D>(sK + (buf ^ 1) * kFlashBN * D * 2, kb, rs_k, (j + 1) * kFlashBN, p.L, tid);
+      lse_load_tile<D>(sK + (buf ^ 1) * kFlashBN * D * 2, kb, rs_k, (j + 1) * kFlashBN, p.Lk, tid);
       asm volatile("cp.async.commit_group;" ::: "memory");
     }
     const uint32_t kt = sK + buf * kFlashBN * D * 2;
@@ -334,7 +335,7 @@ __global__ void __launch_bounds__(kFlashThreads) lse_flash_bf16_kernel(const Lse
     }
     // log2 domain; keys beyond the sequence count as -inf
     const int c_base = j * kFlashBN + wn * NPW * 16 + 2 * t;
-    const bool tail = (j + 1) * kFlashBN > p.L;
+    const bool tail = (j + 1) * kFlashBN > p.Lk;
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
       float mx = -INFINITY;
@@ -344,7 +345,7 @@ __global__ void __launch_bounds__(kFlashThreads) lse_flash_bf16_kernel(const Lse
         for (int e = 0; e < 2; ++e) {
           const int c = c_base + i * 8 + e;
           float v = s[i][2 * r + e] * p.scale_log2;
-          if (tail && c >= p.L) v = -INFINITY;
+          if (tail && c >= p.Lk) v = -INFINITY;
           s[i][2 * r + e] = v;
           mx = fmaxf(mx, v);
         }
@@ -406,14 +407,14 @@ __global__ void __launch_bounds__(256) lse_merge_kernel(const float2* partial, f
 }
 
 // fp32: one CTA per (b, h, i); threads stride over keys with a running (max, sum) in natural-log units
-__global__ void __launch_bounds__(128) lse_f32_kernel(const float* q, const float* k, float* lse, int L, int H,
+__global__ void __launch_bounds__(128) lse_f32_kernel(const float* q, const float* k, float* lse, int L, int Lk, int H,
                                                       int N_h, int N_kv, int D, float scale) {
   __shared__ float sm[4], ss[4];
   const int i = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int64_t tok = (int64_t)N_h * D;
   const float* qt = q + ((int64_t)b * L + (L - H) + i) * tok + (int64_t)h * D;
   float m = -INFINITY, s = 0.f;
-  for (int c = threadIdx.x; c < L; c += blockDim.x) {
+  for (int c = threadIdx.x; c < Lk; c += blockDim.x) {   // the keys the action rows see
     const float* kt = k + ((int64_t)b * L + c) * ((int64_t)N_kv * D) + (int64_t)(h / (N_h / N_kv)) * D;
     float dot = 0.f;
     for (int d = 0; d < D; ++d) dot = fmaf(qt[d], kt[d], dot);
@@ -545,15 +546,15 @@ cudaError_t static_scratch(const Dims& d, float** lse, void** partial) {
 }
 
 cudaError_t launch_action_lse(const Dims& d, const void* q, const void* k, float* lse, void* scratch,
-                              cudaStream_t st, int* launches) {
+                              cudaStream_t st, int* launches, int n_keys) {
   if (d.dtype == 0) {
     ++*launches;
     dim3 grid(d.H, d.N_h, d.B);
-    lse_f32_kernel<<<grid, 128, 0, st>>>((const float*)q, (const float*)k, lse, d.L, d.H, d.N_h, d.N_kv, d.D, d.scale);
+    lse_f32_kernel<<<grid, 128, 0, st>>>((const float*)q, (const float*)k, lse, d.L, n_keys, d.H, d.N_h, d.N_kv, d.D, d.scale);
     return cudaGetLastError();
   }
   // key ranges per CTA: enough CTAs for about four per SM, never more ranges than the scratch has room for
-  const int n_tiles = (d.L + kFlashBN - 1) / kFlashBN;
+  const int n_tiles = (n_keys + kFlashBN - 1) / kFlashBN;
   const int q_chunks = (d.H + 63) / 64;
   const int max_splits = (d.L + kLseKeys - 1) / kLseKeys;
   int sms = 148;
@@ -566,7 +567,7 @@ cudaError_t launch_action_lse(const Dims& d, const void* q, const void* k, float
   const int per = (n_tiles + want - 1) / want;
   const int n_chunks = (n_tiles + per - 1) / per;     // = number of key ranges
   LseFlashParams p{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (float2*)scratch, d.H, d.N_h, d.L, n_chunks, per,
-                   d.scale * kLog2e, d.N_kv};
+                   d.scale * kLog2e, d.N_kv, n_keys};
   const int wm = d.H >= 64 ? 4 : (d.H > 16 ? 2 : 1);    // warps over the query rows (H <= 16, <= 32, more)
   dim3 grid(n_chunks, d.N_h, d.B * q_chunks);
   cudaError_t e = cudaSuccess;

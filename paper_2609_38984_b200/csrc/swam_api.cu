@@ -22,6 +22,7 @@ struct swam_ctx {
   bool has_selection;
   int attn_variant;  // SWAM_ATTN_AUTO | SWAM_ATTN_WARP_MMA
   int sparse_path;   // SWAM_SPARSE_FUSED | SWAM_SPARSE_STAGED
+  int sees[3];       // what observed / future / action rows see: SWAM_SEES_*
   // host-io staging (device): two input slots of (q, k, v) and the persistent output, plus the copy pipeline
   unsigned char* io;
   size_t io_need;
@@ -59,9 +60,33 @@ void count(swam_ctx* c) {
   c->launches_i = 0;
 }
 
+bool full_visibility(const swam_ctx* c) {
+  return c->sees[0] == SWAM_SEES_ALL && c->sees[1] == SWAM_SEES_ALL && c->sees[2] == SWAM_SEES_ALL;
+}
+
+// keys of the full sequence that the action rows see (the normalisers of the scorer run over them)
+int action_keys(const swam_ctx* c) { return c->sees[2] == SWAM_SEES_ALL ? c->d.L : c->d.L - c->d.H; }
+
+// Fills the visibility fields of `a` for a sequence of a.n tokens: the full sequence (future segment of F * N_s
+// tokens) or the packed one (F * K).  False when the context restricts visibility and a.n is neither length.
+bool set_visibility(const swam_ctx* c, AttnArgs& a) {
+  const Dims& d = c->d;
+  a.obs_end = a.fut_end = a.n;
+  a.lim[0] = a.lim[1] = a.lim[2] = a.n;
+  if (full_visibility(c)) return true;
+  if (a.n != d.L && a.n != d.Lp) return false;
+  a.obs_end = d.n_obs;
+  a.fut_end = a.n - d.H;
+  const int ends[3] = {a.obs_end, a.fut_end, a.n};
+  for (int s = 0; s < 3; ++s) a.lim[s] = ends[c->sees[s]];
+  return true;
+}
+
 int run_attention(swam_ctx* c, const void* q, const void* k, const void* v, int n, void* out, float* lse, int lse_row0,
                   int lse_rows, cudaStream_t st) {
   AttnArgs a{q, k, v, out, lse, lse_row0, lse_rows, c->d.B, n, c->d.N_h, c->d.D, c->d.scale, c->d.N_kv};
+  if (!set_visibility(c, a))
+    return fail(c, SWAM_ERR_UNSUPPORTED, "restricted visibility needs the full or the packed sequence length");
   cudaError_t e;
   if (c->d.dtype == SWAM_F32) {
     e = launch_attn_f32(a, st, &c->launches_i);
@@ -118,6 +143,7 @@ int swam_create(const swam_shape* s, swam_ctx** out_ctx) {
   swam_ctx* c = new (std::nothrow) swam_ctx();
   if (!c) return SWAM_ERR_INVALID_ARG;
   memset(c, 0, sizeof(*c));
+  c->sees[0] = c->sees[1] = c->sees[2] = SWAM_SEES_ALL;
   Dims& d = c->d;
   d.B = s->batch; d.n_obs = s->n_obs; d.F = s->n_frames; d.N_s = s->n_spatial; d.H = s->n_action;
   d.N_h = s->n_heads; d.N_kv = s->n_kv_heads > 0 ? s->n_kv_heads : s->n_heads; d.D = s->head_dim; d.Kc = s->k_core; d.Ks = s->k_anchor; d.K = d.Kc + d.Ks;
@@ -230,7 +256,7 @@ int swam_score(swam_ctx* c, const void* q, const void* k, const float* lse_actio
   if (!lse) {
     if (int r = need_ws(c)) return r;
     float* own = (float*)(c->ws + c->off_lse);
-    cudaError_t e = launch_action_lse(c->d, q, k, own, c->ws + c->off_scratch, st, &c->launches_i);
+    cudaError_t e = launch_action_lse(c->d, q, k, own, c->ws + c->off_scratch, st, &c->launches_i, action_keys(c));
     count(c);
     if (e != cudaSuccess) return fail_cuda(c, e, "action lse launch");
     lse = own;
@@ -261,7 +287,7 @@ int swam_score_noalloc(swam_ctx* c, const void* q, const void* k, float* scores,
   if (e != cudaSuccess) return fail_cuda(c, e, "swam_score_noalloc: cudaGetSymbolAddress");
   cudaStream_t st = (cudaStream_t)stream;
   // every normaliser and every partial is written before it is read, so nothing has to start at zero
-  e = launch_action_lse(c->d, q, k, lse, partial, st, &c->launches_i);
+  e = launch_action_lse(c->d, q, k, lse, partial, st, &c->launches_i, action_keys(c));
   count(c);
   if (e != cudaSuccess) return fail_cuda(c, e, "action lse launch");
   e = launch_score(c->d, c->alpha, q, k, lse, scores, st, &c->launches_i);
@@ -384,6 +410,7 @@ int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t 
     void* vp = c->ws + c->off_vp;
     if (int r = swam_pack(c, nullptr, k, v, pm, nullptr, kp, vp, stream)) return r;
     AttnArgs a{q, kp, vp, out, nullptr, 0, 0, d.B, d.Lp, d.N_h, d.D, d.scale, d.N_kv};
+    set_visibility(c, a);
     cudaError_t e = launch_attn_bf16_tc_gather(a, pm, d.L, (int*)(c->ws + c->off_status), c->ws + c->off_attn,
                                                c->attn_scratch, st, &c->launches_i);
     count(c);
@@ -524,6 +551,15 @@ int swam_set_option(swam_ctx* c, int32_t option, int32_t value) {
   if (!c) return SWAM_ERR_INVALID_ARG;
   if (option == SWAM_OPT_ATTN_VARIANT && (value == SWAM_ATTN_AUTO || value == SWAM_ATTN_WARP_MMA)) {
     c->attn_variant = value;
+    return SWAM_OK;
+  }
+  if (option == SWAM_OPT_VISIBILITY) {
+    const int o = value & 3, f = (value >> 2) & 3, a = (value >> 4) & 3;
+    if ((value >> 6) != 0 || o > SWAM_SEES_ALL || f > SWAM_SEES_ALL || a > SWAM_SEES_ALL)
+      return fail(c, SWAM_ERR_INVALID_ARG, "swam_set_option: malformed visibility value");
+    if (f < SWAM_SEES_FUTURE || a < SWAM_SEES_FUTURE)
+      return fail(c, SWAM_ERR_INVALID_ARG, "swam_set_option: future and action rows must see the future tokens");
+    c->sees[0] = o; c->sees[1] = f; c->sees[2] = a;
     return SWAM_OK;
   }
   if (option == SWAM_OPT_SPARSE_PATH && (value == SWAM_SPARSE_FUSED || value == SWAM_SPARSE_STAGED)) {

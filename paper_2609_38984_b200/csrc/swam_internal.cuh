@@ -78,8 +78,9 @@ cudaError_t launch_score(const Dims& d, const Alpha& alpha, const void* q, const
 cudaError_t launch_quality(const Dims& d, const float* scores, float* quality, cudaStream_t st, int* launches);
 // lambda[b,h,i] = log sum over all L keys of exp(scale q_i.k_c); partial: scratch of lse_scratch_bytes().
 size_t lse_scratch_bytes(const Dims& d);
+// n_keys: the leading keys of the sequence that the action rows see (d.L = all of them)
 cudaError_t launch_action_lse(const Dims& d, const void* q, const void* k, float* lse, void* scratch,
-                              cudaStream_t st, int* launches);
+                              cudaStream_t st, int* launches, int n_keys);
 
 // static device scratch of the allocation-free scoring entry point
 constexpr size_t kStaticScratchBytes = 8u << 20;
@@ -122,6 +123,18 @@ struct AttnArgs {
   int B, n, N_h, D;  // n = sequence length of this call
   float scale;
   int N_kv;          // heads of k and v (q and out have N_h); query head h reads head h / (N_h / N_kv)
+  // Segment-prefix visibility: rows [0, obs_end) see the first lim[0] keys, rows [obs_end, fut_end) the first lim[1],
+  // the rest the first lim[2].  Full visibility: every lim = n (then obs_end and fut_end do not matter).
+  int obs_end, fut_end, lim[3];
+  __host__ __device__ bool full_visibility() const { return lim[0] >= n && lim[1] >= n && lim[2] >= n; }
+  __host__ __device__ int row_limit(int row) const { return row < obs_end ? lim[0] : (row < fut_end ? lim[1] : lim[2]); }
+  // the largest limit among rows [r0, r1) (r1 > r0)
+  __host__ __device__ int max_limit(int r0, int r1) const {
+    int m = row_limit(r0);
+    if (r1 - 1 >= obs_end && r0 < fut_end) m = m > lim[1] ? m : lim[1];
+    if (r1 - 1 >= fut_end) m = m > lim[2] ? m : lim[2];
+    return m;
+  }
 };
 cudaError_t attn_prepare(int D, int dtype);
 cudaError_t launch_attn_f32(const AttnArgs& a, cudaStream_t st, int* launches);

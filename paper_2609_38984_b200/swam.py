@@ -20,7 +20,8 @@ LIB_PATH = os.path.join(_HERE, "libswam.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_STATE, ERR_CUDA, ERR_DEVICE_CHECK, ERR_TIMEOUT = range(8)
 F32, BF16 = 0, 1
 REUSE, REFRESH_FULL, REFRESH_LIGHT = 0, 1, 2
-OPT_ATTN_VARIANT, OPT_SPARSE_PATH = 1, 2
+OPT_ATTN_VARIANT, OPT_SPARSE_PATH, OPT_VISIBILITY = 1, 2, 3
+SEES_OBSERVED, SEES_FUTURE, SEES_ALL = 0, 1, 2
 ATTN_AUTO, ATTN_WARP_MMA = 0, 1
 SPARSE_FUSED, SPARSE_STAGED = 0, 1
 
@@ -316,6 +317,10 @@ class Swam:
 
     def set_option(self, option: int, value: int):
         self._chk(self.lib.swam_set_option(self.ctx, option, value))
+
+    def set_visibility(self, observed_rows_see: int, future_rows_see: int, action_rows_see: int):
+        """Segment-prefix visibility: what the rows of each segment see (SEES_OBSERVED / SEES_FUTURE / SEES_ALL)."""
+        self.set_option(OPT_VISIBILITY, observed_rows_see | (future_rows_see << 2) | (action_rows_see << 4))
 
     def launch_count(self) -> int:
         n = ctypes.c_int64()

@@ -636,6 +636,80 @@ def test_step_leaves_the_layer_quality_of_its_scores(wl):
         assert np.abs(qual.cpu().numpy() - want).max() <= 1e-5 * max(1.0, np.abs(want).max())
 
 
+# ------------------------------------------------------------------ visibility constraints (segment prefixes)
+VIS_CASES = [
+    ("tiny", dict()),                                                                           # fp32 kernels
+    ("single_view", dict(n_obs=9, grid_h=6, grid_w=6, n_heads=2, head_dim=32)),                  # mma.sync kernel
+    ("single_view", dict(n_obs=200, grid_h=10, grid_w=9, n_heads=3)),                            # tcgen05, D = 64
+    ("larger_imagination", dict(n_obs=300, grid_h=7, grid_w=9, n_heads=2, batch=2)),             # tcgen05, D = 128
+]
+VIS_SETTINGS = [(0, 1, 2), (0, 2, 2), (2, 1, 1), (1, 1, 2)]   # what observed / future / action rows see
+
+
+@pytest.mark.parametrize("name,kw", VIS_CASES, ids=["f32", "d32", "d64", "d128"])
+@pytest.mark.parametrize("sees", VIS_SETTINGS, ids=["causal", "obs_isolated", "no_action_keys", "obs_sees_future"])
+def test_attention_with_segment_visibility(name, kw, sees):
+    swam = _swam()
+    wl = W.WORKLOADS[name].with_(**kw)
+    x = W.generate_steps(wl, 1)[0]
+    ctx = swam.Swam.from_workload(wl)
+    ctx.set_visibility(*sees)
+    q, k, v = (dev(x[n], wl) for n in "qkv")
+    out, lse = ctx.sparse_attn(q, k, v, want_lse=True)
+    ctx.check()
+    fut_end = wl.n_obs + wl.n_frames * wl.n_spatial
+    want, wlse = ora.attention(x["q"], x["k"], x["v"], visibility=(wl.n_obs, fut_end, sees))
+    check_float(f64(out), want, wl.dtype)
+    assert np.abs(lse.cpu().numpy() - wlse).max() <= (1e-4 if wl.dtype == W.F32 else 2e-3)
+    # the normalisers the scorer computes run over the keys the action rows see
+    got = ctx.score(q, k).cpu().numpy()
+    s64 = ora.score(x["q"], x["k"], wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action,
+                    lse=ora.action_lse(x["q"], x["k"], wl.n_action, n_visible=[wl.n_obs, fut_end, wl.seq_len][sees[2]]))
+    rel = np.abs(got - s64) / np.maximum(s64, 1e-30)
+    assert rel.max() <= 5e-5, rel.max()
+    # a length that is neither the full nor the packed sequence has no segment boundaries
+    with pytest.raises(swam.SwamError) as e:
+        ctx.sparse_attn(q[:, :wl.seq_len - 1].contiguous(), k[:, :wl.seq_len - 1].contiguous(), v[:, :wl.seq_len - 1].contiguous())
+    assert e.value.code == swam.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("wl", [
+    W.WORKLOADS["tiny"],
+    small(batch=2),
+    small("larger_imagination", n_obs=140, grid_h=7, grid_w=9, n_heads=2, steps=3),
+], ids=["f32", "d64", "d128"])
+@pytest.mark.parametrize("sees", [(0, 1, 2), (2, 1, 1)], ids=["causal", "no_action_keys"])
+def test_schedule_with_segment_visibility(wl, sees):
+    """Full and sparse steps under restricted visibility: the packed sequence has its own segment boundaries."""
+    swam = _swam()
+    steps = W.generate_steps(wl)
+    kc, ks = wl.budgets
+    want = ora.run_steps(steps, wl.refresh, wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, kc, ks, sees=sees)
+    outs = []
+    for path in (swam.SPARSE_FUSED, swam.SPARSE_STAGED):
+        ctx = swam.Swam.from_workload(wl)
+        ctx.set_visibility(*sees)
+        ctx.set_option(swam.OPT_SPARSE_PATH, path)
+        log = run_schedule(ctx, wl, steps, wl.refresh)
+        for t, (g, w) in enumerate(zip(log, want)):
+            rel = np.abs(g["scores"] - w["scores"].astype(np.float64)) / np.maximum(w["scores"], 1e-30)
+            assert rel.max() <= SCORE_REL, (t, rel.max())
+            assert np.array_equal(g["sel"], w["sel_idx"]), (t, w["margins"])
+            check_float(g["out"], w["out"], wl.dtype)
+        outs.append(log[-1]["out"])
+    assert np.array_equal(outs[0], outs[1])
+
+
+def test_visibility_option_validation():
+    swam = _swam()
+    ctx = swam.Swam.from_workload(W.WORKLOADS["tiny"])
+    for bad in ((0, 0, 2), (2, 2, 0), (3, 2, 2)):
+        with pytest.raises(swam.SwamError) as e:
+            ctx.set_visibility(*bad)
+        assert e.value.code == swam.ERR_INVALID_ARG
+    ctx.set_visibility(2, 2, 2)
+
+
 def test_reuse_before_refresh_is_a_state_error():
     swam = _swam()
     wl = W.WORKLOADS["tiny"]
