@@ -8,9 +8,14 @@
 //   warps 0-3   softmax of query tile 0: one thread per row reads its S row from TMEM, keeps the reference maximum
 //   warps 4-7   and the running sum (exp2 domain), writes P as bf16 back over S; same for query tile 1
 //   warps 10-11 idle (they complete the third warpgroup, which hands most of its registers to the softmax warps)
-// Work is a sequence of items (key tile, query tile); item i uses score buffer i mod NB (NB = 2 at head dim 128,
-// 3 at head dim 64) and the issuing thread keeps Q K^T NB items ahead of P V, so one tile's exponentials overlap the
-// other tile's MMAs.  O stays in TMEM for the whole key loop; it is rescaled only when a row's maximum has grown by
+// Head dim 64: work is a sequence of items (key tile, query tile); item i uses score buffer i mod 3 and the issuing
+// thread keeps Q K^T three items ahead of P V, so one tile's exponentials overlap the other tile's MMAs.
+// Head dim 128: TMEM (512 columns) holds only two score buffers beside the two outputs, so P does not go back over
+// the scores: each softmax thread stores its bf16 P row into a shared-memory tile laid out like a K-major operand
+// (both products then read both operands from shared memory) and releases its score buffer as soon as the scores are
+// in its registers.  Q K^T of key tile j+1 therefore never waits for P V of tile j; the tensor pipe runs
+// S(0) | S(1), PV(0) | S(2), PV(1) | ... with both query tiles side by side, and K and V tiles share one ring of three
+// shared-memory slots that is filled in exactly that order.  O stays in TMEM for the whole key loop; it is rescaled only when a row's maximum has grown by
 // more than 2^8 beyond the value its exponentials refer to (the result is exact either way: sums and outputs share
 // the same reference maximum).  Work items left over after the last full wave of CTAs are cut over the keys and
 // merged by a small combine kernel.  Every wait on an mbarrier is bounded; when a wait runs out the kernel raises
@@ -111,6 +116,18 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t 
       " mov.b64 da, {%1, %3};\n mov.b64 db, {%2, %3};\n"
       " @q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n}"
       ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "n"(kAccum ? 1 : 0), "r"(el) : "memory");
+}
+// the same with the accumulate flag as a run-time value
+__device__ __forceinline__ void mma_ss_rt(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                          uint32_t accum, uint32_t el) {
+  asm volatile(
+      "{\n .reg .pred p, q;\n .reg .b64 da, db;\n setp.ne.b32 p, %5, 0;\n setp.ne.b32 q, %6, 0;\n"
+      " mov.b64 da, {%1, %3};\n mov.b64 db, {%2, %3};\n"
+      " @q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accum), "r"(el) : "memory");
+}
+__device__ __forceinline__ void st_shared_16(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem desc]
 __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
@@ -263,14 +280,20 @@ struct TcCfg {
   static constexpr int DB = D / 64;                 // 64-column (128-byte) blocks per row
   static constexpr int kSubTile = kTile * 128;      // bytes of one [128 rows x 64 cols] block
   static constexpr int kTileBytes = DB * kSubTile;  // one 128 x D tile
-  static constexpr int kStages = (D == 128) ? 2 : 4;
+  // Head dim 128 keeps P in shared memory (see the kernel's header): its key and value tiles then share ONE ring of
+  // three slots, filled and consumed in the order K_0, K_1, V_0, K_2, V_1, ... in which the tensor pipe uses them, so
+  // that every load has a whole key-tile step to arrive.  Head dim 64 has a ring of kStages slots for K and one for V.
+  static constexpr bool kPSmem = (D == 128);
+  static constexpr int kStages = kPSmem ? 3 : 4;
+  static constexpr int kRingTiles = kPSmem ? kStages : 2 * kStages;
   // score buffers in TMEM: two at D = 128 (S0, S1, O0, O1 fill all 512 columns); at D = 64 the outputs need only 128
   // columns, which leaves room for a third score buffer and lets Q K^T run one tile further ahead of the softmax
   static constexpr int kSBufs = (D == 128) ? 2 : 3;
   // of every 8 element pairs of the softmax pass, this many take their exponential on the FMA pipes (measured: one
-  // in eight is the optimum at head dim 64, where the exp2 unit is 80 % busy; no gain at head dim 128)
-  static constexpr int kPolyOf8 = (D == 64) ? 1 : 0;
-  static constexpr int kSmemData = 2 * kTileBytes + 2 * kStages * kTileBytes;
+  // in eight is the optimum at both head dims; every further eighth costs more FMA-pipe time than it frees on the
+  // exp2 unit)
+  static constexpr int kPolyOf8 = 1;
+  static constexpr int kSmemData = (2 + (kPSmem ? 2 : 0) + kRingTiles) * kTileBytes;   // Q tiles, P tiles, ring(s)
   static constexpr int kSmemBytes = kSmemData + 1024 /*alignment slack*/ + 512 /*barriers*/;
   static constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
   static constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(D >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
@@ -298,9 +321,10 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const uint32_t base = (smem_addr(smem_raw) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_raw + (base - smem_addr(smem_raw));
   const uint32_t sQ = base;                                 // [2][tile]
-  const uint32_t sK = sQ + 2 * C::kTileBytes;               // [ST][tile]
-  const uint32_t sV = sK + ST * C::kTileBytes;              // [ST][tile]
-  const uint32_t bars = sV + ST * C::kTileBytes;
+  const uint32_t sP = sQ + 2 * C::kTileBytes;               // [2][tile], only with P in shared memory
+  const uint32_t sK = sP + (C::kPSmem ? 2 * C::kTileBytes : 0);   // [ST][tile]; the one ring of both with P in shared memory
+  const uint32_t sV = C::kPSmem ? sK : sK + ST * C::kTileBytes;   // [ST][tile]
+  const uint32_t bars = base + C::kSmemData;
   // barrier slots (8 bytes each)
   const uint32_t bar_q = bars;
   auto bar_k_full = [&](int s) { return bars + 8 * (1 + s); };
@@ -318,8 +342,10 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   // queries may be loaded)
   const uint32_t bar_o_free = bars + 8 * (10 + 4 * ST);
   const uint32_t bar_q_free = bars + 8 * (11 + 4 * ST);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + C::kSmemData + 8 * (12 + 4 * ST));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::kSmemData + 8 * (12 + 4 * ST) + 8);
+  // P in shared memory: the softmax threads have read a score buffer into registers (the next Q K^T may overwrite it)
+  auto bar_s_free = [&](int s) { return bars + 8 * (12 + 4 * ST + s); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + C::kSmemData + 8 * (14 + 4 * ST));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::kSmemData + 8 * (14 + 4 * ST) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // Work item = (sample, head, query tile pair), pair fastest.  Items below n_whole walk over all keys; the few items
@@ -375,6 +401,8 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     }
     mbar_init(bar_pv_tile(0), 1);
     mbar_init(bar_pv_tile(1), 1);
+    mbar_init(bar_s_free(0), kTile);
+    mbar_init(bar_s_free(1), kTile);
     mbar_init(bar_o_final, 1);
     mbar_init(bar_o_free, 2 * kTile);
     mbar_init(bar_q_free, (MODE == kDirect) ? 2 : 2 * kTile);
@@ -490,6 +518,27 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
               tma_load_4d(sQ + s * C::kTileBytes + db * C::kSubTile, &map_q, bar_q, db * 64, wk.row0 + s * kTile, wk.h, wk.b);
           return true;
         };
+        if constexpr (C::kPSmem) {
+          // one ring: load m of an item is K_0 (m = 0), K_(m+1)/2 (odd m), V_(m/2-1) (even m), and V of the last tile
+          // at the end.  The ring's slots that a new item's first loads wait for are freed by the previous item, so
+          // those loads go out before the (possibly long) wait for the query tiles.
+          const int n_loads = 2 * wk.n_tiles;
+          const int q_after = (iter == 0) ? -1 : min(ST, n_loads) - 1;
+          if (q_after < 0) ok = load_q();
+          for (int m = 0; m < n_loads && ok; ++m, ++kt) {
+            const int st = kt % ST;
+            ok = mbar_wait(bar_k_empty(st), ((kt / ST) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            const bool is_v = (m == n_loads - 1) || (m > 0 && (m & 1) == 0);
+            const int j = (m == n_loads - 1) ? wk.n_tiles - 1 : (is_v ? m / 2 - 1 : (m + 1) / 2);
+            mbar_expect_tx(bar_k_full(st), C::kTileBytes);
+            for (int db = 0; db < C::DB; ++db)
+              tma_load_4d(sK + st * C::kTileBytes + db * C::kSubTile, is_v ? &map_v : &map_k, bar_k_full(st), db * 64,
+                          (wk.kv_begin + j) * kTile, h_kv, wk.b);
+            if (m == q_after) ok = load_q();
+          }
+          continue;
+        }
         const int q_after = (iter == 0) ? -1 : min(ST, wk.n_tiles) - 1;   // tile after which the queries are requested
         if (q_after < 0) ok = load_q();
         for (int j = 0; j < wk.n_tiles && ok; ++j, ++kt) {
@@ -532,6 +581,17 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           mma_ss<true>(d, a_lo + off, b_lo + off, kDescHi, C::kIdescQK, el);
         }
       };
+      // the same product with P as a K-major operand in shared memory (laid out like a query tile)
+      auto issue_pv_ss = [&](int s, int st, bool accum) {
+        const uint32_t a_lo = desc_lo(sP, 16) + ((uint32_t)(s * C::kTileBytes) >> 4), b_lo = v_lo0 + ((uint32_t)(st * C::kTileBytes) >> 4);
+        const uint32_t d = tm_O(s);
+        mma_ss_rt(d, a_lo, b_lo, kDescHi, C::kIdescPV, accum ? 1u : 0u, el);
+#pragma unroll
+        for (int kk = 1; kk < kTile / 16; ++kk) {
+          constexpr int kSub16 = C::kSubTile >> 4;
+          mma_ss_rt(d, a_lo + (uint32_t)((kk >> 2) * kSub16 + (kk & 3) * 2), b_lo + kk * (2048 >> 4), kDescHi, C::kIdescPV, 1u, el);
+        }
+      };
       auto issue_pv = [&](int s, int buf, int st, bool accum) {
         // O_s += P V : K dimension = 128 keys, 16 keys (two 8-row groups) per instruction; V is MN-major
         const uint32_t b_lo = v_lo0 + ((uint32_t)(st * C::kTileBytes) >> 4);
@@ -554,6 +614,55 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         ok = wait_all(bar_q, iter & 1);
         if (!ok) break;
         if (MODE == kGather) fence_proxy_async();
+        if constexpr (C::kPSmem) {
+          // Order on the tensor pipe: S(0) | S(1), O += P(0) V(0) | S(2), O += P(1) V(1) | ... with both query tiles
+          // side by side in every group.  Score buffer s belongs to query tile s; it is free again as soon as the
+          // softmax threads hold its values in registers, long before their P is ready, so S(j+1) never waits for
+          // the product of tile j.  kt0 counts the key tiles of finished items, it0 the ring loads consumed.
+          auto qk_pair = [&](int j) -> bool {
+            const int st = it0 % ST, g = kt0 + j;
+            if (iter == 0) TRACE(2, j * 8 + 0);
+            if (!wait_all(bar_k_full(st), (it0 / ST) & 1)) return false;
+            if (iter == 0) TRACE(2, j * 8 + 1);
+            for (int sq = 0; sq < 2; ++sq) {
+              if (g > 0 && !wait_all(bar_s_free(sq), (g - 1) & 1)) return false;
+              if (iter == 0) TRACE(2, j * 8 + 2 + sq);
+              tc_fence_after();
+              issue_qk(sq, sq, st);
+              tc_commit(bar_s_full(sq), el);
+            }
+            tc_commit(bar_k_empty(st), el);
+            ++it0;
+            return true;
+          };
+          auto pv_pair = [&](int j) -> bool {
+            const int st = it0 % ST, g = kt0 + j;
+            if (iter == 0) TRACE(2, j * 8 + 4);
+            if (!wait_all(bar_k_full(st), (it0 / ST) & 1)) return false;
+            if (iter == 0) TRACE(2, j * 8 + 5);
+            // the first product of an item overwrites the output accumulators: the previous item's epilogue must
+            // have read them
+            if (j == 0 && iter > 0 && !wait_all(bar_o_free, (iter - 1) & 1)) return false;
+            for (int sq = 0; sq < 2; ++sq) {
+              if (!wait_all(bar_p_full(sq), g & 1)) return false;
+              if (iter == 0) TRACE(2, j * 8 + 6 + sq);
+              tc_fence_after();
+              issue_pv_ss(sq, st, j > 0);
+              tc_commit(bar_pv_tile(sq), el);
+            }
+            tc_commit(bar_k_empty(st), el);
+            ++it0;
+            return true;
+          };
+          ok = qk_pair(0);
+          for (int j = 0; j < wk.n_tiles && ok; ++j) {
+            if (j + 1 < wk.n_tiles) ok = qk_pair(j + 1);
+            if (ok) ok = pv_pair(j);
+          }
+          if (ok) tc_commit(bar_o_final, el);
+          kt0 += wk.n_tiles;
+          continue;
+        }
         const int n_items = 2 * wk.n_tiles;
         int k_waited = 0, v_waited = 0;
         auto qk_item = [&](int it) -> bool {
@@ -614,21 +723,42 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const int h = wk.h, b = wk.b, row0 = wk.row0, kv_begin = wk.kv_begin, n_tiles = wk.n_tiles, slot = wk.slot;
     float m_used = -INFINITY, l_run = 0.f;
     const int row_keys = VIS ? row_limit(row0 + s * kTile + r) : p.n;   // leading keys of the sequence this row sees
+    // 32 packed bf16 pairs of this row's P, part c of four: over the scores in TMEM, or into the row's place in the
+    // shared-memory P tile (the swizzled layout of a K-major operand)
+    const uint32_t p_row = sP + (uint32_t)(s * C::kTileBytes + r * 128);
+    auto store_p16 = [&](uint32_t tS, int c, const uint32_t* v) {
+      if constexpr (C::kPSmem) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int c16 = c * 4 + q;   // 16-byte chunk of the row: 64-key block c16 / 8, chunk c16 % 8
+          st_shared_16(p_row + (uint32_t)((c16 >> 3) * C::kSubTile + (((c16 & 7) ^ (r & 7)) << 4)), v[4 * q], v[4 * q + 1],
+                       v[4 * q + 2], v[4 * q + 3]);
+        }
+      } else {
+        tmem_st16(tS + c * 16, v);
+      }
+    };
     for (int j = 0; j < n_tiles; ++j) {
-      const int item = it0 + 2 * j + s, buf = item % NB;
+      // P in shared memory: tile s owns score buffer s and phases count key tiles; otherwise items share NB buffers
+      const int item = C::kPSmem ? kt0 + j : it0 + 2 * j + s, buf = C::kPSmem ? s : item % NB;
+      const uint32_t s_par = C::kPSmem ? (item & 1) : ((item / NB) & 1);
       const uint32_t tS = tm_S(buf) + lane_off;
-      if (r == 0 && iter == 0) TRACE(s, j * 8 + 0);
-      ok = mbar_wait(bar_s_full(buf), (item / NB) & 1, abort_flag);
+      if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 0);
+      ok = mbar_wait(bar_s_full(buf), s_par, abort_flag);
       if (!ok) break;
-      if (r == 0 && iter == 0) TRACE(s, j * 8 + 1);
+      if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 1);
       if (r == 0 && s == 0 && j == 0 && iter == 0) CTA_T(1);
       tc_fence_after();
       float sv[kTile];
+      const int valid = row_keys - (kv_begin + j) * kTile;  // keys of this tile that this row sees (<= 0: none)
 #pragma unroll
       for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<float(*)[32]>(&sv[c * 32]));
       tmem_ld_wait();
-      if (r == 0 && iter == 0) TRACE(s, j * 8 + 2);
-      const int valid = row_keys - (kv_begin + j) * kTile;  // keys of this tile that this row sees (<= 0: none)
+      if constexpr (C::kPSmem) {
+        tc_fence_before();
+        mbar_arrive(bar_s_free(s));   // the scores are in registers: the next key tile's may be written
+      }
+      if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 2);
       if (valid < kTile) {
 #pragma unroll
         for (int c = 0; c < kTile; ++c)
@@ -654,26 +784,42 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       // (an exponent above the threshold pushes the sum beyond 2^threshold), so no per-element maximum is kept
       const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), negm2 = pack2(-m_used, -m_used);
       uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};
-      // all 64 packed results first, the four stores after: the exp2 unit then sees one uninterrupted stream of 128
-      // instructions per thread instead of four short ones with their fill and drain
+      // P over the scores in TMEM: all 64 packed results first, the four stores after (the exp2 unit then sees one
+      // uninterrupted stream of 128 instructions per thread instead of four short ones with their fill and drain)
       uint32_t pk[64];
-#pragma unroll
-      for (int i = 0; i < 64; ++i) {
-        const uint64_t x2 = fma2(pack2(sv[2 * i], sv[2 * i + 1]), scale2, negm2);
-        float p0, p1;
-        if ((i & 7) < C::kPolyOf8) {
-          exp2_poly2(x2, p0, p1);
-        } else {
-          float t0, t1;
-          unpack2(x2, t0, t1);
-          p0 = ex2(t0);
-          p1 = ex2(t1);
+      if constexpr (C::kPSmem) {
+        // the P tile is free once the previous product of this query tile has read it (usually long ago)
+        if (item > 0) {
+          ok = mbar_wait(bar_pv_tile(s), (item - 1) & 1, abort_flag);
+          if (!ok) break;
         }
-        acc2[i & 3] = add2(acc2[i & 3], pack2(p0, p1));
-        pk[i] = pack_bf16x2(p0, p1);
       }
 #pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_st16(tS + c * 16, &pk[c * 16]);
+      for (int i = 0; i < 64; ++i) {
+        float p0, p1;
+        if ((i & 7) < C::kPolyOf8) {
+          exp2_poly2(fma2(pack2(sv[2 * i], sv[2 * i + 1]), scale2, negm2), p0, p1);
+          acc2[i & 3] = add2(acc2[i & 3], pack2(p0, p1));
+        } else {
+          float t0, t1;
+          unpack2(fma2(pack2(sv[2 * i], sv[2 * i + 1]), scale2, negm2), t0, t1);
+          p0 = ex2(t0);
+          p1 = ex2(t1);
+          acc2[i & 3] = add2(acc2[i & 3], pack2(p0, p1));
+        }
+        pk[i] = pack_bf16x2(p0, p1);
+        // shared-memory stores drain while the exponentials go on; the TMEM stores of the other variant wait until
+        // all 128 exponentials have been issued
+        if constexpr (C::kPSmem) {
+          if ((i & 15) == 15) store_p16(tS, i >> 4, &pk[i - 15]);
+        }
+      }
+      if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 5);
+      if constexpr (!C::kPSmem) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) store_p16(tS, c, &pk[c * 16]);
+      }
+      if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 7);
       float sum;
       {
         float a0, a1;
@@ -720,15 +866,16 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             sum += p0 + p1;
             pk[i] = pack_bf16x2(p0, p1);
           }
-          tmem_st16(tS + c * 16, pk);
+          store_p16(tS, c, pk);
         }
       }
       l_run += sum;
-      if (r == 0 && iter == 0) TRACE(s, j * 8 + 3);
+      if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 3);
       tmem_st_wait();
       tc_fence_before();
+      if constexpr (C::kPSmem) fence_proxy_async();   // P was written through the generic proxy; the tensor core reads it through the async one
       mbar_arrive(bar_p_full(buf));
-      if (r == 0 && iter == 0) TRACE(s, j * 8 + 4);
+      if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 4);
     }
     // epilogue
     if (ok) ok = mbar_wait(bar_o_final, iter & 1, abort_flag);
