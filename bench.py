@@ -35,7 +35,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel's launches in one cycle (dense launch + packed
 # launch), from the ncu captures summarised in profiles/attn_bf16_tc_*.txt
 DOMINANT_KERNEL_DRAM_BYTES = {
-    "larger_imagination": int((228.192768 + 55.545344 + 87.191808 + 10.293248) * 1e6),
+    "larger_imagination": int((228.190464 + 57.358848 + 87.189248 + 10.544896) * 1e6),
     "multi_view": int((639.990784 + 198.666496 + 257.344768 + 72.386048) * 1e6),   # profiles/attn_bf16_tc_multi_view.txt
 }
 
