@@ -291,13 +291,19 @@ def test_attention_work_distribution_over_persistent_ctas(head_dim, n_heads, n):
     assert torch.equal(out, tc.sparse_attn(q, k, v))          # and the same bits again
 
 
-def test_attention_short_sequences():
+@pytest.mark.parametrize("name,lengths", [
+    ("single_view", (1, 2, 63, 64, 65, 127, 129, 200)),
+    # head dim 128: one to five key tiles, i.e. every start-up sequence of the ring that K and V tiles share there
+    ("larger_imagination", (1, 127, 128, 129, 256, 257, 384, 385, 513, 600)),
+], ids=["d64", "d128"])
+def test_attention_short_sequences(name, lengths):
     """seq_len below the full length, down to one token."""
     swam = _swam()
-    wl = small()
+    wl = small(name, n_obs=160, grid_h=10, grid_w=9, n_heads=3) if name != "single_view" else small()
     x = W.generate_steps(wl, 1)[0]
     ctx = swam.Swam.from_workload(wl)
-    for n in (1, 2, 63, 64, 65, 127, 129, 200):
+    assert max(lengths) <= wl.seq_len
+    for n in lengths:
         q, k, v = (dev(np.ascontiguousarray(x[m][:, :n]), wl) for m in "qkv")
         out = ctx.sparse_attn(q, k, v)
         want, _ = ora.attention(x["q"][:, :n], x["k"][:, :n], x["v"][:, :n])
