@@ -283,7 +283,10 @@ struct TcCfg {
   // Head dim 128 keeps P in shared memory (see the kernel's header): its key and value tiles then share ONE ring of
   // three slots, filled and consumed in the order K_0, K_1, V_0, K_2, V_1, ... in which the tensor pipe uses them, so
   // that every load has a whole key-tile step to arrive.  Head dim 64 has a ring of kStages slots for K and one for V.
+  // (head dim 64 keeps P in TMEM: its three score buffers already let Q K^T run ahead, and with P in shared memory
+  // the same launch was 7 % slower)
   static constexpr bool kPSmem = (D == 128);
+  static constexpr int kPTileBytes = 2 * kSubTile;   // a 128 x 128 bf16 P tile: two 64-key blocks
   static constexpr int kStages = kPSmem ? 3 : 4;
   static constexpr int kRingTiles = kPSmem ? kStages : 2 * kStages;
   // score buffers in TMEM: two at D = 128 (S0, S1, O0, O1 fill all 512 columns); at D = 64 the outputs need only 128
@@ -293,7 +296,7 @@ struct TcCfg {
   // in eight is the optimum at both head dims; every further eighth costs more FMA-pipe time than it frees on the
   // exp2 unit)
   static constexpr int kPolyOf8 = 1;
-  static constexpr int kSmemData = (2 + (kPSmem ? 2 : 0) + kRingTiles) * kTileBytes;   // Q tiles, P tiles, ring(s)
+  static constexpr int kSmemData = (2 + kRingTiles) * kTileBytes + (kPSmem ? 2 * kPTileBytes : 0);   // Q tiles, ring(s), P tiles
   static constexpr int kSmemBytes = kSmemData + 1024 /*alignment slack*/ + 512 /*barriers*/;
   static constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
   static constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(D >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
@@ -322,7 +325,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   unsigned char* base_ptr = smem_raw + (base - smem_addr(smem_raw));
   const uint32_t sQ = base;                                 // [2][tile]
   const uint32_t sP = sQ + 2 * C::kTileBytes;               // [2][tile], only with P in shared memory
-  const uint32_t sK = sP + (C::kPSmem ? 2 * C::kTileBytes : 0);   // [ST][tile]; the one ring of both with P in shared memory
+  const uint32_t sK = sP + (C::kPSmem ? 2 * C::kPTileBytes : 0);   // [ST][tile]; the one ring of both with P in shared memory
   const uint32_t sV = C::kPSmem ? sK : sK + ST * C::kTileBytes;   // [ST][tile]
   const uint32_t bars = base + C::kSmemData;
   // barrier slots (8 bytes each)
@@ -583,7 +586,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       };
       // the same product with P as a K-major operand in shared memory (laid out like a query tile)
       auto issue_pv_ss = [&](int s, int st, bool accum) {
-        const uint32_t a_lo = desc_lo(sP, 16) + ((uint32_t)(s * C::kTileBytes) >> 4), b_lo = v_lo0 + ((uint32_t)(st * C::kTileBytes) >> 4);
+        const uint32_t a_lo = desc_lo(sP, 16) + ((uint32_t)(s * C::kPTileBytes) >> 4), b_lo = v_lo0 + ((uint32_t)(st * C::kTileBytes) >> 4);
         const uint32_t d = tm_O(s);
         mma_ss_rt(d, a_lo, b_lo, kDescHi, C::kIdescPV, accum ? 1u : 0u, el);
 #pragma unroll
@@ -725,7 +728,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const int row_keys = VIS ? row_limit(row0 + s * kTile + r) : p.n;   // leading keys of the sequence this row sees
     // 32 packed bf16 pairs of this row's P, part c of four: over the scores in TMEM, or into the row's place in the
     // shared-memory P tile (the swizzled layout of a K-major operand)
-    const uint32_t p_row = sP + (uint32_t)(s * C::kTileBytes + r * 128);
+    const uint32_t p_row = sP + (uint32_t)(s * C::kPTileBytes + r * 128);
     auto store_p16 = [&](uint32_t tS, int c, const uint32_t* v) {
       if constexpr (C::kPSmem) {
 #pragma unroll
