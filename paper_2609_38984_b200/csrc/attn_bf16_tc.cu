@@ -753,7 +753,6 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       if (r == 0 && s == 0 && j == 0 && iter == 0) CTA_T(1);
       tc_fence_after();
       float sv[kTile];
-      const int valid = row_keys - (kv_begin + j) * kTile;  // keys of this tile that this row sees (<= 0: none)
 #pragma unroll
       for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<float(*)[32]>(&sv[c * 32]));
       tmem_ld_wait();
@@ -762,6 +761,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         mbar_arrive(bar_s_free(s));   // the scores are in registers: the next key tile's may be written
       }
       if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 2);
+      const int valid = row_keys - (kv_begin + j) * kTile;  // keys of this tile that this row sees (<= 0: none)
       if (valid < kTile) {
 #pragma unroll
         for (int c = 0; c < kTile; ++c)
@@ -799,17 +799,17 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       }
 #pragma unroll
       for (int i = 0; i < 64; ++i) {
+        const uint64_t x2 = fma2(pack2(sv[2 * i], sv[2 * i + 1]), scale2, negm2);
         float p0, p1;
         if ((i & 7) < C::kPolyOf8) {
-          exp2_poly2(fma2(pack2(sv[2 * i], sv[2 * i + 1]), scale2, negm2), p0, p1);
-          acc2[i & 3] = add2(acc2[i & 3], pack2(p0, p1));
+          exp2_poly2(x2, p0, p1);
         } else {
           float t0, t1;
-          unpack2(fma2(pack2(sv[2 * i], sv[2 * i + 1]), scale2, negm2), t0, t1);
+          unpack2(x2, t0, t1);
           p0 = ex2(t0);
           p1 = ex2(t1);
-          acc2[i & 3] = add2(acc2[i & 3], pack2(p0, p1));
         }
+        acc2[i & 3] = add2(acc2[i & 3], pack2(p0, p1));
         pk[i] = pack_bf16x2(p0, p1);
         // shared-memory stores drain while the exponentials go on; the TMEM stores of the other variant wait until
         // all 128 exponentials have been issued
