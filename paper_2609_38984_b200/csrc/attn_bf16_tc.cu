@@ -296,7 +296,14 @@ struct TcCfg {
   // in eight is the optimum at both head dims; every further eighth costs more FMA-pipe time than it frees on the
   // exp2 unit)
   static constexpr int kPolyOf8 = 1;
-  static constexpr int kSmemData = (2 + kRingTiles) * kTileBytes + (kPSmem ? 2 * kPTileBytes : 0);   // Q tiles, ring(s), P tiles
+  // The epilogue stages a query tile's bf16 output in shared memory for the TMA store.  Head dim 64 has room for two
+  // staging tiles of their own: the query tiles are then free as soon as the item's last Q K^T has run, and the next
+  // item's queries load (and its first Q K^T run) under the current item's tail (3 % on the multi-view launches).
+  // Head dim 128 has no room left and stages in the finished query tiles (staging in the P tiles instead, which are
+  // also free by then, was 1 % slower: the next item's first P stores then wait for the copy engine).
+  static constexpr bool kStageOwn = !kPSmem;
+  static constexpr int kStageBytes = kStageOwn ? 2 * kTileBytes : 0;
+  static constexpr int kSmemData = (2 + kRingTiles) * kTileBytes + (kPSmem ? 2 * kPTileBytes : 0) + kStageBytes;   // Q tiles, ring(s), P tiles, staging
   static constexpr int kSmemBytes = kSmemData + 1024 /*alignment slack*/ + 512 /*barriers*/;
   static constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
   static constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(D >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
@@ -327,6 +334,8 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const uint32_t sP = sQ + 2 * C::kTileBytes;               // [2][tile], only with P in shared memory
   const uint32_t sK = sP + (C::kPSmem ? 2 * C::kPTileBytes : 0);   // [ST][tile]; the one ring of both with P in shared memory
   const uint32_t sV = C::kPSmem ? sK : sK + ST * C::kTileBytes;   // [ST][tile]
+  const uint32_t sStage = C::kStageOwn ? sV + ST * C::kTileBytes : sQ;   // [2] output staging tiles
+  constexpr uint32_t kStageStride = C::kTileBytes;
   const uint32_t bars = base + C::kSmemData;
   // barrier slots (8 bytes each)
   const uint32_t bar_q = bars;
@@ -341,14 +350,16 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   // P V of a query tile's item has completed: that tile's output accumulator is up to date
   auto bar_pv_tile = [&](int s) { return bars + 8 * (8 + 4 * ST + s); };
   // a CTA works through several items: the output accumulators have been read (the next item's first P V may
-  // overwrite them), and the output staging in the query tiles has been read by the copy engine (the next item's
-  // queries may be loaded)
+  // overwrite them), and the query tiles are free (the next item's queries may be loaded): with staging tiles of
+  // their own, when the item's last Q K^T has run; otherwise when the copy engine has read the output staged in them
   const uint32_t bar_o_free = bars + 8 * (10 + 4 * ST);
   const uint32_t bar_q_free = bars + 8 * (11 + 4 * ST);
   // P in shared memory: the softmax threads have read a score buffer into registers (the next Q K^T may overwrite it)
   auto bar_s_free = [&](int s) { return bars + 8 * (12 + 4 * ST + s); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + C::kSmemData + 8 * (14 + 4 * ST));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::kSmemData + 8 * (14 + 4 * ST) + 8);
+  // direct mode: the copy engine has read query tile s's staged output (its threads may write that memory again)
+  auto bar_stage_free = [&](int s) { return bars + 8 * (14 + 4 * ST + s); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + C::kSmemData + 8 * (16 + 4 * ST));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::kSmemData + 8 * (16 + 4 * ST) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // Work item = (sample, head, query tile pair), pair fastest.  Items below n_whole walk over all keys; the few items
@@ -408,7 +419,9 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     mbar_init(bar_s_free(1), kTile);
     mbar_init(bar_o_final, 1);
     mbar_init(bar_o_free, 2 * kTile);
-    mbar_init(bar_q_free, (MODE == kDirect) ? 2 : 2 * kTile);
+    mbar_init(bar_q_free, C::kStageOwn ? 1 : ((MODE == kDirect) ? 2 : 2 * kTile));
+    mbar_init(bar_stage_free(0), 1);
+    mbar_init(bar_stage_free(1), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -678,6 +691,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           issue_qk(sq, g % NB, st);
           tc_commit(bar_s_full(g % NB), el);
           if (sq == 1) tc_commit(bar_k_empty(st), el);   // both query tiles have used this key tile
+          if (C::kStageOwn && it == n_items - 1) tc_commit(bar_q_free, el);   // the query tiles have been read for the last time
           return true;
         };
         for (int it = 0; it < NB && it < n_items && ok; ++it) ok = qk_item(it);
@@ -901,15 +915,20 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         dst[D + 1] = l_run;
         tc_fence_before();
         mbar_arrive(bar_o_free);          // the accumulator row has been read
-        // nothing was staged in the query tiles: they are free as far as this thread is concerned
-        if (MODE != kDirect || ((warp & 3) == 0 && lane == 0)) mbar_arrive(bar_q_free);
+        // nothing was staged (the barriers' phases still count items)
+        if (C::kStageOwn) {
+          if (MODE == kDirect && (warp & 3) == 0 && lane == 0) mbar_arrive(bar_stage_free(s));
+        } else if (MODE != kDirect || ((warp & 3) == 0 && lane == 0)) {
+          mbar_arrive(bar_q_free);
+        }
       }
     } else {
-    // O / l -> bf16 -> swizzled staging in the (finished) Q tile -> TMA store; rows beyond n are clipped
+    // O / l -> bf16 -> swizzled staging tile -> TMA store; rows beyond n are clipped
+    if (ok && MODE == kDirect && C::kStageOwn && iter > 0) ok = mbar_wait(bar_stage_free(s), (iter - 1) & 1, abort_flag);
     if (ok) {
       tc_fence_after();
       const float inv = 1.f / l_run;
-      unsigned char* stage = base_ptr + s * C::kTileBytes;
+      unsigned char* stage = base_ptr + (sStage - base) + s * kStageStride;
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
         float ov[32];
@@ -943,22 +962,22 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const int orow = p.pack_map[(int64_t)b * p.n + prow];
         if (orow >= 0 && orow < p.n_full) {
           for (int db = 0; db < C::DB; ++db)
-            tma_store_4d(&map_o, sQ + s * C::kTileBytes + db * C::kSubTile + r * 128, db * 64, orow, h, b);
-          tma_store_commit_wait();
+            tma_store_4d(&map_o, sStage + s * kStageStride + db * C::kSubTile + r * 128, db * 64, orow, h, b);
+          tma_store_commit_wait();   // the thread's own staged row has been read before it writes there again
         } else {
           atomicOr(p.status, ST_BAD_MAP);
         }
       }
-      if (ok) mbar_arrive(bar_q_free);    // this thread's staged row has been read (or was never sent)
+      if (!C::kStageOwn && ok) mbar_arrive(bar_q_free);    // this thread's staged row has been read (or was never sent)
     } else {
       asm volatile("bar.sync %0, 128;" ::"r"(1 + s) : "memory");  // the four warps of this query tile
       if (ok && (warp & 3) == 0 && lane == 0) {
         if (row0 + s * kTile < p.n) {
           for (int db = 0; db < C::DB; ++db)
-            tma_store_4d(&map_o, sQ + s * C::kTileBytes + db * C::kSubTile, db * 64, row0 + s * kTile, h, b);
+            tma_store_4d(&map_o, sStage + s * kStageStride + db * C::kSubTile, db * 64, row0 + s * kTile, h, b);
           tma_store_commit_wait();
         }
-        mbar_arrive(bar_q_free);          // this tile's staging has been read (or was never sent)
+        mbar_arrive(C::kStageOwn ? bar_stage_free(s) : bar_q_free);   // this tile's staging has been read (or was never sent)
       }
     }
     }
