@@ -36,7 +36,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # launch), from the ncu captures summarised in profiles/attn_bf16_tc_*.txt
 DOMINANT_KERNEL_DRAM_BYTES = {
     "larger_imagination": int((228.190464 + 57.358848 + 87.189248 + 10.544896) * 1e6),
-    "multi_view": int((639.990784 + 198.666496 + 257.344768 + 72.386048) * 1e6),   # profiles/attn_bf16_tc_multi_view.txt
+    "multi_view": int((639.915008 + 198.356224 + 257.400064 + 68.903424) * 1e6),   # profiles/attn_bf16_tc_multi_view.txt
 }
 
 
