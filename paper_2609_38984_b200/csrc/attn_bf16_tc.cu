@@ -261,6 +261,7 @@ struct TcParams {
   const int32_t* pack_map;  // scatter and gather modes: [B, n] row of the full tensors that each attended row stands for
   int n_full;               // scatter and gather modes: rows per sample of the full tensors
   const __nv_bfloat16* q_full;  // gather mode: the full [B, n_full, N_h, D] query tensor
+  __nv_bfloat16* out_full;      // scatter and gather modes: the full [B, n_full, N_h, D] output tensor
   int lse_row0, lse_rows;
   int n, N_h;
   int kv_group;        // query heads per key/value head
@@ -310,9 +311,10 @@ struct TcCfg {
 };
 
 // MODE = kDirect: the tensor maps cover [B, n, N_h, D] tensors in boxes of 128 rows; one output store per query tile.
-// MODE = kScatter (Eq. 7 fused into the packed attention): inputs as before, but map_o covers the FULL
-// [B, n_full, N_h, D] output in boxes of one row, and each attended row goes straight to its original position
-// pack_map[b, row]; the rows the packed sequence omits are never touched and keep the cached values they hold.
+// MODE = kScatter (Eq. 7 fused into the packed attention): inputs as before, but the output is the FULL
+// [B, n_full, N_h, D] tensor and each attended row goes straight to its original position pack_map[b, row] (plain
+// 16-byte stores from the staged tile; map_o is not used); the rows the packed sequence omits are never touched and
+// keep the cached values they hold.
 // MODE = kGather (the query third of Sec. 4.2's pack fused in as well): K and V are packed tensors as before, but Q is
 // the full tensor; two warps fetch the query rows pack_map names with 16-byte asynchronous copies, writing the same
 // swizzled tile layout the tensor map would, so the packed Q never exists in memory.  map_q is not used.  (K and V
@@ -954,21 +956,38 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       mbar_arrive(bar_o_free);            // the accumulator row has been read
     }
     if (MODE != kDirect) {
-      // each thread sends the row it has just staged (it reads only its own writes, so its own proxy fence is all the
-      // ordering the copy engine needs); the 128-byte swizzle is a function of the shared-memory address, so a
-      // one-row box at the row's offset reads the same bytes the 128-row box would
+      // Eq. 7's scatter: every staged row goes to the place pack_map names in the full tensor.  The warps of the
+      // tile write the rows with 16-byte stores, a row (or two) per instruction, so each row leaves as one
+      // contiguous segment; thread r looks up row r's destination and the others get it by shuffle.  (One-row TMA
+      // stores, 512 per item, took the copy engine longer than these 16 or 32 store instructions per thread.)
       const int prow = row0 + s * kTile + r;
+      int my_orow = -1;
       if (ok && prow < p.n) {
-        const int orow = p.pack_map[(int64_t)b * p.n + prow];
-        if (orow >= 0 && orow < p.n_full) {
-          for (int db = 0; db < C::DB; ++db)
-            tma_store_4d(&map_o, sStage + s * kStageStride + db * C::kSubTile + r * 128, db * 64, orow, h, b);
-          tma_store_commit_wait();   // the thread's own staged row has been read before it writes there again
-        } else {
+        my_orow = p.pack_map[(int64_t)b * p.n + prow];
+        if (my_orow < 0 || my_orow >= p.n_full) {
           atomicOr(p.status, ST_BAD_MAP);
+          my_orow = -1;
         }
       }
-      if (!C::kStageOwn && ok) mbar_arrive(bar_q_free);    // this thread's staged row has been read (or was never sent)
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + s) : "memory");  // every row of this query tile has been staged
+      {
+        constexpr int CPR = D / 8;         // 16-byte chunks per row
+        constexpr int RPI = 32 / CPR;      // rows per warp instruction
+        const int cc = lane % CPR, sub = lane / CPR;
+        const unsigned char* stage = base_ptr + (sStage - base) + s * kStageStride + (cc >> 3) * C::kSubTile;
+        __nv_bfloat16* dst = p.out_full + ((int64_t)b * p.n_full * p.N_h + h) * D + cc * 8;
+        const int64_t row_stride = (int64_t)p.N_h * D;
+#pragma unroll 4
+        for (int it = 0; it < 32 / RPI; ++it) {
+          const int rl = it * RPI + sub;                    // row among this warp's 32
+          const int orow = __shfl_sync(0xffffffffu, my_orow, rl);
+          const int rr = (warp & 3) * 32 + rl;
+          if (orow >= 0)
+            *reinterpret_cast<uint4*>(dst + orow * row_stride) =
+                *reinterpret_cast<const uint4*>(stage + rr * 128 + (((cc & 7) ^ (rr & 7)) << 4));
+        }
+      }
+      if (!C::kStageOwn && ok) mbar_arrive(bar_q_free);    // this thread has read what it sends from the staged tile
     } else {
       asm volatile("bar.sync %0, 128;" ::"r"(1 + s) : "memory");  // the four warps of this query tile
       if (ok && (warp & 3) == 0 && lane == 0) {
@@ -1122,11 +1141,14 @@ template <int D, int MODE, bool VIS>
 cudaError_t launch_tc_v(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, float* partial,
                         size_t partial_bytes, cudaStream_t st, int* launches) {
   CUtensorMap mq, mk, mv, mo;
-  if (!(MODE != kDirect ? make_map(&mo, a.out, a.B, n_full, a.N_h, D, 1) : make_map(&mo, a.out, a.B, a.n, a.N_h, D)))
-    return cudaErrorInvalidValue;
   if (!make_map(&mk, a.k, a.B, a.n, a.N_kv, D) || !make_map(&mv, a.v, a.B, a.n, a.N_kv, D)) return cudaErrorInvalidValue;
+  if (MODE != kDirect) {
+    mo = mk;   // not used by the kernel: the scattering epilogue writes the full output tensor with plain stores
+  } else if (!make_map(&mo, a.out, a.B, a.n, a.N_h, D)) {
+    return cudaErrorInvalidValue;
+  }
   if (MODE == kGather) {
-    mq = mo;   // not used by the kernel
+    mq = mk;   // not used by the kernel
   } else if (!make_map(&mq, a.q, a.B, a.n, a.N_h, D)) {
     return cudaErrorInvalidValue;
   }
@@ -1152,7 +1174,7 @@ cudaError_t launch_tc_v(const AttnArgs& a, const int32_t* pack_map, int n_full, 
 #ifdef SWAM_TC_TRACE
       (long long*)partial_trace_buffer(),
 #endif
-      a.lse, status, partial, pack_map, n_full, (const __nv_bfloat16*)a.q, a.lse_row0, a.lse_rows, a.n, a.N_h, a.N_h / a.N_kv, pairs, n_whole + (splits ? rem * splits : 0), n_whole, splits, per,
+      a.lse, status, partial, pack_map, n_full, (const __nv_bfloat16*)a.q, (__nv_bfloat16*)a.out, a.lse_row0, a.lse_rows, a.n, a.N_h, a.N_h / a.N_kv, pairs, n_whole + (splits ? rem * splits : 0), n_whole, splits, per,
       a.scale * kLog2e, a.obs_end, a.fut_end, a.lim[0], a.lim[1], a.lim[2]};
   const int grid = p.total_work < sms ? p.total_work : sms;   // one CTA per SM; each walks through its share of the work
   ++*launches;
