@@ -35,8 +35,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel's launches in one cycle (dense launch + packed
 # launch), from the ncu captures summarised in profiles/attn_bf16_tc_*.txt
 DOMINANT_KERNEL_DRAM_BYTES = {
-    "larger_imagination": int((228.190464 + 57.358848 + 87.189248 + 10.544896) * 1e6),
-    "multi_view": int((639.915008 + 198.356224 + 257.400064 + 68.903424) * 1e6),   # profiles/attn_bf16_tc_multi_view.txt
+    "larger_imagination": int((228.235008 + 57.636608 + 87.190784 + 10.338048) * 1e6),
+    "multi_view": int((639.513856 + 198.916352 + 257.552896 + 69.681920) * 1e6),   # profiles/attn_bf16_tc_multi_view.txt
 }
 
 
