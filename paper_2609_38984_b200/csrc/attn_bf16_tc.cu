@@ -444,8 +444,8 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   // register budget: the softmax warpgroups hold a whole S row per thread, the third warpgroup (MMA issuer, TMA
   // producer, two idle warps) needs almost nothing
   // (setmaxnreg is a warpgroup-wide instruction: all four warps of a warpgroup execute the same one.  The kernel
-  // starts with 168 registers per thread (384 threads, one CTA per SM); lowering the third warpgroup to 48 releases
-  // 120 x 128 = 15360 registers, and raising the two softmax warpgroups to 224 takes 56 x 256 = 14336 of them.  An
+  // starts with 168 registers per thread (384 threads, one CTA per SM); lowering the third warpgroup to 56 releases
+  // 112 x 128 = 14336 registers, and raising the two softmax warpgroups to 224 takes exactly those 56 x 256 = 14336.  An
   // increase beyond what was released would wait forever.)
   if (warp >= 8) {
    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
