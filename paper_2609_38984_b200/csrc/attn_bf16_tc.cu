@@ -329,6 +329,12 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o, const TcParams p) {
   using C = TcCfg<D>;
   constexpr int ST = C::kStages;
+  // Where the epilogue stages the output: tiles of its own (head dim 64), the P tiles (head dim 128 in the
+  // scattering modes, where the staged rows leave by plain loads and stores and are gone when the next item's first
+  // P stores come), or the finished query tiles (head dim 128, direct mode).  In the first two cases the query
+  // tiles are released by the issuing warp after the item's last Q K^T.
+  constexpr bool kStageP = C::kPSmem && MODE != kDirect;
+  constexpr bool kQEarly = C::kStageOwn || kStageP;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_addr(smem_raw) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_raw + (base - smem_addr(smem_raw));
@@ -336,8 +342,8 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const uint32_t sP = sQ + 2 * C::kTileBytes;               // [2][tile], only with P in shared memory
   const uint32_t sK = sP + (C::kPSmem ? 2 * C::kPTileBytes : 0);   // [ST][tile]; the one ring of both with P in shared memory
   const uint32_t sV = C::kPSmem ? sK : sK + ST * C::kTileBytes;   // [ST][tile]
-  const uint32_t sStage = C::kStageOwn ? sV + ST * C::kTileBytes : sQ;   // [2] output staging tiles
-  constexpr uint32_t kStageStride = C::kTileBytes;
+  const uint32_t sStage = C::kStageOwn ? sV + ST * C::kTileBytes : (kStageP ? sP : sQ);   // [2] output staging tiles
+  constexpr uint32_t kStageStride = kStageP ? C::kPTileBytes : C::kTileBytes;
   const uint32_t bars = base + C::kSmemData;
   // barrier slots (8 bytes each)
   const uint32_t bar_q = bars;
@@ -358,7 +364,8 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const uint32_t bar_q_free = bars + 8 * (11 + 4 * ST);
   // P in shared memory: the softmax threads have read a score buffer into registers (the next Q K^T may overwrite it)
   auto bar_s_free = [&](int s) { return bars + 8 * (12 + 4 * ST + s); };
-  // direct mode: the copy engine has read query tile s's staged output (its threads may write that memory again)
+  // the staged output of query tile s has been read (its threads may write that memory again): by the copy engine
+  // in direct mode, by the tile's own threads in the scattering modes
   auto bar_stage_free = [&](int s) { return bars + 8 * (14 + 4 * ST + s); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + C::kSmemData + 8 * (16 + 4 * ST));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::kSmemData + 8 * (16 + 4 * ST) + 8);
@@ -421,9 +428,9 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     mbar_init(bar_s_free(1), kTile);
     mbar_init(bar_o_final, 1);
     mbar_init(bar_o_free, 2 * kTile);
-    mbar_init(bar_q_free, C::kStageOwn ? 1 : ((MODE == kDirect) ? 2 : 2 * kTile));
-    mbar_init(bar_stage_free(0), 1);
-    mbar_init(bar_stage_free(1), 1);
+    mbar_init(bar_q_free, kQEarly ? 1 : ((MODE == kDirect) ? 2 : 2 * kTile));
+    mbar_init(bar_stage_free(0), (MODE == kDirect) ? 1 : kTile);
+    mbar_init(bar_stage_free(1), (MODE == kDirect) ? 1 : kTile);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -650,6 +657,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
               tc_commit(bar_s_full(sq), el);
             }
             tc_commit(bar_k_empty(st), el);
+            if (kQEarly && j == wk.n_tiles - 1) tc_commit(bar_q_free, el);   // the query tiles have been read for the last time
             ++it0;
             return true;
           };
@@ -693,7 +701,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           issue_qk(sq, g % NB, st);
           tc_commit(bar_s_full(g % NB), el);
           if (sq == 1) tc_commit(bar_k_empty(st), el);   // both query tiles have used this key tile
-          if (C::kStageOwn && it == n_items - 1) tc_commit(bar_q_free, el);   // the query tiles have been read for the last time
+          if (kQEarly && it == n_items - 1) tc_commit(bar_q_free, el);   // the query tiles have been read for the last time
           return true;
         };
         for (int it = 0; it < NB && it < n_items && ok; ++it) ok = qk_item(it);
@@ -807,9 +815,14 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       // uninterrupted stream of 128 instructions per thread instead of four short ones with their fill and drain)
       uint32_t pk[64];
       if constexpr (C::kPSmem) {
-        // the P tile is free once the previous product of this query tile has read it (usually long ago)
+        // the P tile is free once the previous product of this query tile has read it (usually long ago), and,
+        // where the previous item's output was staged in it, once every thread of the tile has sent its rows
         if (item > 0) {
           ok = mbar_wait(bar_pv_tile(s), (item - 1) & 1, abort_flag);
+          if (!ok) break;
+        }
+        if (kStageP && j == 0 && iter > 0) {
+          ok = mbar_wait(bar_stage_free(s), (iter - 1) & 1, abort_flag);
           if (!ok) break;
         }
       }
@@ -918,7 +931,9 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tc_fence_before();
         mbar_arrive(bar_o_free);          // the accumulator row has been read
         // nothing was staged (the barriers' phases still count items)
-        if (C::kStageOwn) {
+        if (kStageP) {
+          mbar_arrive(bar_stage_free(s));
+        } else if (C::kStageOwn) {
           if (MODE == kDirect && (warp & 3) == 0 && lane == 0) mbar_arrive(bar_stage_free(s));
         } else if (MODE != kDirect || ((warp & 3) == 0 && lane == 0)) {
           mbar_arrive(bar_q_free);
@@ -987,7 +1002,11 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 *reinterpret_cast<const uint4*>(stage + rr * 128 + (((cc & 7) ^ (rr & 7)) << 4));
         }
       }
-      if (!C::kStageOwn && ok) mbar_arrive(bar_q_free);    // this thread has read what it sends from the staged tile
+      // this thread has read what it sends from the staged tile
+      if (ok) {
+        if (kStageP) mbar_arrive(bar_stage_free(s));
+        else if (!C::kStageOwn) mbar_arrive(bar_q_free);
+      }
     } else {
       asm volatile("bar.sync %0, 128;" ::"r"(1 + s) : "memory");  // the four warps of this query tile
       if (ok && (warp & 3) == 0 && lane == 0) {
