@@ -6,7 +6,11 @@
  * allocates device memory and, unless stated otherwise, never synchronises: work
  * is enqueued on the caller's stream (`stream` is a cudaStream_t passed as
  * void*; NULL is the default stream).  The caller owns every tensor and the
- * workspace; the context owns host memory only.
+ * workspace; the context owns host memory only.  The calls that do block the
+ * host: swam_bind_workspace (one small synchronous cudaMemset of the status
+ * word), swam_check (synchronises the stream and the internal copy streams)
+ * and swam_destroy (destroys the internal streams and events, if any);
+ * swam_bind_host_io creates two internal streams and five events on first use.
  *
  * Notation (the paper's): B batch, N_o observed tokens, F future latent frames,
  * N_s tokens per future frame, H action tokens, N_h heads, D head dim,
@@ -192,6 +196,13 @@ int swam_state_import(swam_ctx* ctx, const void* dev_buf, void* stream);
 /* Synchronises `stream`, reads and clears the device status word; returns SWAM_OK, SWAM_ERR_DEVICE_CHECK,
  * SWAM_ERR_TIMEOUT or SWAM_ERR_CUDA. */
 int swam_check(swam_ctx* ctx, void* stream);
+
+/* Self-test of the failure reporting of device-side waits (no counterpart in the paper).  Every wait inside the
+ * library's kernels is bounded; when a bound runs out the kernel raises the timeout bit of the status word and returns.
+ * This call makes that happen harmlessly: it enqueues a one-warp kernel that waits on a barrier nothing ever completes,
+ * gives up after limit_cycles SM clock cycles (1 .. 1e8, i.e. at most some 50 ms) and returns by itself.  The next
+ * swam_check then yields SWAM_ERR_TIMEOUT (and clears the word); the context stays usable.  Needs a bound workspace. */
+int swam_selftest_timeout(swam_ctx* ctx, uint64_t limit_cycles, void* stream);
 
 /* Options.  SWAM_OPT_ATTN_VARIANT selects the bf16 attention kernel: SWAM_ATTN_AUTO (default) runs the
  * tcgen05/TMEM kernel for head_dim 64 and 128 and the warp-level mma.sync kernel for head_dim 32;

@@ -46,22 +46,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
 // bounded wait: false when the limit ran out or another role already gave up
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try(bar, parity)) return true;
-  const unsigned long long t0 = clock64();
-  while (true) {
-    if (mbar_try(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if ((unsigned long long)(clock64() - t0) > kWaitCycles) { *abort_flag = 1; return false; }
-  }
+  return mbar_wait_bounded(bar, parity, kWaitCycles, abort_flag);
 }
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
@@ -239,29 +226,14 @@ __device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
   return ((addr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
 }
 
-#ifdef SWAM_TC_TRACE
-__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define CTA_T(k_) do { if (p.trace) p.trace[3 * 4096 + blockIdx.x * 4 + (k_)] = gtime(); } while (0)
-#else
-#define CTA_T(k_) do { } while (0)
-#endif
-#ifdef SWAM_TC_TRACE
-#define TRACE(slot_, idx_) do { if (blockIdx.x == 0 && p.trace) p.trace[(slot_) * 4096 + (idx_)] = clock64(); } while (0)
-#else
-#define TRACE(slot_, idx_) do { } while (0)
-#endif
-
 struct TcParams {
-#ifdef SWAM_TC_TRACE
-  long long* trace;
-#endif
   float* lse;
   int* status;
   float* partial;      // split items: [slot][2 tiles][128 rows][D + 4]: unnormalised O, then reference max and sum
-  const int32_t* pack_map;  // scatter and gather modes: [B, n] row of the full tensors that each attended row stands for
-  int n_full;               // scatter and gather modes: rows per sample of the full tensors
+  const int32_t* pack_map;  // gather mode: [B, n] row of the full tensors that each attended row stands for
+  int n_full;               // gather mode: rows per sample of the full tensors
   const __nv_bfloat16* q_full;  // gather mode: the full [B, n_full, N_h, D] query tensor
-  __nv_bfloat16* out_full;      // scatter and gather modes: the full [B, n_full, N_h, D] output tensor
+  __nv_bfloat16* out_full;      // gather mode: the full [B, n_full, N_h, D] output tensor
   int lse_row0, lse_rows;
   int n, N_h;
   int kv_group;        // query heads per key/value head
@@ -311,15 +283,14 @@ struct TcCfg {
 };
 
 // MODE = kDirect: the tensor maps cover [B, n, N_h, D] tensors in boxes of 128 rows; one output store per query tile.
-// MODE = kScatter (Eq. 7 fused into the packed attention): inputs as before, but the output is the FULL
-// [B, n_full, N_h, D] tensor and each attended row goes straight to its original position pack_map[b, row] (plain
-// 16-byte stores from the staged tile; map_o is not used); the rows the packed sequence omits are never touched and
-// keep the cached values they hold.
-// MODE = kGather (the query third of Sec. 4.2's pack fused in as well): K and V are packed tensors as before, but Q is
-// the full tensor; two warps fetch the query rows pack_map names with 16-byte asynchronous copies, writing the same
-// swizzled tile layout the tensor map would, so the packed Q never exists in memory.  map_q is not used.  (K and V
-// are shared by every query tile pair of a head: packing them once is cheaper than gathering them in every CTA.)
-enum { kDirect = 0, kScatter = 1, kGather = 2 };
+// MODE = kGather (the sparse step with Eq. 7's scatter and the query third of Sec. 4.2's pack fused in): K and V are
+// packed tensors as before, but Q and the output are the FULL [B, n_full, N_h, D] tensors.  Two warps fetch the query
+// rows pack_map names with 16-byte asynchronous copies, writing the same swizzled tile layout the tensor map would, so
+// the packed Q never exists in memory, and each attended row goes straight to its original position
+// pack_map[b, row] (plain 16-byte stores from the staged tile); the rows the packed sequence omits are never touched
+// and keep the cached values they hold.  map_q and map_o are not used.  (K and V are shared by every query tile pair
+// of a head: packing them once is cheaper than gathering them in every CTA.)
+enum { kDirect = 0, kGather = 2 };
 constexpr int kGatherThreads = 64;   // warps 10 and 11
 
 // VIS: visibility is restricted (per-row key limits); false = every row sees all n keys and none of that code exists
@@ -408,7 +379,6 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     return k;
   };
 
-  if (threadIdx.x == 0) CTA_T(0);
   if (threadIdx.x == 0) {
     // direct loads: one arrival (the expect_tx) plus the bytes; gathered loads: one arrival per producer thread
     mbar_init(bar_q, (MODE == kGather) ? kGatherThreads : 1);
@@ -646,12 +616,9 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           // the product of tile j.  kt0 counts the key tiles of finished items, it0 the ring loads consumed.
           auto qk_pair = [&](int j) -> bool {
             const int st = it0 % ST, g = kt0 + j;
-            if (iter == 0) TRACE(2, j * 8 + 0);
             if (!wait_all(bar_k_full(st), (it0 / ST) & 1)) return false;
-            if (iter == 0) TRACE(2, j * 8 + 1);
             for (int sq = 0; sq < 2; ++sq) {
               if (g > 0 && !wait_all(bar_s_free(sq), (g - 1) & 1)) return false;
-              if (iter == 0) TRACE(2, j * 8 + 2 + sq);
               tc_fence_after();
               issue_qk(sq, sq, st);
               tc_commit(bar_s_full(sq), el);
@@ -663,15 +630,12 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           };
           auto pv_pair = [&](int j) -> bool {
             const int st = it0 % ST, g = kt0 + j;
-            if (iter == 0) TRACE(2, j * 8 + 4);
             if (!wait_all(bar_k_full(st), (it0 / ST) & 1)) return false;
-            if (iter == 0) TRACE(2, j * 8 + 5);
             // the first product of an item overwrites the output accumulators: the previous item's epilogue must
             // have read them
             if (j == 0 && iter > 0 && !wait_all(bar_o_free, (iter - 1) & 1)) return false;
             for (int sq = 0; sq < 2; ++sq) {
               if (!wait_all(bar_p_full(sq), g & 1)) return false;
-              if (iter == 0) TRACE(2, j * 8 + 6 + sq);
               tc_fence_after();
               issue_pv_ss(sq, st, j > 0);
               tc_commit(bar_pv_tile(sq), el);
@@ -712,7 +676,6 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             if (!ok) break;
             v_waited = j + 1;
           }
-          if (iter == 0) TRACE(2, it * 4 + 0);
           ok = wait_all(bar_p_full(buf), (g / NB) & 1);
           if (!ok) break;
           if (it == 0 && iter > 0) {
@@ -721,14 +684,11 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             ok = wait_all(bar_o_free, (iter - 1) & 1);
             if (!ok) break;
           }
-          if (iter == 0) TRACE(2, it * 4 + 1);
           tc_fence_after();
           issue_pv(sq, buf, st, j > 0);
-          if (iter == 0) TRACE(2, it * 4 + 2);
           tc_commit(bar_pv_tile(sq), el);
           if (sq == 1) tc_commit(bar_v_empty(st), el);
           if (it + NB < n_items) ok = qk_item(it + NB);
-          if (iter == 0) TRACE(2, it * 4 + 3);
         }
         if (ok) tc_commit(bar_o_final, el);
         kt0 += wk.n_tiles;
@@ -770,11 +730,8 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       const int item = C::kPSmem ? kt0 + j : it0 + 2 * j + s, buf = C::kPSmem ? s : item % NB;
       const uint32_t s_par = C::kPSmem ? (item & 1) : ((item / NB) & 1);
       const uint32_t tS = tm_S(buf) + lane_off;
-      if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 0);
       ok = mbar_wait(bar_s_full(buf), s_par, abort_flag);
       if (!ok) break;
-      if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 1);
-      if (r == 0 && s == 0 && j == 0 && iter == 0) CTA_T(1);
       tc_fence_after();
       float sv[kTile];
 #pragma unroll
@@ -784,7 +741,6 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tc_fence_before();
         mbar_arrive(bar_s_free(s));   // the scores are in registers: the next key tile's may be written
       }
-      if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 2);
       const int valid = row_keys - (kv_begin + j) * kTile;  // keys of this tile that this row sees (<= 0: none)
       if (valid < kTile) {
 #pragma unroll
@@ -846,12 +802,10 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           if ((i & 15) == 15) store_p16(tS, i >> 4, &pk[i - 15]);
         }
       }
-      if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 5);
       if constexpr (!C::kPSmem) {
 #pragma unroll
         for (int c = 0; c < 4; ++c) store_p16(tS, c, &pk[c * 16]);
       }
-      if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 7);
       float sum;
       {
         float a0, a1;
@@ -902,16 +856,13 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
       }
       l_run += sum;
-      if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 3);
       tmem_st_wait();
       tc_fence_before();
       if constexpr (C::kPSmem) fence_proxy_async();   // P was written through the generic proxy; the tensor core reads it through the async one
       mbar_arrive(bar_p_full(buf));
-      if ((r & 63) == 0 && iter == 0) TRACE(s + (r >> 6) * 6, j * 8 + 4);
     }
     // epilogue
     if (ok) ok = mbar_wait(bar_o_final, iter & 1, abort_flag);
-    if (r == 0 && s == 0 && iter == 0) CTA_T(2);
     if (slot >= 0) {
       // a piece of a split item: unnormalised O, reference max and sum go to scratch; the combine kernel finishes
       if (ok) {
@@ -1026,7 +977,6 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0) CTA_T(3);
   if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, ST_TIMEOUT);
   if (warp == 8) {
     tc_fence_after();
@@ -1136,26 +1086,8 @@ bool make_map(CUtensorMap* map, const void* ptr, int B, int n, int N_h, int D, i
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-#ifdef SWAM_TC_TRACE
-void* g_trace = nullptr;
-void* partial_trace_buffer() {
-  if (!g_trace) { cudaMalloc(&g_trace, 8 * 4096 * 8); cudaMemset(g_trace, 0, 8 * 4096 * 8); }
-  return g_trace;
-}
-#endif
-
-int sm_count_tc() {
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
-  }
-  return sms;
-}
-
-// kScatter: a.out is the full [B, n_full, N_h, D] tensor and pack_map [B, a.n] names the row each attended row goes
-// to.  kGather: a.q is the full tensor as well and pack_map also names the query rows.
+// kGather: a.q and a.out are the full [B, n_full, N_h, D] tensors and pack_map [B, a.n] names the row of them that
+// each attended row stands for.
 template <int D, int MODE, bool VIS>
 cudaError_t launch_tc_v(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, float* partial,
                         size_t partial_bytes, cudaStream_t st, int* launches) {
@@ -1176,7 +1108,7 @@ cudaError_t launch_tc_v(const AttnArgs& a, const int32_t* pack_map, int n_full, 
   const int pairs = (a.n + 2 * kTile - 1) / (2 * kTile);
   const int items = pairs * a.N_h * a.B;
   const int n_tiles = (a.n + kTile - 1) / kTile;
-  const int sms = sm_count_tc();
+  const int sms = sm_count();
   // one CTA per SM: the items beyond the last full wave are cut over the keys into pieces that fill the idle SMs
   int rem = items % sms, splits = 0, per = n_tiles;
   if (items > sms && rem > 0 && rem <= sms / 2 && n_tiles >= 4 && a.full_visibility()) {
@@ -1190,9 +1122,6 @@ cudaError_t launch_tc_v(const AttnArgs& a, const int32_t* pack_map, int n_full, 
   }
   const int n_whole = splits ? items - rem : items;
   TcParams p{
-#ifdef SWAM_TC_TRACE
-      (long long*)partial_trace_buffer(),
-#endif
       a.lse, status, partial, pack_map, n_full, (const __nv_bfloat16*)a.q, (__nv_bfloat16*)a.out, a.lse_row0, a.lse_rows, a.n, a.N_h, a.N_h / a.N_kv, pairs, n_whole + (splits ? rem * splits : 0), n_whole, splits, per,
       a.scale * kLog2e, a.obs_end, a.fut_end, a.lim[0], a.lim[1], a.lim[2]};
   const int grid = p.total_work < sms ? p.total_work : sms;   // one CTA per SM; each walks through its share of the work
@@ -1216,10 +1145,6 @@ cudaError_t launch_tc_d(const AttnArgs& a, const int32_t* pack_map, int n_full, 
 
 }  // namespace
 
-#ifdef SWAM_TC_TRACE
-extern "C" void swam_debug_trace(long long* host) { cudaMemcpy(host, g_trace, 8 * 4096 * 8, cudaMemcpyDeviceToHost); }
-#endif
-
 size_t attn_tc_scratch_bytes(int D) {
   // room for one piece per SM (the split pieces never outnumber the SMs); 160 covers the SM count of this part
   return (size_t)160 * 2 * kTile * (D + 4) * sizeof(float);
@@ -1230,15 +1155,6 @@ cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, void* scratch, s
   switch (a.D) {
     case 64: return launch_tc_d<64, kDirect>(a, nullptr, a.n, status, (float*)scratch, scratch_bytes, st, launches);
     case 128: return launch_tc_d<128, kDirect>(a, nullptr, a.n, status, (float*)scratch, scratch_bytes, st, launches);
-    default: return cudaErrorInvalidConfiguration;
-  }
-}
-
-cudaError_t launch_attn_bf16_tc_scatter(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, void* scratch,
-                                        size_t scratch_bytes, cudaStream_t st, int* launches) {
-  switch (a.D) {
-    case 64: return launch_tc_d<64, kScatter>(a, pack_map, n_full, status, (float*)scratch, scratch_bytes, st, launches);
-    case 128: return launch_tc_d<128, kScatter>(a, pack_map, n_full, status, (float*)scratch, scratch_bytes, st, launches);
     default: return cudaErrorInvalidConfiguration;
   }
 }

@@ -19,18 +19,6 @@ constexpr unsigned long long kWaitCycles = 4000000000ull;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  const unsigned long long t0 = clock64();
-  while (true) {
-    uint32_t ok;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    if (ok) return true;
-    if ((unsigned long long)(clock64() - t0) > kWaitCycles) return false;
-  }
-}
-
 struct RowCopyParams {
   const unsigned char* src[3];
   unsigned char* dst[3];
@@ -76,7 +64,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) row_copy_bulk_kernel(const Row
 
   auto retire_one = [&]() {  // wait for the oldest load, send it out, free one ring slot
     const int st = (int)(stored % kStages);
-    if (!mbar_wait_bounded(bar0 + 8 * st, (uint32_t)((stored / kStages) & 1))) { ok = false; return; }
+    if (!mbar_wait_bounded(bar0 + 8 * st, (uint32_t)((stored / kStages) & 1), kWaitCycles, nullptr)) { ok = false; return; }
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                  ::"l"(p.dst[pend_z[st]] + pend_dst[st]), "r"(ring_a + st * kSegMax), "r"(p.seg_bytes) : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -183,13 +171,6 @@ __global__ void __launch_bounds__(kBlendThreads) blend_kernel(const BlendParams 
   }
 }
 
-int sm_count() {
-  int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  return sms;
-}
-
 cudaError_t launch_row_copy(RowCopyParams& p, int batch, cudaStream_t st) {
   int segs = 1;
   while (p.row_bytes / segs > kSegMax || (p.row_bytes % (segs * 16)) != 0) {
@@ -201,12 +182,9 @@ cudaError_t launch_row_copy(RowCopyParams& p, int batch, cudaStream_t st) {
   p.units = (long long)p.n_tensors * batch * p.n_rows * segs;
   if (p.units == 0) return cudaSuccess;
   const size_t smem = (size_t)kWarps * kStages * kSegMax;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(row_copy_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  // the opt-in is per device, and a process may hold contexts on several: set it on every launch
+  cudaError_t e = cudaFuncSetAttribute(row_copy_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
   long long ctas = (p.units + kWarps * 4 - 1) / (kWarps * 4);  // at least four units per warp
   const int sms = sm_count();
   if (ctas > sms) ctas = sms;

@@ -460,12 +460,7 @@ template <int D, int NT>
 cudaError_t launch_score_bf16(const Dims& d, const ScoreParams& p, cudaStream_t st) {
   // 32 keys per CTA, except when that gives between one and two CTAs per SM: then 64-key CTAs (one per SM, half the
   // query-fragment staging) finish sooner
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
-  }
+  const int sms = sm_count();
   const long long n32 = (long long)((d.N_s + 31) / 32) * d.F * d.B;
   if (n32 > sms && n32 <= 2 * sms) return launch_score_bf16_hg<D, NT, 4, 4>(d, p, st);
   return launch_score_bf16_hg<D, NT, 4, 2>(d, p, st);
@@ -557,18 +552,14 @@ cudaError_t launch_action_lse(const Dims& d, const void* q, const void* k, float
   const int n_tiles = (n_keys + kFlashBN - 1) / kFlashBN;
   const int q_chunks = (d.H + 63) / 64;
   const int max_splits = (d.L + kLseKeys - 1) / kLseKeys;
-  int sms = 148;
-  {
-    int dev = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  }
+  const int sms = sm_count();
   int want = (4 * sms + d.N_h * d.B * q_chunks - 1) / (d.N_h * d.B * q_chunks);
   want = want < 1 ? 1 : (want > max_splits ? max_splits : want);
   const int per = (n_tiles + want - 1) / want;
   const int n_chunks = (n_tiles + per - 1) / per;     // = number of key ranges
   LseFlashParams p{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (float2*)scratch, d.H, d.N_h, d.L, n_chunks, per,
                    d.scale * kLog2e, d.N_kv, n_keys};
-  const int wm = d.H >= 64 ? 4 : (d.H > 16 ? 2 : 1);    // warps over the query rows (H <= 16, <= 32, more)
+  const int wm = d.H > 32 ? 4 : (d.H > 16 ? 2 : 1);     // warps over the query rows, 16 each: H <= 16, <= 32, more
   dim3 grid(n_chunks, d.N_h, d.B * q_chunks);
   cudaError_t e = cudaSuccess;
   *launches += 2;

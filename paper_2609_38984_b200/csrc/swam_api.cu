@@ -276,6 +276,7 @@ int swam_score_noalloc(swam_ctx* c, const void* q, const void* k, float* scores,
   if (!c || !q || !k || !scores) return fail(c, SWAM_ERR_INVALID_ARG, "swam_score_noalloc: null argument");
   if (!aligned16(q) || !aligned16(k) || !aligned16(scores))
     return fail(c, SWAM_ERR_INVALID_ARG, "swam_score_noalloc: misaligned pointer");
+  if (int r = check_device(c)) return r;   // the built-in array's address differs from device to device
   if (static_scratch_need(c->d) > kStaticScratchBytes) {
     snprintf(c->err, sizeof(c->err), "swam_score_noalloc: this shape needs %zu bytes of scratch, the built-in array holds %zu",
              static_scratch_need(c->d), (size_t)kStaticScratchBytes);
@@ -544,6 +545,18 @@ int swam_check(swam_ctx* c, void* stream) {
              (word & ST_BAD_COUNT) ? " [selection count mismatch]" : "", (word & ST_TIMEOUT) ? " [bounded wait ran out]" : "");
     return (word & ST_TIMEOUT) ? SWAM_ERR_TIMEOUT : SWAM_ERR_DEVICE_CHECK;
   }
+  return SWAM_OK;
+}
+
+int swam_selftest_timeout(swam_ctx* c, uint64_t limit_cycles, void* stream) {
+  if (!c) return SWAM_ERR_INVALID_ARG;
+  if (limit_cycles == 0 || limit_cycles > 100000000ull)
+    return fail(c, SWAM_ERR_INVALID_ARG, "swam_selftest_timeout: limit must lie in [1, 1e8] cycles");
+  if (int r = need_ws(c)) return r;
+  if (int r = check_device(c)) return r;
+  cudaError_t e = launch_wait_probe((int*)(c->ws + c->off_status), limit_cycles, (cudaStream_t)stream, &c->launches_i);
+  count(c);
+  if (e != cudaSuccess) return fail_cuda(c, e, "wait self-test launch");
   return SWAM_OK;
 }
 

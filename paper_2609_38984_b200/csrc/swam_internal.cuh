@@ -70,6 +70,40 @@ __device__ __forceinline__ void quality_of_scores(const float* s, int F, int N_s
 }
 __host__ __device__ inline int quality_parts(int F) { return F >= 32 ? 1 : 32 / F; }
 
+// Bounded wait on an mbarrier phase, shared by every kernel that waits (attention roles, the bulk-copy ring, the
+// self-test): polls until the phase with `parity` completes, `limit_cycles` SM clocks have passed, or (when
+// abort_flag is given) another role of the CTA has already given up.  Returns false in the last two cases; on expiry
+// it raises *abort_flag so that the CTA's other roles stop waiting too.  The caller reports ST_TIMEOUT and returns.
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, unsigned long long limit_cycles,
+                                                  volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = clock64();
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (abort_flag && *abort_flag) return false;
+    if ((unsigned long long)(clock64() - t0) > limit_cycles) {
+      if (abort_flag) *abort_flag = 1;
+      return false;
+    }
+  }
+}
+
+// SMs of the current device (queried on every call: a process may hold contexts on several devices)
+inline int sm_count() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+    sms = 148;
+  return sms;
+}
+
 // ---- score.cu -------------------------------------------------------------
 // S[b,f,j] (Eq. 12) from the action rows of q, the future rows of k and lambda [B,N_h,H].
 cudaError_t launch_score(const Dims& d, const Alpha& alpha, const void* q, const void* k, const float* lse,
@@ -111,6 +145,10 @@ cudaError_t launch_pack(const Dims& d, const void* const src[3], void* const dst
 cudaError_t launch_scatter(const Dims& d, const void* out_p, const int32_t* pack_map, const int32_t* inv_map,
                            const void* cached, void* out, int* status, cudaStream_t st, int* launches);
 
+// ---- wait_probe.cu --------------------------------------------------------
+// one warp waits, bounded by limit_cycles, on a barrier that nothing completes, and reports ST_TIMEOUT
+cudaError_t launch_wait_probe(int* status, unsigned long long limit_cycles, cudaStream_t st, int* launches);
+
 // ---- attn_*.cu ------------------------------------------------------------
 struct AttnArgs {
   const void* q;
@@ -136,7 +174,6 @@ struct AttnArgs {
     return m;
   }
 };
-cudaError_t attn_prepare(int D, int dtype);
 cudaError_t launch_attn_f32(const AttnArgs& a, cudaStream_t st, int* launches);
 cudaError_t launch_attn_bf16_mma(const AttnArgs& a, cudaStream_t st, int* launches);
 // tcgen05 / TMEM / TMA kernel, head_dim 64 or 128; bounded waits report through the status word
@@ -144,13 +181,10 @@ cudaError_t launch_attn_bf16_mma(const AttnArgs& a, cudaStream_t st, int* launch
 size_t attn_tc_scratch_bytes(int D);
 cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, void* scratch, size_t scratch_bytes, cudaStream_t st,
                                 int* launches);
-// Packed attention with Eq. 7's scatter fused into the epilogue: q, k, v are the packed tensors [B, a.n, N_h, D];
-// a.out is the FULL output tensor [B, n_full, N_h, D], and attended row i of sample b is written to row
-// pack_map[b, i] of it.  Rows that pack_map does not name are not touched.  a.lse is ignored.
-cudaError_t launch_attn_bf16_tc_scatter(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, void* scratch,
-                                        size_t scratch_bytes, cudaStream_t st, int* launches);
-// The same with the query third of Sec. 4.2's pack fused in too: a.q and a.out are FULL tensors [B, n_full, N_h, D],
-// a.k and a.v packed ones; the kernel fetches query row pack_map[b, i] for attended row i itself.
+// Packed attention with Eq. 7's scatter and the query third of Sec. 4.2's pack fused in: a.k and a.v are packed
+// tensors [B, a.n, N_kv, D]; a.q and a.out are FULL tensors [B, n_full, N_h, D].  The kernel fetches query row
+// pack_map[b, i] for attended row i itself and writes the result to row pack_map[b, i] of a.out.  Rows that pack_map
+// does not name are not touched.  a.lse is ignored.
 cudaError_t launch_attn_bf16_tc_gather(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, void* scratch,
                                        size_t scratch_bytes, cudaStream_t st, int* launches);
 

@@ -30,7 +30,7 @@ EXPORTS = [
     "swam_select", "swam_aggregate", "swam_select_maps",
     "swam_pack", "swam_sparse_attn", "swam_scatter", "swam_step", "swam_host_io_bytes", "swam_bind_host_io",
     "swam_step_host", "swam_host_join", "swam_get_selection", "swam_get_scores", "swam_set_selection", "swam_state_bytes",
-    "swam_state_export", "swam_state_import", "swam_check", "swam_set_option", "swam_launch_count",
+    "swam_state_export", "swam_state_import", "swam_check", "swam_selftest_timeout", "swam_set_option", "swam_launch_count",
     "swam_last_error", "swam_version",
 ]
 
@@ -87,6 +87,7 @@ def load_library() -> ctypes.CDLL:
         lib.swam_state_export.argtypes = [vp, vp, vp]
         lib.swam_state_import.argtypes = [vp, vp, vp]
         lib.swam_check.argtypes = [vp, vp]
+        lib.swam_selftest_timeout.argtypes = [vp, ctypes.c_uint64, vp]
         lib.swam_set_option.argtypes = [vp, i32, i32]
         lib.swam_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
         lib.swam_last_error.argtypes = [vp]
@@ -314,6 +315,10 @@ class Swam:
 
     def check(self):
         self._chk(self.lib.swam_check(self.ctx, _stream()))
+
+    def selftest_timeout(self, limit_cycles: int = 100_000):
+        """Enqueue the wait self-test: the next check() raises SwamError(ERR_TIMEOUT)."""
+        self._chk(self.lib.swam_selftest_timeout(self.ctx, limit_cycles, _stream()))
 
     def set_option(self, option: int, value: int):
         self._chk(self.lib.swam_set_option(self.ctx, option, value))

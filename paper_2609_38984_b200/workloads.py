@@ -117,19 +117,21 @@ WORKLOADS: Dict[str, Workload] = {
     "multi_view": Workload("multi_view", 8, 1728, 4, 3, 24, 24, 32, 24, 64, BF16, 0.25, 10, 2, 3, blobs=1),
 }
 
-# Shapes of the models the paper evaluates (Table 5): camera views, future latent frames, tokens per future frame,
-# denoising steps, and the integer budgets K_c + K_s; refresh = steps means that only the first step is a full step,
-# the paper's default (Sec. 4.2).  The paper does not print head counts, head sizes, the number of action tokens or the
-# size of the observed frame: those are stand-ins (one observed latent frame of N_s tokens, 8 action tokens per
-# future frame).  Cosmos 3 Edge's three views differ in size (340 tokens per frame do not split into three equal
-# grids), so it is laid out as one 20 x 17 grid.
+# Shapes of the models the paper evaluates (Table 5 and App. B.2): camera views, future latent frames, tokens per
+# future frame, denoising steps, the integer budgets K_c + K_s, and the action horizon of 32 tokens that all three
+# backbones share, which gives four frame-aligned queries per future frame for the Cosmos models (8 frames) and
+# sixteen for FastWAM-Joint (2 frames).  refresh = steps means that only the first step is a full step, the paper's
+# default (Sec. 4.2).  The paper does not print head counts, head sizes or the size of the observed frame: those are
+# stand-ins (one observed latent frame of N_s tokens).  Cosmos 3 Edge's three views differ in size (340 tokens per
+# frame do not split into three equal grids), so it is laid out as one 20 x 17 grid.
+PAPER_ACTION_HORIZON = 32
 PAPER_SHAPES: Dict[str, Workload] = {
-    "cosmos3_nano": Workload("cosmos3_nano", 1, 360, 8, 3, 10, 12, 64, 16, 128, BF16, 184 / 360, 4, 4, 11, blobs=1,
-                             k_core=80, k_anchor=104),
-    "cosmos3_edge": Workload("cosmos3_edge", 1, 340, 8, 1, 20, 17, 64, 16, 128, BF16, 184 / 340, 4, 4, 12, blobs=2,
-                             k_core=80, k_anchor=104),
-    "fastwam_joint": Workload("fastwam_joint", 1, 98, 2, 2, 7, 7, 16, 12, 64, BF16, 31 / 98, 10, 10, 13, blobs=1,
-                              k_core=19, k_anchor=12),
+    "cosmos3_nano": Workload("cosmos3_nano", 1, 360, 8, 3, 10, 12, PAPER_ACTION_HORIZON, 16, 128, BF16, 184 / 360, 4, 4, 11,
+                             blobs=1, k_core=80, k_anchor=104),
+    "cosmos3_edge": Workload("cosmos3_edge", 1, 340, 8, 1, 20, 17, PAPER_ACTION_HORIZON, 16, 128, BF16, 184 / 340, 4, 4, 12,
+                             blobs=2, k_core=80, k_anchor=104),
+    "fastwam_joint": Workload("fastwam_joint", 1, 98, 2, 2, 7, 7, PAPER_ACTION_HORIZON, 12, 64, BF16, 31 / 98, 10, 10, 13,
+                              blobs=1, k_core=19, k_anchor=12),
 }
 
 # Retained tokens per frame in the paper's pruning-ratio ablation on 360-token frames (Sec. 5.4: ratios 28.89 %,

@@ -107,7 +107,9 @@ def test_select_is_deterministic():
     small("larger_imagination", n_obs=40, grid_h=7, grid_w=9, n_heads=5),   # bf16, D = 128
     small(n_frames=2, n_action=32, head_dim=32),          # g = 16 (two query tiles), D = 32
     small(n_frames=8, n_action=32),                       # g = 4 (padded query tile)
-], ids=["tiny_f32", "d64", "d128", "g16_d32", "g4"])
+    small(n_frames=10, n_action=40),                      # H = 40: more than two 16-row query blocks, fewer than four
+    small("larger_imagination", n_obs=40, grid_h=7, grid_w=9, n_heads=5, n_frames=3, n_action=48),   # H = 48, g = 16
+], ids=["tiny_f32", "d64", "d128", "g16_d32", "g4", "h40", "h48_g16_d128"])
 @pytest.mark.parametrize("given_lse", [True, False])
 def test_score_matches_oracle(wl, given_lse):
     swam = _swam()
@@ -128,6 +130,32 @@ def test_score_matches_oracle(wl, given_lse):
     if not given_lse:
         _, lse_dev, _ = ctx.cached_scores()
         assert np.abs(lse_dev.cpu().numpy() - lse64).max() <= 1e-4
+
+
+@pytest.mark.parametrize("n_frames,n_action", [(10, 40), (12, 48), (3, 48)], ids=["h40", "h48_g4", "h48_g16"])
+def test_normalisers_computed_on_the_device_cover_every_action_row(n_frames, n_action):
+    """Action counts between 33 and 63 need all four 16-row query blocks of the normaliser kernel: the scores of
+    swam_score (no normalisers given), of swam_score_noalloc and of a light refresh step are checked on them."""
+    swam = _swam()
+    wl = small(n_frames=n_frames, n_action=n_action)
+    x = W.generate_steps(wl, 1)[0]
+    q, k, v = (dev(x[n], wl) for n in "qkv")
+    lse64 = ora.action_lse(x["q"], x["k"], wl.n_action)
+    want = ora.score(x["q"], x["k"], wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, lse=lse64)
+    ctx = swam.Swam.from_workload(wl)
+    got = {"score": ctx.score(q, k).cpu().numpy().astype(np.float64)}
+    _, lse_dev, _ = ctx.cached_scores()
+    assert np.abs(lse_dev.cpu().numpy() - lse64).max() <= 1e-4
+    na = torch.full((wl.batch, wl.n_frames, wl.n_spatial), float("nan"), device="cuda")
+    swam.Swam.from_workload(wl, bind=False).score_noalloc(q, k, na)
+    got["noalloc"] = na.cpu().numpy().astype(np.float64)
+    out = ctx.empty_full().zero_()
+    ctx.step(q, k, v, swam.REFRESH_LIGHT, out)
+    ctx.check()
+    got["light"] = ctx.cached_scores()[0].cpu().numpy().astype(np.float64)
+    for name, g in got.items():
+        rel = np.abs(g - want) / np.maximum(want, 1e-30)
+        assert np.isfinite(g).all() and rel.max() <= SCORE_REL, (name, rel.max())
 
 
 def test_score_custom_weights():
@@ -714,6 +742,31 @@ def test_visibility_option_validation():
             ctx.set_visibility(*bad)
         assert e.value.code == swam.ERR_INVALID_ARG
     ctx.set_visibility(2, 2, 2)
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_survives():
+    """Failure detection without a fault: a one-warp kernel waits, with a limit of 1e5 cycles, on a barrier that
+    nothing completes; it returns by itself, swam_check reports the timeout once, and the next calls work."""
+    swam = _swam()
+    wl = small()
+    x = W.generate_steps(wl, 1)[0]
+    ctx = swam.Swam.from_workload(wl)
+    q, k, v = (dev(x[n], wl) for n in "qkv")
+    out = ctx.empty_full().zero_()
+    ctx.step(q, k, v, swam.REFRESH_FULL, out)
+    ctx.check()
+    before = out.clone()
+    ctx.selftest_timeout(100_000)
+    with pytest.raises(swam.SwamError) as e:
+        ctx.check()
+    assert e.value.code == swam.ERR_TIMEOUT and "bounded wait" in str(e.value)
+    ctx.check()                                   # the word was cleared: no second report
+    ctx.step(q, k, v, swam.REFRESH_FULL, out)     # and the context still computes the same thing
+    ctx.check()
+    assert torch.equal(out, before)
+    with pytest.raises(swam.SwamError) as e:
+        ctx.selftest_timeout(0)
+    assert e.value.code == swam.ERR_INVALID_ARG
 
 
 def test_reuse_before_refresh_is_a_state_error():

@@ -1,4 +1,6 @@
 """Host-side checks of the synthetic workload generator (no GPU)."""
+import os
+
 import numpy as np
 
 from paper_2609_38984_b200 import workloads as W
@@ -65,6 +67,13 @@ def test_paper_shapes_and_ablation_budgets():
         assert wl.n_action % wl.n_frames == 0 and wl.group % 4 == 0
         # the default schedule: only the first step is a full step
         assert W.refresh_schedule(wl.steps, wl.refresh) == [True] + [False] * (wl.steps - 1)
+    # App. B.2: action horizon and aligned queries per frame, as stored in the golden file
+    golden = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "budgets.txt")
+    rows = [ln.split() for ln in open(golden) if ln.startswith("queries ")]
+    assert len(rows) == 3
+    for _, name, horizon, per_frame in rows:
+        wl = W.PAPER_SHAPES[name]
+        assert (wl.n_action, wl.group) == (int(horizon), int(per_frame))
     nano = W.PAPER_SHAPES["cosmos3_nano"]
     # pruning ratios of the ablation: 1 - K / N_s
     assert [round(100 * (1 - k / nano.n_spatial), 2) for k in W.PAPER_PRUNING_BUDGETS] == [28.89, 48.89, 68.89]
