@@ -287,6 +287,9 @@ def test_budget_rule_against_paper_ratios():
                 assert round(100 * (1 - k / n), 2) == pct
                 kc, ks = W.budgets_from_keep(1 - pct / 100, n)
                 assert kc + ks == k
+            elif t[0] == "queries":
+                # App. B.2's query groups: the printed weights exist for exactly these group sizes
+                assert int(t[2]) == 32 and len(ora.query_weights(int(t[3]))) == int(t[3])
             else:
                 n, kc, ks, k = map(int, t[1:])
                 assert kc + ks == k <= n
