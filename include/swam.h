@@ -204,6 +204,11 @@ int swam_check(swam_ctx* ctx, void* stream);
  * swam_check then yields SWAM_ERR_TIMEOUT (and clears the word); the context stays usable.  Needs a bound workspace. */
 int swam_selftest_timeout(swam_ctx* ctx, uint64_t limit_cycles, void* stream);
 
+/* Enqueues an empty kernel (no counterpart in the paper).  Selection (call 2) reads at most a few hundred KB and is
+ * bound by launch and dependent-pass latency, not by memory bandwidth; timing this call in the same harness gives the
+ * launch floor that its time is reported against. */
+int swam_launch_floor(swam_ctx* ctx, void* stream);
+
 /* Options.  SWAM_OPT_ATTN_VARIANT selects the bf16 attention kernel: SWAM_ATTN_AUTO (default) runs the
  * tcgen05/TMEM kernel for head_dim 64 and 128 and the warp-level mma.sync kernel for head_dim 32;
  * SWAM_ATTN_WARP_MMA forces the mma.sync kernel (an independent on-device second opinion used by the tests).

@@ -560,6 +560,14 @@ int swam_selftest_timeout(swam_ctx* c, uint64_t limit_cycles, void* stream) {
   return SWAM_OK;
 }
 
+int swam_launch_floor(swam_ctx* c, void* stream) {
+  if (!c) return SWAM_ERR_INVALID_ARG;
+  cudaError_t e = launch_noop((cudaStream_t)stream, &c->launches_i);
+  count(c);
+  if (e != cudaSuccess) return fail_cuda(c, e, "empty kernel launch");
+  return SWAM_OK;
+}
+
 int swam_set_option(swam_ctx* c, int32_t option, int32_t value) {
   if (!c) return SWAM_ERR_INVALID_ARG;
   if (option == SWAM_OPT_ATTN_VARIANT && (value == SWAM_ATTN_AUTO || value == SWAM_ATTN_WARP_MMA)) {

@@ -148,6 +148,8 @@ cudaError_t launch_scatter(const Dims& d, const void* out_p, const int32_t* pack
 // ---- wait_probe.cu --------------------------------------------------------
 // one warp waits, bounded by limit_cycles, on a barrier that nothing completes, and reports ST_TIMEOUT
 cudaError_t launch_wait_probe(int* status, unsigned long long limit_cycles, cudaStream_t st, int* launches);
+// an empty kernel: the launch-latency floor
+cudaError_t launch_noop(cudaStream_t st, int* launches);
 
 // ---- attn_*.cu ------------------------------------------------------------
 struct AttnArgs {

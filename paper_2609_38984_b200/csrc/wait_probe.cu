@@ -1,4 +1,5 @@
-// Self-test of the failure-reporting path of the device-side waits.
+// Two diagnostic kernels: the self-test of the failure-reporting path of the device-side waits, and an empty kernel
+// whose launch is the latency floor that the latency-bound stages (selection) are reported against.
 //
 // Every wait in the library's kernels (attention roles on their mbarriers, the bulk-copy ring of pack and scatter) goes
 // through mbar_wait_bounded and, when its limit runs out, raises the timeout bit of the status word and lets the
@@ -26,7 +27,15 @@ __global__ void __launch_bounds__(32) wait_probe_kernel(int* status, unsigned lo
   }
 }
 
+__global__ void __launch_bounds__(32) noop_kernel() {}
+
 }  // namespace
+
+cudaError_t launch_noop(cudaStream_t st, int* launches) {
+  ++*launches;
+  noop_kernel<<<1, 32, 0, st>>>();
+  return cudaGetLastError();
+}
 
 cudaError_t launch_wait_probe(int* status, unsigned long long limit_cycles, cudaStream_t st, int* launches) {
   ++*launches;

@@ -30,7 +30,7 @@ EXPORTS = [
     "swam_select", "swam_aggregate", "swam_select_maps",
     "swam_pack", "swam_sparse_attn", "swam_scatter", "swam_step", "swam_host_io_bytes", "swam_bind_host_io",
     "swam_step_host", "swam_host_join", "swam_get_selection", "swam_get_scores", "swam_set_selection", "swam_state_bytes",
-    "swam_state_export", "swam_state_import", "swam_check", "swam_selftest_timeout", "swam_set_option", "swam_launch_count",
+    "swam_state_export", "swam_state_import", "swam_check", "swam_selftest_timeout", "swam_launch_floor", "swam_set_option", "swam_launch_count",
     "swam_last_error", "swam_version",
 ]
 
@@ -88,6 +88,7 @@ def load_library() -> ctypes.CDLL:
         lib.swam_state_import.argtypes = [vp, vp, vp]
         lib.swam_check.argtypes = [vp, vp]
         lib.swam_selftest_timeout.argtypes = [vp, ctypes.c_uint64, vp]
+        lib.swam_launch_floor.argtypes = [vp, vp]
         lib.swam_set_option.argtypes = [vp, i32, i32]
         lib.swam_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
         lib.swam_last_error.argtypes = [vp]
