@@ -216,7 +216,8 @@ __global__ void __launch_bounds__(kQualThreads) quality_kernel(const float* scor
                                                                int parts) {
   extern __shared__ double2 part_sums[];  // [F * (parts + 1)]
   const int b = blockIdx.x;
-  quality_of_scores(scores + (int64_t)b * F * N_s, F, N_s, parts, part_sums, quality + b * 3, kQualThreads);
+  quality_of_scores(scores + (int64_t)b * F * N_s, F, N_s, parts, part_sums, quality + b * 3, (int)threadIdx.x, kQualThreads,
+                    [] { __syncthreads(); });
 }
 
 // ---- action-row normalisers over all L keys -----------------------------------------------------------

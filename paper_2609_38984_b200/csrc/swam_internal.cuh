@@ -22,14 +22,16 @@ struct Alpha {
 };
 
 // Layer quality (Eq. 9) of one sample's scores S [F, N_s] (global or shared memory): R = sum S / F, E = mean normalised
-// spatial entropy, Q = R (1 - E), written to out3[0..2].  Called by every thread of a CTA of `n_threads` threads
-// (a multiple of 32); part_sums: shared memory, F * (parts + 1) entries.  With a_f = sum_j s and b_f = sum_j s ln s the
-// entropy of frame f is ln a_f - b_f / a_f.  Warps take (frame, part) units, one thread per frame then forms the
-// frame's sum and entropy term (the double-precision logarithm is the expensive part), and one thread adds the frames
-// up in ascending order: the result does not depend on which kernel calls it.
+// spatial entropy, Q = R (1 - E), written to out3[0..2].  Called by every thread of a group of `n_threads` threads
+// (a multiple of 32; `tid` = index inside the group, `sync` = the group's barrier); part_sums: shared memory,
+// F * (parts + 1) entries.  With a_f = sum_j s and b_f = sum_j s ln s the entropy of frame f is ln a_f - b_f / a_f.
+// Warps take (frame, part) units, one thread per frame then forms the frame's sum and entropy term (the
+// double-precision logarithm is the expensive part), and one thread adds the frames up in ascending order: the result
+// does not depend on which kernel, or how many threads, compute it.
+template <typename SyncFn>
 __device__ __forceinline__ void quality_of_scores(const float* s, int F, int N_s, int parts, double2* part_sums,
-                                                  float* out3, int n_threads) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+                                                  float* out3, int tid, int n_threads, SyncFn sync) {
+  const int lane = tid & 31, warp = tid >> 5;
   const int per = (N_s + parts - 1) / parts;
   for (int u = warp; u < F * parts; u += n_threads / 32) {
     const int f = u / parts, part = u % parts;
@@ -47,15 +49,15 @@ __device__ __forceinline__ void quality_of_scores(const float* s, int F, int N_s
     }
     if (lane == 0) part_sums[u] = make_double2(a, bq);
   }
-  __syncthreads();
+  sync();
   double2* frame_terms = part_sums + F * parts;   // (a_f, entropy term of frame f)
-  for (int f = threadIdx.x; f < F; f += n_threads) {
+  for (int f = tid; f < F; f += n_threads) {
     double a = 0.0, bq = 0.0;
     for (int q = 0; q < parts; ++q) { a += part_sums[f * parts + q].x; bq += part_sums[f * parts + q].y; }
     frame_terms[f] = make_double2(a, (a > 0.0) ? log(a) - bq / a : 0.0);
   }
-  __syncthreads();
-  if (threadIdx.x == 0) {
+  sync();
+  if (tid == 0) {
     double total = 0.0, ent = 0.0;
     for (int f = 0; f < F; ++f) {
       total += frame_terms[f].x;
