@@ -120,11 +120,6 @@ struct KeyRange {
 
 // Group-wide KeyRange of per-thread partial results.  Ends with the group holding the result in registers; the
 // scratch slots it used are free again after the group's next barrier.
-__device__ __forceinline__ void warp_range(uint32_t& mn, uint32_t& mx, int& cnt) {
-  mn = __reduce_min_sync(0xffffffffu, mn);
-  mx = __reduce_max_sync(0xffffffffu, mx);
-  cnt = __reduce_add_sync(0xffffffffu, cnt);
-}
 __device__ __forceinline__ void warp_range(uint64_t& mn, uint64_t& mx, int& cnt) {
   // lexicographic over the two 32-bit halves
   const uint32_t mn_hi = __reduce_min_sync(0xffffffffu, (uint32_t)(mn >> 32));

@@ -10,7 +10,8 @@ steps' selections (IoU of retained sets and the Eq. 13 overlap of the normalised
 score + select at every step), and how far the sparse output is from the dense one (relative L2; a reported
 number, not a pass/fail: the paper gives no figure for it).
 
-  python -m paper_2609_38984_b200.sweep [--keeps 0.1,0.3] [--refresh 1,2,4] [--steps 10]
+  python -m paper_2609_38984_b200.sweep [--keeps 0.1,0.3] [--refresh 1,2,4] [--steps 10] > sweep.jsonl
+  python -m paper_2609_38984_b200.sweep --summarise sweep.jsonl        # the records as a text table (no GPU needed)
   python -m paper_2609_38984_b200.sweep --shape cosmos3_nano --variants combined,core_only,stable_only,random \
          --budgets 256,184,112 --refresh first,1,2
 """
@@ -135,8 +136,28 @@ def run_config(wl: W.Workload, refresh: int, n_steps: int, dev_steps, dense_outs
     }
 
 
+def summarise(path: str) -> str:
+    """The JSON lines of a sweep run as a fixed-width text table (one row per configuration)."""
+    rows = [json.loads(ln) for ln in open(path) if ln.startswith("{")]
+    head = ("shape", "variant", "keep", "R", "K_c+K_s", "L'", "score", "select", "pack", "attn_p", "scatter", "attn_d",
+            "full", "sparse", "sched(graph)", "Mtok/s", "IoU", "Eq13", "relL2")
+    out = ["  ".join(f"{h:>12}" for h in head)]
+    for r in rows:
+        st = r["stage_us"]
+        rel = r["rel_l2_vs_dense_per_step"]
+        cells = (r["shape"][:12], r["variant"][:12], f"{r['keep']:.3f}", r["refresh"], f"{r['k_core']}+{r['k_anchor']}",
+                 r["packed_len"], st["score"], st["select"], st["pack"], st["attn_packed"], st["scatter"], st["attn_dense"],
+                 r["full_step_us"], r["sparse_step_us"] if r["sparse_step_us"] is not None else "-",
+                 r["schedule_graph_us"] if r["schedule_graph_us"] is not None else "-", f"{r['tokens_per_s'] / 1e6:.2f}",
+                 r["iou_consecutive_steps"] if r["iou_consecutive_steps"] is not None else "-",
+                 r["overlap_eq13_consecutive_steps"], f"{max(rel):.3f}")
+        out.append("  ".join(f"{str(c):>12}" for c in cells))
+    return "\n".join(out)
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--summarise", default="", help="print the JSON lines of an earlier run as a text table and exit")
     ap.add_argument("--shape", default="sweep", choices=["sweep"] + sorted(W.PAPER_SHAPES))
     ap.add_argument("--keeps", default=",".join(str(k) for k in W.SWEEP_KEEPS), help="keep ratios (shape 'sweep')")
     ap.add_argument("--budgets", default="", help="retained tokens per frame (paper shapes); default: the shape's own")
@@ -145,6 +166,9 @@ def main():
                     help="refresh intervals; 'first' = only the first step is a full step")
     ap.add_argument("--steps", type=int, default=0, help="denoising steps (default: 10, or the paper shape's own)")
     args = ap.parse_args()
+    if args.summarise:
+        print(summarise(args.summarise))
+        return
     variants = args.variants.split(",")
     if args.shape == "sweep":
         base = W.sweep_workload(1.0, 1)

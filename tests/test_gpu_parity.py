@@ -1,7 +1,7 @@
 """Parity of the CUDA path (through the C-ABI) against the CPU oracle, stage by stage and end to end.
 
 Bars: selected indices, pack maps and inverse maps bit-exact; packed/scattered tensors bit-exact; scores within
-1e-4 max-abs and 2e-5 relative; attention outputs within 1e-4 max-abs (fp32) or 2e-2 max-abs with relative
+1e-4 max-abs and 1e-5 relative; attention outputs within 1e-4 max-abs (fp32) or 2e-2 max-abs with relative
 L2 <= 1e-2 (bf16).
 """
 import numpy as np
@@ -13,7 +13,7 @@ from paper_2609_38984_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
 
-SCORE_REL = 2e-5
+SCORE_REL = 1e-5
 
 
 def _swam():
@@ -612,7 +612,7 @@ def test_grouped_query_stages_match_oracle(name, kw):
     for given in (torch.from_numpy(lse_act).cuda(), None):
         got = ctx.score(q, k, given).cpu().numpy()
         rel = np.abs(got - s64) / np.maximum(s64, 1e-30)
-        assert rel.max() <= (2e-5 if given is not None else 5e-5), rel.max()
+        assert rel.max() <= SCORE_REL, rel.max()
     sel, pm, im = ctx.select(ctx.score(q, k))
     qp, kp, vp = ctx.pack(q, k, v, pm)
     assert kp.shape[2] == wl.kv_heads and qp.shape[2] == wl.n_heads
@@ -700,7 +700,7 @@ def test_attention_with_segment_visibility(name, kw, sees):
     s64 = ora.score(x["q"], x["k"], wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action,
                     lse=ora.action_lse(x["q"], x["k"], wl.n_action, n_visible=[wl.n_obs, fut_end, wl.seq_len][sees[2]]))
     rel = np.abs(got - s64) / np.maximum(s64, 1e-30)
-    assert rel.max() <= 5e-5, rel.max()
+    assert rel.max() <= SCORE_REL, rel.max()
     # a length that is neither the full nor the packed sequence has no segment boundaries
     with pytest.raises(swam.SwamError) as e:
         ctx.sparse_attn(q[:, :wl.seq_len - 1].contiguous(), k[:, :wl.seq_len - 1].contiguous(), v[:, :wl.seq_len - 1].contiguous())
@@ -900,6 +900,38 @@ def test_cycle_replayed_from_a_cuda_graph_equals_eager():
     assert torch.equal(out_e, out_g)
     for a, b in zip(eager.selection(), graphed.selection()):
         assert torch.equal(a, b)
+
+
+def test_sweep_tool_reports_consistent_numbers_on_a_small_shape():
+    """The keep-ratio x refresh-interval sweep tool on a small shape: every key of its record is there, the overlap
+    measures lie in [0, 1], and keeping every token reproduces the dense output."""
+    swam = _swam()
+    from paper_2609_38984_b200 import sweep
+    base = small("larger_imagination", n_obs=40, grid_h=7, grid_w=9, n_heads=2, steps=4, seed=4)
+    n_steps = 4
+    host = W.generate_steps(base, n_steps)
+    dev_steps = [{n: dev(x[n], base) for n in "qkv"} for x in host]
+    dense_ctx = swam.Swam.from_workload(base)
+    dense_outs = [dense_ctx.sparse_attn(x["q"], x["k"], x["v"]) for x in dev_steps]
+    for keep, refresh in ((0.3, 2), (1.0, 2), (0.5, 1), (0.2, 4)):
+        wl = W.variant_workload(base.with_(keep=keep, k_core=None, k_anchor=None), "combined").with_(steps=n_steps, refresh=refresh)
+        rec = sweep.run_config(wl, refresh, n_steps, dev_steps, dense_outs)
+        for key in ("shape", "variant", "keep", "refresh", "k_core", "k_anchor", "packed_len", "steps", "full_steps", "stage_us",
+                    "full_step_us", "sparse_step_us", "schedule_us", "schedule_graph_us", "tokens_per_s",
+                    "iou_consecutive_steps", "overlap_eq13_consecutive_steps", "rel_l2_vs_dense_per_step"):
+            assert key in rec, key
+        assert sorted(rec["stage_us"]) == ["attn_dense", "attn_packed", "pack", "scatter", "score", "select"]
+        assert all(v > 0 for v in rec["stage_us"].values()) and rec["tokens_per_s"] > 0 and rec["schedule_graph_us"] > 0
+        assert rec["full_steps"] == len([t for t in range(n_steps) if t % refresh == 0])
+        assert rec["packed_len"] == wl.packed_len and rec["k_core"] + rec["k_anchor"] == wl.k_keep
+        assert 0.0 <= rec["iou_consecutive_steps"] <= 1.0 and 0.0 <= rec["overlap_eq13_consecutive_steps"] <= 1.0
+        assert len(rec["rel_l2_vs_dense_per_step"]) == n_steps
+        if keep == 1.0 or refresh == 1:
+            # every token kept, or every step dense: the output is the dense output (up to the kernel's own
+            # run-to-run identical arithmetic: same kernel, same inputs)
+            assert max(rec["rel_l2_vs_dense_per_step"]) <= 1e-6, rec["rel_l2_vs_dense_per_step"]
+        else:
+            assert rec["rel_l2_vs_dense_per_step"][0] <= 1e-6          # step 0 is a full step
 
 
 def test_keep_nothing_leaves_only_observed_and_action_rows():

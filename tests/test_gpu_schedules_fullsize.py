@@ -17,7 +17,7 @@ from paper_2609_38984_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
 
-SCORE_REL = 2e-5   # relative error of a score; the measured maxima are listed in the design notes
+SCORE_REL = 1e-5   # relative error of a score (measured maxima: below 1e-6 at every benchmark shape)
 TILE = 128
 
 

@@ -14,7 +14,7 @@ from paper_2609_38984_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
 
-SCORE_REL = 2e-5
+SCORE_REL = 1e-5
 
 
 @pytest.mark.parametrize("name,kw", [
