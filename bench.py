@@ -263,7 +263,7 @@ def measure_workload(wl0, args, rank, local_rank, world, device, peaks, peak_kin
         return ms, clocks
 
     ms_burst, clocks_burst = timed(0.0, 0.5)
-    ms_steady, clocks_steady = timed(STEADY_PRELOAD_S, 0.0)
+    ms_steady, clocks_steady = timed(args.preload_seconds, 0.0)
     ctx.check()
     tokens_per_cycle = wl.batch * (wl.seq_len + (R - 1) * wl.packed_len)
     value = world * tokens_per_cycle * args.steps / (ms_steady * 1e-3)
@@ -301,11 +301,12 @@ def measure_workload(wl0, args, rank, local_rank, world, device, peaks, peak_kin
            "ms_per_step_burst": ms_burst / args.steps, "clocks": clocks_steady, "clocks_burst": clocks_burst,
            "e2e": e2e, "gpu_launches": int(launches_per_cycle * args.steps),
            "config": config_of(wl0, wl, world, {
-               "timing": f"CUDA-graph replays, CUDA events; value: {args.steps} cycles right after >= {STEADY_PRELOAD_S:g} s "
+               "timing": f"CUDA-graph replays, CUDA events; value: {args.steps} cycles right after >= {args.preload_seconds:g} s "
                          f"of back-to-back replays (steady state under the power cap); value_burst: {args.steps} cycles "
                          f"after 0.5 s idle and {warm} warm-up cycles",
                "stage_timing": f"per stage: {N_ROT} rotating input sets (each launch reads cold data), launches replayed "
-                               "back to back from a CUDA graph for >= 0.3 s (attention, steps) or >= 0.05 s (others) "
+                               f"back to back from a CUDA graph for >= {args.stage_seconds:g} s (attention, steps) or >= "
+                               f"{args.stage_seconds / 6:g} s (others) "
                                "after a run-in of the same length, CUDA events around the loop"})}
     if rank != 0:
         return rec
@@ -329,7 +330,9 @@ def measure_workload(wl0, args, rank, local_rank, world, device, peaks, peak_kin
     fut = wl.n_frames * wl.n_spatial
     stage_clocks = {}
 
-    def stage(make, min_s=0.05, clock_key=None):
+    long_s, short_s = args.stage_seconds, args.stage_seconds / 6
+
+    def stage(make, min_s=short_s, clock_key=None):
         smp = ClockSampler(local_rank, period_s=0.002).start() if clock_key else None
         us = per_launch_us([make(i) for i in range(N_ROT)], min_s)
         if smp:
@@ -347,10 +350,10 @@ def measure_workload(wl0, args, rank, local_rank, world, device, peaks, peak_kin
         return lambda i: lambda: lib.swam_step(ctx.ctx, P(rot[i]["q"]), P(rot[i]["k"]), P(rot[i]["v"]), mode, P(outs[i]), S())
 
     stage_us = {
-        "attn_dense": stage(dense_call, 0.3, "attn_dense"),
-        "attn_packed": stage(packed_call, 0.3, "attn_packed"),
-        "full_step": stage(step_call(swam.REFRESH_FULL), 0.3, "full_step"),
-        "sparse_step": stage(step_call(swam.REUSE), 0.3, "sparse_step"),
+        "attn_dense": stage(dense_call, long_s, "attn_dense"),
+        "attn_packed": stage(packed_call, long_s, "attn_packed"),
+        "full_step": stage(step_call(swam.REFRESH_FULL), long_s, "full_step"),
+        "sparse_step": stage(step_call(swam.REUSE), long_s, "sparse_step"),
     }
     burst_us = {"attn_dense": first_launches_us([dense_call(i) for i in range(N_ROT)]),
                 "attn_packed": first_launches_us([packed_call(i) for i in range(N_ROT)])}
@@ -368,7 +371,7 @@ def measure_workload(wl0, args, rank, local_rank, world, device, peaks, peak_kin
                                                              None, P(packed[i][1]), P(packed[i][2]), S())),
             "scatter": stage(lambda i: lambda: lib.swam_scatter(ctx.ctx, P(outs_p[i]), P(pm), P(im), P(outs[i]), P(outs[i]),
                                                                 S())),
-            "light_refresh_step": stage(step_call(swam.REFRESH_LIGHT), 0.1),
+            "light_refresh_step": stage(step_call(swam.REFRESH_LIGHT), long_s / 3),
         })
     ctx.check()
     algo = {  # algorithmic bytes / flops per launch
@@ -615,6 +618,10 @@ def main():
                     help="further workloads measured the same way and reported under `also` (one GPU only); '' = none")
     ap.add_argument("--impl", default="swam", choices=["swam", "reference"])
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="host-core budget of the oracle baseline")
+    ap.add_argument("--preload-seconds", type=float, default=STEADY_PRELOAD_S,
+                    help="back-to-back replays before the steady-state timed region (shorten only for profiler runs)")
+    ap.add_argument("--stage-seconds", type=float, default=0.3,
+                    help="length of the per-stage timing loops of the attention launches and steps (others: a sixth)")
     ap.add_argument("--reference-seconds", type=float, default=120.0,
                     help="host-core budget of the whole --impl reference run (all warm-up and timed steps)")
     args = ap.parse_args()
