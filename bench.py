@@ -355,6 +355,11 @@ def measure_workload(wl0, args, rank, local_rank, world, device, peaks, peak_kin
         "full_step": stage(step_call(swam.REFRESH_FULL), long_s, "full_step"),
         "sparse_step": stage(step_call(swam.REUSE), long_s, "sparse_step"),
     }
+    if wl.dtype == W.BF16 and wl.head_dim >= 64:
+        # the sparse step with the key and value rows gathered inside the attention kernel (one launch, nothing packed)
+        ctx.set_option(swam.OPT_SPARSE_PATH, swam.SPARSE_FUSED_KV)
+        stage_us["sparse_step_kv_gathered_in_kernel"] = stage(step_call(swam.REUSE), long_s)
+        ctx.set_option(swam.OPT_SPARSE_PATH, swam.SPARSE_FUSED)
     burst_us = {"attn_dense": first_launches_us([dense_call(i) for i in range(N_ROT)]),
                 "attn_packed": first_launches_us([packed_call(i) for i in range(N_ROT)])}
     if detail:
@@ -408,7 +413,7 @@ def measure_workload(wl0, args, rank, local_rank, world, device, peaks, peak_kin
                             "launch_floor_us": round(stage_us["launch_floor"], 2),
                             "ratio_to_launch_floor": round(stage_us["select"] / stage_us["launch_floor"], 2),
                             "bytes": int(B * (fut * 4 + (wl.n_frames * wl.k_keep + Lp + L) * 4))}
-    for name in ("full_step", "sparse_step", "light_refresh_step"):
+    for name in ("full_step", "sparse_step", "sparse_step_kv_gathered_in_kernel", "light_refresh_step"):
         if name in stage_us:
             stages[name] = {"us": round(stage_us[name], 2)}
 

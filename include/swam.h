@@ -217,8 +217,12 @@ int swam_launch_floor(swam_ctx* ctx, void* stream);
  * SWAM_SPARSE_FUSED (default) packs only K and V; the tcgen05 attention kernel fetches its query rows from the full
  * Q through pack_map and writes each retained row straight to its original position in `out`, so that the packed Q,
  * the packed output and the scatter pass do not exist; SWAM_SPARSE_STAGED runs swam_pack, swam_sparse_attn and
- * swam_scatter one after the other.  The fused path needs bf16, head_dim 64 or 128 and SWAM_ATTN_AUTO; every other
- * configuration runs staged.  Both paths produce the same bits.
+ * swam_scatter one after the other; SWAM_SPARSE_FUSED_KV goes one step beyond FUSED: the attention kernel also
+ * fetches the key and value rows through pack_map (TMA row gathers), so that nothing is packed at all and the sparse
+ * step is one launch.  Every query tile pair of a head then repeats the gather of that head's rows, which measures
+ * slower than packing K and V once at the benchmark shapes; it is offered for shapes with few query tiles.  The fused
+ * paths need bf16, head_dim 64 or 128 and SWAM_ATTN_AUTO; every other configuration runs staged.  All three paths
+ * produce the same bits.
  *
  * SWAM_OPT_VISIBILITY sets the backbone's visibility constraints (App. A.2) in the form this library supports: the
  * joint sequence is [observed | future | action], and the rows of each of the three segments see a prefix of it, up to
@@ -231,7 +235,7 @@ int swam_launch_floor(swam_ctx* ctx, void* stream);
  * keys the action rows see. */
 enum { SWAM_OPT_ATTN_VARIANT = 1, SWAM_OPT_SPARSE_PATH = 2, SWAM_OPT_VISIBILITY = 3 };
 enum { SWAM_ATTN_AUTO = 0, SWAM_ATTN_WARP_MMA = 1 };
-enum { SWAM_SPARSE_FUSED = 0, SWAM_SPARSE_STAGED = 1 };
+enum { SWAM_SPARSE_FUSED = 0, SWAM_SPARSE_STAGED = 1, SWAM_SPARSE_FUSED_KV = 2 };
 enum { SWAM_SEES_OBSERVED = 0, SWAM_SEES_FUTURE = 1, SWAM_SEES_ALL = 2 };
 #define SWAM_VISIBILITY(observed_rows_see, future_rows_see, action_rows_see) \
   ((observed_rows_see) | ((future_rows_see) << 2) | ((action_rows_see) << 4))

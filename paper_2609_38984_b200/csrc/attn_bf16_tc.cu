@@ -57,6 +57,13 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
+// four rows of a 2-D tensor (row coordinates y0..y3, first column x) into four consecutive 128-byte rows of shared memory
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y0, int y1, int y2,
+                                            int y3) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y0), "r"(y1), "r"(y2), "r"(y3) : "memory");
+}
 __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
   asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
                ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
@@ -231,7 +238,8 @@ struct TcParams {
   int* status;
   float* partial;      // split items: [slot][2 tiles][128 rows][D + 4]: unnormalised O, then reference max and sum
   const int32_t* pack_map;  // gather mode: [B, n] row of the full tensors that each attended row stands for
-  int n_full;               // gather mode: rows per sample of the full tensors
+  int n_full;               // gather modes: rows per sample of the full tensors
+  int kv_rows;              // kGatherKV: rows of the 2-D view of K and V, B * n_full (a row coordinate beyond the tensor)
   const __nv_bfloat16* q_full;  // gather mode: the full [B, n_full, N_h, D] query tensor
   __nv_bfloat16* out_full;      // gather mode: the full [B, n_full, N_h, D] output tensor
   int lse_row0, lse_rows;
@@ -290,7 +298,12 @@ struct TcCfg {
 // pack_map[b, row] (plain 16-byte stores from the staged tile); the rows the packed sequence omits are never touched
 // and keep the cached values they hold.  map_q and map_o are not used.  (K and V are shared by every query tile pair
 // of a head: packing them once is cheaper than gathering them in every CTA.)
-enum { kDirect = 0, kGather = 2 };
+// MODE = kGatherKV: as kGather, and K and V are the FULL tensors as well: the producer warp fetches each key tile's
+// rows through pack_map with TMA row gathers (tile::gather4: every lane names four rows of the 2-D view
+// [B * n_full, N_kv * D] and gets them as four consecutive rows of the swizzled tile), so that no packed tensor exists
+// at all.  Every query tile pair of a head repeats the gather of that head's keys and values, which is why it is an
+// option and not the default (see swam_set_option).
+enum { kDirect = 0, kGather = 2, kGatherKV = 3 };
 constexpr int kGatherThreads = 64;   // warps 10 and 11
 
 // VIS: visibility is restricted (per-row key limits); false = every row sees all n keys and none of that code exists
@@ -299,6 +312,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1)
 attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o, const TcParams p) {
   using C = TcCfg<D>;
+  constexpr bool kGath = MODE == kGather || MODE == kGatherKV;   // the queries are gathered by warps 10 and 11
   constexpr int ST = C::kStages;
   // Where the epilogue stages the output: tiles of its own (head dim 64), the P tiles (head dim 128 in the
   // scattering modes, where the staged rows leave by plain loads and stores and are gone when the next item's first
@@ -381,7 +395,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 
   if (threadIdx.x == 0) {
     // direct loads: one arrival (the expect_tx) plus the bytes; gathered loads: one arrival per producer thread
-    mbar_init(bar_q, (MODE == kGather) ? kGatherThreads : 1);
+    mbar_init(bar_q, kGath ? kGatherThreads : 1);
     for (int s = 0; s < ST; ++s) {
       mbar_init(bar_k_full(s), 1);
       mbar_init(bar_k_empty(s), 1);
@@ -426,7 +440,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   // increase beyond what was released would wait forever.)
   if (warp >= 8) {
    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-   if (MODE == kGather && warp >= 10) {
+   if (kGath && warp >= 10) {
     // ------------------------------------------------------------------ gathering producers of Q (64 threads)
     // Tile row rr <- row pack_map[b, prow0 + rr] of the full tensor; 16-byte chunk cc of a row lands where the
     // 128-byte-swizzled box layout puts it: sub-tile cc / 8, row rr, chunk (cc % 8) ^ (rr % 8).  Rows beyond the
@@ -494,19 +508,53 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     }
     cp_async_wait_all();   // nothing of this thread is still on its way into shared memory at exit
    } else if (warp == 9) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ TMA producer (one lane; the whole warp when
+    // the key and value rows are gathered)
+    if (MODE == kGatherKV || lane == 0) {
+      // a failed wait ends the loops; when the whole warp runs them it must leave them together
+      auto wait = [&](uint32_t bar, uint32_t parity) {
+        bool r = mbar_wait(bar, parity, abort_flag);
+        if constexpr (MODE == kGatherKV) r = __all_sync(0xffffffffu, r ? 1 : 0) != 0;
+        return r;
+      };
       bool ok = true;
       int kt = 0;      // key/value tiles loaded so far by this CTA: ring slot kt % ST, pass kt / ST
       int iter = 0;
       for (int work = blockIdx.x; work < p.total_work && ok; work += gridDim.x, ++iter) {
         const Work wk = decode(work);
         const int h_kv = wk.h / p.kv_group;
+        // key tile `tile` of K or V into the ring slot at `dst`, completing on `bar`
+        auto load_kv = [&](uint32_t dst, bool is_v, int tile, uint32_t bar) {
+          if constexpr (MODE == kGatherKV) {
+            if (lane == 0) mbar_expect_tx(bar, C::kTileBytes);
+            __syncwarp();
+            // this lane's four rows of the tile: attended rows 4 * lane .. + 3; rows beyond the packed sequence and
+            // map entries out of range (flagged) name a row past the end of the tensor, which reads as zeros
+            int y[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int row = tile * kTile + 4 * lane + e;
+              y[e] = p.kv_rows;
+              if (row < p.n) {
+                const int o = p.pack_map[(int64_t)wk.b * p.n + row];
+                if (o < 0 || o >= p.n_full) atomicOr(p.status, ST_BAD_MAP);
+                else y[e] = wk.b * p.n_full + o;
+              }
+            }
+            for (int db = 0; db < C::DB; ++db)
+              tma_gather4(dst + db * C::kSubTile + lane * 4 * 128, is_v ? &map_v : &map_k, bar, h_kv * D + db * 64, y[0], y[1],
+                          y[2], y[3]);
+          } else {
+            mbar_expect_tx(bar, C::kTileBytes);
+            for (int db = 0; db < C::DB; ++db)
+              tma_load_4d(dst + db * C::kSubTile, is_v ? &map_v : &map_k, bar, db * 64, tile * kTile, h_kv, wk.b);
+          }
+        };
         // The first item's queries go first.  A later item's queries have to wait until the previous item's output has
         // left the query tiles, so that item's first key/value tiles (as many as the ring holds) are requested before.
         auto load_q = [&]() {
-          if (MODE == kGather) return true;
-          if (iter > 0 && !mbar_wait(bar_q_free, (iter - 1) & 1, abort_flag)) return false;
+          if (kGath) return true;
+          if (iter > 0 && !wait(bar_q_free, (iter - 1) & 1)) return false;
           mbar_expect_tx(bar_q, 2 * C::kTileBytes);
           for (int s = 0; s < 2; ++s)
             for (int db = 0; db < C::DB; ++db)
@@ -522,14 +570,11 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           if (q_after < 0) ok = load_q();
           for (int m = 0; m < n_loads && ok; ++m, ++kt) {
             const int st = kt % ST;
-            ok = mbar_wait(bar_k_empty(st), ((kt / ST) & 1) ^ 1, abort_flag);
+            ok = wait(bar_k_empty(st), ((kt / ST) & 1) ^ 1);
             if (!ok) break;
             const bool is_v = (m == n_loads - 1) || (m > 0 && (m & 1) == 0);
             const int j = (m == n_loads - 1) ? wk.n_tiles - 1 : (is_v ? m / 2 - 1 : (m + 1) / 2);
-            mbar_expect_tx(bar_k_full(st), C::kTileBytes);
-            for (int db = 0; db < C::DB; ++db)
-              tma_load_4d(sK + st * C::kTileBytes + db * C::kSubTile, is_v ? &map_v : &map_k, bar_k_full(st), db * 64,
-                          (wk.kv_begin + j) * kTile, h_kv, wk.b);
+            load_kv(sK + st * C::kTileBytes, is_v, wk.kv_begin + j, bar_k_full(st));
             if (m == q_after) ok = load_q();
           }
           continue;
@@ -539,16 +584,12 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         for (int j = 0; j < wk.n_tiles && ok; ++j, ++kt) {
           const int st = kt % ST;
           const uint32_t par = ((kt / ST) & 1) ^ 1;  // first pass over the ring: slots start empty
-          ok = mbar_wait(bar_k_empty(st), par, abort_flag);
+          ok = wait(bar_k_empty(st), par);
           if (!ok) break;
-          mbar_expect_tx(bar_k_full(st), C::kTileBytes);
-          for (int db = 0; db < C::DB; ++db)
-            tma_load_4d(sK + st * C::kTileBytes + db * C::kSubTile, &map_k, bar_k_full(st), db * 64, (wk.kv_begin + j) * kTile, h_kv, wk.b);
-          ok = mbar_wait(bar_v_empty(st), par, abort_flag);
+          load_kv(sK + st * C::kTileBytes, false, wk.kv_begin + j, bar_k_full(st));
+          ok = wait(bar_v_empty(st), par);
           if (!ok) break;
-          mbar_expect_tx(bar_v_full(st), C::kTileBytes);
-          for (int db = 0; db < C::DB; ++db)
-            tma_load_4d(sV + st * C::kTileBytes + db * C::kSubTile, &map_v, bar_v_full(st), db * 64, (wk.kv_begin + j) * kTile, h_kv, wk.b);
+          load_kv(sV + st * C::kTileBytes, true, wk.kv_begin + j, bar_v_full(st));
           if (j == q_after) ok = load_q();
         }
       }
@@ -608,7 +649,7 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         // async proxy: the reader fences after the wait
         ok = wait_all(bar_q, iter & 1);
         if (!ok) break;
-        if (MODE == kGather) fence_proxy_async();
+        if (kGath) fence_proxy_async();
         if constexpr (C::kPSmem) {
           // Order on the tensor pipe: S(0) | S(1), O += P(0) V(0) | S(2), O += P(1) V(1) | ... with both query tiles
           // side by side in every group.  Score buffer s belongs to query tile s; it is free again as soon as the
@@ -1086,19 +1127,40 @@ bool make_map(CUtensorMap* map, const void* ptr, int B, int n, int N_h, int D, i
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// [B * n, N_h * D] bf16 viewed as a 2-D tensor (column, row) for row gathers: box = 64 columns x 1 row (a gather
+// instruction names four rows), 128-byte swizzle; rows past the end read as zeros
+bool make_row_map(CUtensorMap* map, const void* ptr, long long rows, int cols) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {64, 1};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // kGather: a.q and a.out are the full [B, n_full, N_h, D] tensors and pack_map [B, a.n] names the row of them that
 // each attended row stands for.
 template <int D, int MODE, bool VIS>
 cudaError_t launch_tc_v(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, float* partial,
                         size_t partial_bytes, cudaStream_t st, int* launches) {
   CUtensorMap mq, mk, mv, mo;
-  if (!make_map(&mk, a.k, a.B, a.n, a.N_kv, D) || !make_map(&mv, a.v, a.B, a.n, a.N_kv, D)) return cudaErrorInvalidValue;
+  if (MODE == kGatherKV) {
+    // a.k and a.v are the full tensors too
+    const long long rows = (long long)a.B * n_full;
+    if (rows >= 0x7fffffffll) return cudaErrorInvalidConfiguration;
+    if (!make_row_map(&mk, a.k, rows, a.N_kv * D) || !make_row_map(&mv, a.v, rows, a.N_kv * D)) return cudaErrorInvalidValue;
+  } else if (!make_map(&mk, a.k, a.B, a.n, a.N_kv, D) || !make_map(&mv, a.v, a.B, a.n, a.N_kv, D)) {
+    return cudaErrorInvalidValue;
+  }
   if (MODE != kDirect) {
     mo = mk;   // not used by the kernel: the scattering epilogue writes the full output tensor with plain stores
   } else if (!make_map(&mo, a.out, a.B, a.n, a.N_h, D)) {
     return cudaErrorInvalidValue;
   }
-  if (MODE == kGather) {
+  if (MODE != kDirect) {
     mq = mk;   // not used by the kernel
   } else if (!make_map(&mq, a.q, a.B, a.n, a.N_h, D)) {
     return cudaErrorInvalidValue;
@@ -1122,7 +1184,7 @@ cudaError_t launch_tc_v(const AttnArgs& a, const int32_t* pack_map, int n_full, 
   }
   const int n_whole = splits ? items - rem : items;
   TcParams p{
-      a.lse, status, partial, pack_map, n_full, (const __nv_bfloat16*)a.q, (__nv_bfloat16*)a.out, a.lse_row0, a.lse_rows, a.n, a.N_h, a.N_h / a.N_kv, pairs, n_whole + (splits ? rem * splits : 0), n_whole, splits, per,
+      a.lse, status, partial, pack_map, n_full, a.B * n_full, (const __nv_bfloat16*)a.q, (__nv_bfloat16*)a.out, a.lse_row0, a.lse_rows, a.n, a.N_h, a.N_h / a.N_kv, pairs, n_whole + (splits ? rem * splits : 0), n_whole, splits, per,
       a.scale * kLog2e, a.obs_end, a.fut_end, a.lim[0], a.lim[1], a.lim[2]};
   const int grid = p.total_work < sms ? p.total_work : sms;   // one CTA per SM; each walks through its share of the work
   ++*launches;
@@ -1159,8 +1221,15 @@ cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, void* scratch, s
   }
 }
 
-cudaError_t launch_attn_bf16_tc_gather(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, void* scratch,
-                                       size_t scratch_bytes, cudaStream_t st, int* launches) {
+cudaError_t launch_attn_bf16_tc_gather(const AttnArgs& a, const int32_t* pack_map, int n_full, bool gather_kv, int* status,
+                                       void* scratch, size_t scratch_bytes, cudaStream_t st, int* launches) {
+  if (gather_kv) {
+    switch (a.D) {
+      case 64: return launch_tc_d<64, kGatherKV>(a, pack_map, n_full, status, (float*)scratch, scratch_bytes, st, launches);
+      case 128: return launch_tc_d<128, kGatherKV>(a, pack_map, n_full, status, (float*)scratch, scratch_bytes, st, launches);
+      default: return cudaErrorInvalidConfiguration;
+    }
+  }
   switch (a.D) {
     case 64: return launch_tc_d<64, kGather>(a, pack_map, n_full, status, (float*)scratch, scratch_bytes, st, launches);
     case 128: return launch_tc_d<128, kGather>(a, pack_map, n_full, status, (float*)scratch, scratch_bytes, st, launches);

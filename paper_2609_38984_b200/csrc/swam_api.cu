@@ -401,18 +401,24 @@ int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t 
     if (e != cudaSuccess) return fail_cuda(c, e, "select launch");
     c->has_selection = true;
   }
-  if (mode != SWAM_REFRESH_FULL && c->sparse_path == SWAM_SPARSE_FUSED && d.dtype == SWAM_BF16 && d.D >= 64 &&
+  if (mode != SWAM_REFRESH_FULL && c->sparse_path != SWAM_SPARSE_STAGED && d.dtype == SWAM_BF16 && d.D >= 64 &&
       c->attn_variant == SWAM_ATTN_AUTO) {
     // K and V are packed by the copy kernel (every query tile of a head reads them); the attention kernel fetches
     // its query rows from the full Q itself and writes each result row straight to its place in `out`.  The omitted
     // rows keep the cached value they already hold (Eq. 7), so neither a packed Q, nor a packed output, nor a scatter
     // pass exist.
-    void* kp = c->ws + c->off_kp;
-    void* vp = c->ws + c->off_vp;
-    if (int r = swam_pack(c, nullptr, k, v, pm, nullptr, kp, vp, stream)) return r;
+    // With SWAM_SPARSE_FUSED_KV the kernel gathers the key and value rows as well and nothing is packed.
+    const bool gather_kv = c->sparse_path == SWAM_SPARSE_FUSED_KV;
+    const void* kp = k;
+    const void* vp = v;
+    if (!gather_kv) {
+      kp = c->ws + c->off_kp;
+      vp = c->ws + c->off_vp;
+      if (int r = swam_pack(c, nullptr, k, v, pm, nullptr, c->ws + c->off_kp, c->ws + c->off_vp, stream)) return r;
+    }
     AttnArgs a{q, kp, vp, out, nullptr, 0, 0, d.B, d.Lp, d.N_h, d.D, d.scale, d.N_kv};
     set_visibility(c, a);
-    cudaError_t e = launch_attn_bf16_tc_gather(a, pm, d.L, (int*)(c->ws + c->off_status), c->ws + c->off_attn,
+    cudaError_t e = launch_attn_bf16_tc_gather(a, pm, d.L, gather_kv, (int*)(c->ws + c->off_status), c->ws + c->off_attn,
                                                c->attn_scratch, st, &c->launches_i);
     count(c);
     if (e != cudaSuccess) return fail_cuda(c, e, "fused sparse attention launch");
@@ -583,7 +589,8 @@ int swam_set_option(swam_ctx* c, int32_t option, int32_t value) {
     c->sees[0] = o; c->sees[1] = f; c->sees[2] = a;
     return SWAM_OK;
   }
-  if (option == SWAM_OPT_SPARSE_PATH && (value == SWAM_SPARSE_FUSED || value == SWAM_SPARSE_STAGED)) {
+  if (option == SWAM_OPT_SPARSE_PATH &&
+      (value == SWAM_SPARSE_FUSED || value == SWAM_SPARSE_STAGED || value == SWAM_SPARSE_FUSED_KV)) {
     c->sparse_path = value;
     return SWAM_OK;
   }

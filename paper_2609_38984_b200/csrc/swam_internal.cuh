@@ -189,7 +189,9 @@ cudaError_t launch_attn_bf16_tc(const AttnArgs& a, int* status, void* scratch, s
 // tensors [B, a.n, N_kv, D]; a.q and a.out are FULL tensors [B, n_full, N_h, D].  The kernel fetches query row
 // pack_map[b, i] for attended row i itself and writes the result to row pack_map[b, i] of a.out.  Rows that pack_map
 // does not name are not touched.  a.lse is ignored.
-cudaError_t launch_attn_bf16_tc_gather(const AttnArgs& a, const int32_t* pack_map, int n_full, int* status, void* scratch,
-                                       size_t scratch_bytes, cudaStream_t st, int* launches);
+// gather_kv: a.k and a.v are FULL tensors [B, n_full, N_kv, D] as well and the kernel fetches the key and value rows
+// pack_map names itself (TMA row gathers), so that no packed tensor exists.
+cudaError_t launch_attn_bf16_tc_gather(const AttnArgs& a, const int32_t* pack_map, int n_full, bool gather_kv, int* status,
+                                       void* scratch, size_t scratch_bytes, cudaStream_t st, int* launches);
 
 }  // namespace swam

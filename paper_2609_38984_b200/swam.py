@@ -23,7 +23,7 @@ REUSE, REFRESH_FULL, REFRESH_LIGHT = 0, 1, 2
 OPT_ATTN_VARIANT, OPT_SPARSE_PATH, OPT_VISIBILITY = 1, 2, 3
 SEES_OBSERVED, SEES_FUTURE, SEES_ALL = 0, 1, 2
 ATTN_AUTO, ATTN_WARP_MMA = 0, 1
-SPARSE_FUSED, SPARSE_STAGED = 0, 1
+SPARSE_FUSED, SPARSE_STAGED, SPARSE_FUSED_KV = 0, 1, 2
 
 EXPORTS = [
     "swam_create", "swam_destroy", "swam_workspace_bytes", "swam_bind_workspace", "swam_score", "swam_score_noalloc",

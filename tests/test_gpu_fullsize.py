@@ -113,6 +113,15 @@ def test_full_size_cycle_matches_oracle(name, wl, n_rows):
     staged.check()
     assert torch.equal(out_s, out)
     del staged, out_s
+    # ... and so does the variant in which the kernel gathers the key and value rows itself
+    gkv = swam.Swam.from_workload(wl)
+    gkv.set_option(swam.OPT_SPARSE_PATH, swam.SPARSE_FUSED_KV)
+    out_g = out_full.clone()
+    gkv.step(d0["q"], d0["k"], d0["v"], swam.REFRESH_FULL, out_g)
+    gkv.step(d1["q"], d1["k"], d1["v"], swam.REUSE, out_g)
+    gkv.check()
+    assert torch.equal(out_g, out)
+    del gkv, out_g
 
     # ---- every element: tcgen05 kernel vs the independent mma.sync kernel ----------------------------------
     other = swam.Swam.from_workload(wl)

@@ -440,11 +440,12 @@ def test_light_refresh_step():
 ], ids=["d64", "d128", "d128_long_obs", "keep_all", "keep_none"])
 @pytest.mark.parametrize("mode", ["reuse", "light"])
 def test_fused_sparse_step_equals_staged_bit_for_bit(wl, mode):
-    """Packed attention with the scatter fused into its epilogue and pack -> attention -> scatter give the same bits."""
+    """Packed attention with the scatter and the query gather fused in, the same with the key and value rows gathered
+    by the kernel as well, and pack -> attention -> scatter give the same bits."""
     swam = _swam()
     x0, x1 = W.generate_steps(wl, 2)
     outs = []
-    for path in (swam.SPARSE_FUSED, swam.SPARSE_STAGED):
+    for path in (swam.SPARSE_FUSED, swam.SPARSE_STAGED, swam.SPARSE_FUSED_KV):
         ctx = swam.Swam.from_workload(wl)
         ctx.set_option(swam.OPT_SPARSE_PATH, path)
         out = ctx.empty_full().zero_()
@@ -455,8 +456,8 @@ def test_fused_sparse_step_equals_staged_bit_for_bit(wl, mode):
                  swam.REUSE if mode == "reuse" else swam.REFRESH_LIGHT, out)
         ctx.check()
         outs.append((out.clone(), ctx.launch_count() - n1))
-    assert torch.equal(outs[0][0], outs[1][0])
-    assert outs[0][1] < outs[1][1]          # the fused step launches fewer kernels
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[2][0], outs[1][0])
+    assert outs[2][1] < outs[0][1] < outs[1][1]          # each degree of fusion launches fewer kernels
 
 
 # ------------------------------------------------------------------ ablations and shapes of the paper's evaluation
