@@ -562,11 +562,13 @@ def test_exported_state_continues_in_another_context():
         b.import_state(state[:-1])
 
 
-def test_corrupt_installed_selection_is_reported_not_followed():
+@pytest.mark.parametrize("path", ["fused", "kv_gathered_in_kernel"])
+def test_corrupt_installed_selection_is_reported_not_followed(path):
     swam = _swam()
     wl = small()
     x0, x1 = W.generate_steps(wl, 2)
     ctx = swam.Swam.from_workload(wl)
+    ctx.set_option(swam.OPT_SPARSE_PATH, swam.SPARSE_FUSED if path == "fused" else swam.SPARSE_FUSED_KV)
     out = ctx.empty_full().zero_()
     ctx.step(dev(x0["q"], wl), dev(x0["k"], wl), dev(x0["v"], wl), swam.REFRESH_FULL, out)
     before = out.clone()
@@ -632,7 +634,13 @@ def test_grouped_query_schedule_matches_oracle(name, kw):
     wl = W.WORKLOADS[name].with_(steps=3, **kw)
     steps = W.generate_steps(wl)
     ctx = swam.Swam.from_workload(wl)
-    compare_schedule(wl, steps, wl.refresh, run_schedule(ctx, wl, steps, wl.refresh))
+    log = run_schedule(ctx, wl, steps, wl.refresh)
+    compare_schedule(wl, steps, wl.refresh, log)
+    # the sparse path that gathers key and value rows inside the attention kernel reads the narrower K and V too
+    gkv = swam.Swam.from_workload(wl)
+    gkv.set_option(swam.OPT_SPARSE_PATH, swam.SPARSE_FUSED_KV)
+    log_g = run_schedule(gkv, wl, steps, wl.refresh)
+    assert all(np.array_equal(a["out"], b["out"]) for a, b in zip(log, log_g))
     # light refresh and the host-buffer path see the narrower K and V as well
     out = ctx.empty_full().zero_()
     x0, x1 = steps[0], steps[1]
@@ -721,7 +729,7 @@ def test_schedule_with_segment_visibility(wl, sees):
     kc, ks = wl.budgets
     want = ora.run_steps(steps, wl.refresh, wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, kc, ks, sees=sees)
     outs = []
-    for path in (swam.SPARSE_FUSED, swam.SPARSE_STAGED):
+    for path in (swam.SPARSE_FUSED, swam.SPARSE_STAGED, swam.SPARSE_FUSED_KV):
         ctx = swam.Swam.from_workload(wl)
         ctx.set_visibility(*sees)
         ctx.set_option(swam.OPT_SPARSE_PATH, path)
@@ -732,7 +740,7 @@ def test_schedule_with_segment_visibility(wl, sees):
             assert np.array_equal(g["sel"], w["sel_idx"]), (t, w["margins"])
             check_float(g["out"], w["out"], wl.dtype)
         outs.append(log[-1]["out"])
-    assert np.array_equal(outs[0], outs[1])
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[2], outs[1])
 
 
 def test_visibility_option_validation():
