@@ -783,11 +783,14 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         mbar_arrive(bar_s_free(s));   // the scores are in registers: the next key tile's may be written
       }
       const int valid = row_keys - (kv_begin + j) * kTile;  // keys of this tile that this row sees (<= 0: none)
-      if (valid < kTile) {
+      auto mask_tail = [&]() {
+        if (valid < kTile) {
 #pragma unroll
-        for (int c = 0; c < kTile; ++c)
-          if (c >= valid) sv[c] = -INFINITY;
-      }
+          for (int c = 0; c < kTile; ++c)
+            if (c >= valid) sv[c] = -INFINITY;
+        }
+      };
+      mask_tail();
       if (j == 0) {
         // the first tile fixes the reference maximum of the row (tree of independent partial maxima)
         float m8[8];
@@ -843,10 +846,6 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           if ((i & 15) == 15) store_p16(tS, i >> 4, &pk[i - 15]);
         }
       }
-      if constexpr (!C::kPSmem) {
-#pragma unroll
-        for (int c = 0; c < 4; ++c) store_p16(tS, c, &pk[c * 16]);
-      }
       float sum;
       {
         float a0, a1;
@@ -854,7 +853,22 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         sum = a0 + a1;
       }
       const bool grew = !(sum <= 256.f * 128.f);  // some exponent above 2^8 (or 128 of them near it); also catches inf, NaN
-      if (__any_sync(0xffffffffu, grew)) {
+      const bool redo = __any_sync(0xffffffffu, grew);
+      if constexpr (!C::kPSmem) {
+        // P goes over the scores in TMEM only now that the pass is known to stand: the rare redo below reads the
+        // scores again from there, so that they need not stay in registers beside the packed results
+        if (!redo) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) store_p16(tS, c, &pk[c * 16]);
+        }
+      }
+      if (redo) {
+        if constexpr (!C::kPSmem) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<float(*)[32]>(&sv[c * 32]));
+          tmem_ld_wait();
+          mask_tail();
+        }
         // rare: the row's true maximum relative to the reference
         float mraw = sv[0];
 #pragma unroll
