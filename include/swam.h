@@ -12,6 +12,13 @@
  * and swam_destroy (destroys the internal streams and events, if any);
  * swam_bind_host_io creates two internal streams and five events on first use.
  *
+ * Tracing: every call that enqueues work opens an NVTX range named after itself
+ * in the NVTX domain "swam" for the time it spends on the host, and swam_step
+ * opens one more range per stage inside its own ("dense_attention", "swam_score",
+ * "select", "swam_pack", "packed_attention", "swam_scatter"; Sec. 4.2's full and
+ * sparse step).  Without an NVTX tool attached to the process a range costs two
+ * calls of an empty function.
+ *
  * Notation (the paper's): B batch, N_o observed tokens, F future latent frames,
  * N_s tokens per future frame, H action tokens, N_h heads, D head dim,
  * g = H/F queries per frame-aligned group, K = K_c + K_s retained tokens per

@@ -5,6 +5,8 @@
 
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/swam.h"
 #include "swam_internal.cuh"
 
@@ -36,6 +38,29 @@ struct swam_ctx {
 };
 
 namespace {
+
+// Tracing: every call below that launches work opens an NVTX range named after itself in the domain "swam", and
+// swam_step opens one more per stage inside its own, so that a timeline tool shows which kernels belong to which
+// call and stage.  NVTX is header-only; without a tool attached a push or pop is a call through a pointer to an empty
+// function.
+nvtxDomainHandle_t trace_domain() {
+  static nvtxDomainHandle_t dom = nvtxDomainCreateA("swam");
+  return dom;
+}
+struct Range {
+  explicit Range(const char* name) {
+    nvtxEventAttributes_t a;
+    memset(&a, 0, sizeof(a));
+    a.version = NVTX_VERSION;
+    a.size = NVTX_EVENT_ATTRIB_STRUCT_SIZE;
+    a.messageType = NVTX_MESSAGE_TYPE_ASCII;
+    a.message.ascii = name;
+    nvtxDomainRangePushEx(trace_domain(), &a);
+  }
+  ~Range() { nvtxDomainRangePop(trace_domain()); }
+  Range(const Range&) = delete;
+  Range& operator=(const Range&) = delete;
+};
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -207,6 +232,7 @@ int swam_workspace_bytes(const swam_ctx* ctx, size_t* bytes) {
 }
 
 int swam_bind_workspace(swam_ctx* c, void* dev_ptr, size_t bytes) {
+  Range trace_range("swam_bind_workspace");
   if (!c || !dev_ptr) return SWAM_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(dev_ptr) & 255u) != 0) return fail(c, SWAM_ERR_INVALID_ARG, "workspace not 256-byte aligned");
   if (bytes < c->ws_need) return fail(c, SWAM_ERR_WORKSPACE, "workspace too small");
@@ -228,6 +254,7 @@ int swam_host_io_bytes(const swam_ctx* ctx, size_t* bytes) {
 }
 
 int swam_bind_host_io(swam_ctx* c, void* dev_ptr, size_t bytes) {
+  Range trace_range("swam_bind_host_io");
   if (!c || !dev_ptr) return SWAM_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(dev_ptr) & 255u) != 0) return fail(c, SWAM_ERR_INVALID_ARG, "staging not 256-byte aligned");
   if (bytes < c->io_need) return fail(c, SWAM_ERR_WORKSPACE, "staging area too small");
@@ -249,6 +276,7 @@ int swam_bind_host_io(swam_ctx* c, void* dev_ptr, size_t bytes) {
 
 int swam_score(swam_ctx* c, const void* q, const void* k, const float* lse_action, float* scores, float* quality,
                void* stream) {
+  Range trace_range("swam_score");
   if (!c || !q || !k || !scores) return fail(c, SWAM_ERR_INVALID_ARG, "swam_score: null argument");
   if (!aligned16(q) || !aligned16(k) || !aligned16(scores)) return fail(c, SWAM_ERR_INVALID_ARG, "swam_score: misaligned pointer");
   cudaStream_t st = (cudaStream_t)stream;
@@ -273,6 +301,7 @@ int swam_score(swam_ctx* c, const void* q, const void* k, const float* lse_actio
 }
 
 int swam_score_noalloc(swam_ctx* c, const void* q, const void* k, float* scores, void* stream) {
+  Range trace_range("swam_score_noalloc");
   if (!c || !q || !k || !scores) return fail(c, SWAM_ERR_INVALID_ARG, "swam_score_noalloc: null argument");
   if (!aligned16(q) || !aligned16(k) || !aligned16(scores))
     return fail(c, SWAM_ERR_INVALID_ARG, "swam_score_noalloc: misaligned pointer");
@@ -298,6 +327,7 @@ int swam_score_noalloc(swam_ctx* c, const void* q, const void* k, float* scores,
 }
 
 int swam_select(swam_ctx* c, const float* scores, int32_t* sel_idx, int32_t* pack_map, int32_t* inv_map, void* stream) {
+  Range trace_range("swam_select");
   if (!c || !scores) return fail(c, SWAM_ERR_INVALID_ARG, "swam_select: null argument");
   if (int r = need_ws(c)) return r;
   cudaError_t e = launch_select(c->d, scores, nullptr, sel_idx, pack_map, inv_map, (int*)(c->ws + c->off_status),
@@ -309,6 +339,7 @@ int swam_select(swam_ctx* c, const float* scores, int32_t* sel_idx, int32_t* pac
 
 int swam_aggregate(swam_ctx* c, const float* layer_scores, const float* layer_quality, int32_t n_layers, int32_t k_layer,
                    float* v_core, float* v_all, int32_t* core_layers, void* stream) {
+  Range trace_range("swam_aggregate");
   if (!c || !layer_scores || !layer_quality || !v_core || !v_all) return fail(c, SWAM_ERR_INVALID_ARG, "swam_aggregate: null argument");
   if (n_layers <= 0 || k_layer <= 0 || k_layer > n_layers) return fail(c, SWAM_ERR_INVALID_ARG, "swam_aggregate: need 0 < k_layer <= n_layers");
   if (n_layers > max_layers()) return fail(c, SWAM_ERR_UNSUPPORTED, "swam_aggregate: too many layers");
@@ -321,6 +352,7 @@ int swam_aggregate(swam_ctx* c, const float* layer_scores, const float* layer_qu
 
 int swam_select_maps(swam_ctx* c, const float* core_scores, const float* anchor_scores, int32_t* sel_idx, int32_t* pack_map,
                      int32_t* inv_map, void* stream) {
+  Range trace_range("swam_select_maps");
   if (!c || !core_scores || !anchor_scores) return fail(c, SWAM_ERR_INVALID_ARG, "swam_select_maps: null argument");
   if (int r = need_ws(c)) return r;
   cudaError_t e = launch_select(c->d, core_scores, anchor_scores, sel_idx, pack_map, inv_map, (int*)(c->ws + c->off_status),
@@ -332,6 +364,7 @@ int swam_select_maps(swam_ctx* c, const float* core_scores, const float* anchor_
 
 int swam_pack(swam_ctx* c, const void* q, const void* k, const void* v, const int32_t* pack_map, void* qp, void* kp,
               void* vp, void* stream) {
+  Range trace_range("swam_pack");
   if (!c || !pack_map) return fail(c, SWAM_ERR_INVALID_ARG, "swam_pack: null argument");
   if ((!q) != (!qp) || (!k) != (!kp) || (!v) != (!vp)) return fail(c, SWAM_ERR_INVALID_ARG, "swam_pack: unpaired tensor");
   const void* ptrs[6] = {q, k, v, qp, kp, vp};
@@ -348,6 +381,7 @@ int swam_pack(swam_ctx* c, const void* q, const void* k, const void* v, const in
 
 int swam_sparse_attn(swam_ctx* c, const void* qp, const void* kp, const void* vp, int32_t seq_len, void* out_p, float* lse,
                      void* stream) {
+  Range trace_range("swam_sparse_attn");
   if (!c || !qp || !kp || !vp || !out_p) return fail(c, SWAM_ERR_INVALID_ARG, "swam_sparse_attn: null argument");
   if (seq_len <= 0 || seq_len > c->d.L) return fail(c, SWAM_ERR_INVALID_ARG, "swam_sparse_attn: seq_len out of range");
   if (!aligned16(qp) || !aligned16(kp) || !aligned16(vp) || !aligned16(out_p))
@@ -357,6 +391,7 @@ int swam_sparse_attn(swam_ctx* c, const void* qp, const void* kp, const void* vp
 
 int swam_scatter(swam_ctx* c, const void* out_p, const int32_t* pack_map, const int32_t* inv_map, const void* cached,
                  void* out, void* stream) {
+  Range trace_range("swam_scatter");
   if (!c || !out_p || !pack_map || !out || !cached) return fail(c, SWAM_ERR_INVALID_ARG, "swam_scatter: null argument");
   if (cached != out && !inv_map) return fail(c, SWAM_ERR_INVALID_ARG, "swam_scatter: inv_map needed when cached != out");
   if (!aligned16(out_p) || !aligned16(cached) || !aligned16(out)) return fail(c, SWAM_ERR_INVALID_ARG, "swam_scatter: misaligned pointer");
@@ -369,6 +404,7 @@ int swam_scatter(swam_ctx* c, const void* out_p, const int32_t* pack_map, const 
 }
 
 int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t mode, void* out, void* stream) {
+  Range trace_range("swam_step");
   if (!c || !q || !k || !v || !out) return fail(c, SWAM_ERR_INVALID_ARG, "swam_step: null argument");
   if (mode != SWAM_REUSE && mode != SWAM_REFRESH_FULL && mode != SWAM_REFRESH_LIGHT)
     return fail(c, SWAM_ERR_INVALID_ARG, "swam_step: unknown mode");
@@ -388,6 +424,7 @@ int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t 
 
   if (mode == SWAM_REFRESH_FULL) {
     // dense joint attention fills the cache and yields the action-row normalisers over all L keys
+    Range stage("dense_attention");
     if (int r = run_attention(c, q, k, v, d.L, out, lse, d.L - d.H, d.H, st)) return r;
   }
   if (mode != SWAM_REUSE) {
@@ -395,6 +432,7 @@ int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t 
     // the Eq. 9 diagnostics ride along with the selection kernel, which holds the scores in shared memory anyway
     const bool fold = select_can_fold_quality(d);
     if (int r = swam_score(c, q, k, lse_in, scores, fold ? nullptr : quality, stream)) return r;
+    Range stage("select");
     cudaError_t e = launch_select(d, scores, nullptr, sel, pm, im, (int*)(c->ws + c->off_status), st, &c->launches_i,
                                   quality);
     count(c);
@@ -416,6 +454,7 @@ int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t 
       vp = c->ws + c->off_vp;
       if (int r = swam_pack(c, nullptr, k, v, pm, nullptr, c->ws + c->off_kp, c->ws + c->off_vp, stream)) return r;
     }
+    Range stage("packed_attention");
     AttnArgs a{q, kp, vp, out, nullptr, 0, 0, d.B, d.Lp, d.N_h, d.D, d.scale, d.N_kv};
     set_visibility(c, a);
     cudaError_t e = launch_attn_bf16_tc_gather(a, pm, d.L, gather_kv, (int*)(c->ws + c->off_status), c->ws + c->off_attn,
@@ -428,7 +467,10 @@ int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t 
     void* vp = c->ws + c->off_vp;
     void* op = c->ws + c->off_op;
     if (int r = swam_pack(c, q, k, v, pm, qp, kp, vp, stream)) return r;
-    if (int r = run_attention(c, qp, kp, vp, d.Lp, op, nullptr, 0, 0, st)) return r;
+    {
+      Range stage("packed_attention");
+      if (int r = run_attention(c, qp, kp, vp, d.Lp, op, nullptr, 0, 0, st)) return r;
+    }
     if (int r = swam_scatter(c, op, pm, im, out, out, stream)) return r;
   }
   return SWAM_OK;
@@ -436,6 +478,7 @@ int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t 
 
 int swam_step_host(swam_ctx* c, const void* q_host, const void* k_host, const void* v_host, int32_t mode, void* out_host,
                    void* stream) {
+  Range trace_range("swam_step_host");
   if (!c || !q_host || !k_host || !v_host || !out_host) return fail(c, SWAM_ERR_INVALID_ARG, "swam_step_host: null argument");
   if (!c->io) return fail(c, SWAM_ERR_WORKSPACE, "swam_step_host: no staging area bound");
   cudaStream_t st = (cudaStream_t)stream;
@@ -468,6 +511,7 @@ int swam_step_host(swam_ctx* c, const void* q_host, const void* k_host, const vo
 }
 
 int swam_host_join(swam_ctx* c, void* stream) {
+  Range trace_range("swam_host_join");
   if (!c) return SWAM_ERR_INVALID_ARG;
   if (!c->s_in) return fail(c, SWAM_ERR_WORKSPACE, "swam_host_join: no staging area bound");
   cudaError_t e = cudaStreamWaitEvent((cudaStream_t)stream, c->ev_d2h, 0);
@@ -484,6 +528,7 @@ int swam_get_selection(const swam_ctx* c, const int32_t** sel_idx, const int32_t
 }
 
 int swam_set_selection(swam_ctx* c, const int32_t* sel_idx, const int32_t* pack_map, const int32_t* inv_map, void* stream) {
+  Range trace_range("swam_set_selection");
   if (!c || !sel_idx || !pack_map || !inv_map) return fail(c, SWAM_ERR_INVALID_ARG, "swam_set_selection: null argument");
   if (int r = need_ws(c)) return r;
   const Dims& d = c->d;
@@ -507,6 +552,7 @@ int swam_state_bytes(const swam_ctx* c, size_t* bytes) {
 }
 
 int swam_state_export(swam_ctx* c, void* dev_buf, void* stream) {
+  Range trace_range("swam_state_export");
   if (!c || !dev_buf) return fail(c, SWAM_ERR_INVALID_ARG, "swam_state_export: null argument");
   if (int r = need_ws(c)) return r;
   if (!c->has_selection) return fail(c, SWAM_ERR_STATE, "swam_state_export: no refresh step has run yet");
@@ -517,6 +563,7 @@ int swam_state_export(swam_ctx* c, void* dev_buf, void* stream) {
 }
 
 int swam_state_import(swam_ctx* c, const void* dev_buf, void* stream) {
+  Range trace_range("swam_state_import");
   if (!c || !dev_buf) return fail(c, SWAM_ERR_INVALID_ARG, "swam_state_import: null argument");
   if (int r = need_ws(c)) return r;
   cudaError_t e = cudaMemcpyAsync(c->ws + c->off_scores, dev_buf, c->off_scratch - c->off_scores, cudaMemcpyDeviceToDevice,
@@ -535,6 +582,7 @@ int swam_get_scores(const swam_ctx* c, const float** scores, const float** lse_a
 }
 
 int swam_check(swam_ctx* c, void* stream) {
+  Range trace_range("swam_check");
   if (!c) return SWAM_ERR_INVALID_ARG;
   if (int r = need_ws(c)) return r;
   cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
