@@ -20,7 +20,7 @@ struct swam_ctx {
   unsigned char* ws;
   size_t ws_bytes;
   size_t off_status, off_scores, off_quality, off_lse, off_sel, off_pack, off_inv, off_scratch, off_qp, off_kp,
-      off_vp, off_op, off_attn, attn_scratch, ws_need;
+      off_vp, off_op, off_attn, off_logits, off_lam2, off_counters, attn_scratch, ws_need;
   bool has_selection;
   int attn_variant;  // SWAM_ATTN_AUTO | SWAM_ATTN_WARP_MMA
   int sparse_path;   // SWAM_SPARSE_FUSED | SWAM_SPARSE_STAGED
@@ -195,6 +195,7 @@ int swam_create(const swam_shape* s, swam_ctx** out_ctx) {
   size_t off = 0;
   auto put = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   c->off_status = put(256);
+  c->off_counters = put(score_counter_bytes(d));   // directly behind the status word: one memset clears both
   c->off_scores = put((size_t)d.B * d.F * d.N_s * 4);
   c->off_quality = put((size_t)d.B * 3 * 4);
   c->off_lse = put((size_t)d.B * d.N_h * d.H * 4);
@@ -208,6 +209,8 @@ int swam_create(const swam_shape* s, swam_ctx** out_ctx) {
   c->off_op = put(packed_bytes(d));
   c->attn_scratch = (d.dtype == SWAM_BF16 && d.D >= 64) ? attn_tc_scratch_bytes(d.D) : 0;
   c->off_attn = put(c->attn_scratch);
+  c->off_logits = put(score_logits_bytes(d));
+  c->off_lam2 = put((size_t)d.B * d.N_h * d.H * 4);
   c->ws_need = off;
   c->io_need = 7 * align_up(full_bytes(d), 256);
   *out_ctx = c;
@@ -239,7 +242,7 @@ int swam_bind_workspace(swam_ctx* c, void* dev_ptr, size_t bytes) {
   if (int r = check_device(c)) return r;
   cudaError_t e = select_prepare(c->d);
   if (e != cudaSuccess) return fail_cuda(c, e, "select_prepare");
-  e = cudaMemset(dev_ptr, 0, 256);
+  e = cudaMemset(dev_ptr, 0, c->off_counters + score_counter_bytes(c->d));   // status word and arrival tickets
   if (e != cudaSuccess) return fail_cuda(c, e, "cudaMemset(status)");
   c->ws = (unsigned char*)dev_ptr;
   c->ws_bytes = bytes;
@@ -281,19 +284,31 @@ int swam_score(swam_ctx* c, const void* q, const void* k, const float* lse_actio
   if (!aligned16(q) || !aligned16(k) || !aligned16(scores)) return fail(c, SWAM_ERR_INVALID_ARG, "swam_score: misaligned pointer");
   cudaStream_t st = (cudaStream_t)stream;
   const float* lse = lse_action;
-  if (!lse) {
+  if (!lse && score_one_pass_supported(c->d)) {
+    // one pass over the keys: the normalisers' kernel leaves the future keys' products behind and a small second
+    // kernel turns them into scores, instead of a second read of every future key
     if (int r = need_ws(c)) return r;
-    float* own = (float*)(c->ws + c->off_lse);
-    cudaError_t e = launch_action_lse(c->d, q, k, own, c->ws + c->off_scratch, st, &c->launches_i, action_keys(c));
+    cudaError_t e = launch_score_one_pass(c->d, c->alpha, q, k, (float*)(c->ws + c->off_lse), (float*)(c->ws + c->off_lam2),
+                                          c->ws + c->off_scratch, (unsigned int*)(c->ws + c->off_counters),
+                                          (float*)(c->ws + c->off_logits), (int*)(c->ws + c->off_status), scores, st,
+                                          &c->launches_i, action_keys(c));
     count(c);
-    if (e != cudaSuccess) return fail_cuda(c, e, "action lse launch");
-    lse = own;
+    if (e != cudaSuccess) return fail_cuda(c, e, "one-pass score launch");
+  } else {
+    if (!lse) {
+      if (int r = need_ws(c)) return r;
+      float* own = (float*)(c->ws + c->off_lse);
+      cudaError_t e = launch_action_lse(c->d, q, k, own, c->ws + c->off_scratch, st, &c->launches_i, action_keys(c));
+      count(c);
+      if (e != cudaSuccess) return fail_cuda(c, e, "action lse launch");
+      lse = own;
+    }
+    cudaError_t e = launch_score(c->d, c->alpha, q, k, lse, scores, st, &c->launches_i);
+    count(c);
+    if (e != cudaSuccess) return fail_cuda(c, e, "score launch");
   }
-  cudaError_t e = launch_score(c->d, c->alpha, q, k, lse, scores, st, &c->launches_i);
-  count(c);
-  if (e != cudaSuccess) return fail_cuda(c, e, "score launch");
   if (quality) {
-    e = launch_quality(c->d, scores, quality, st, &c->launches_i);
+    cudaError_t e = launch_quality(c->d, scores, quality, st, &c->launches_i);
     count(c);
     if (e != cudaSuccess) return fail_cuda(c, e, "quality launch");
   }
@@ -593,7 +608,8 @@ int swam_check(swam_ctx* c, void* stream) {
   e = cudaMemcpy(&word, c->ws + c->off_status, sizeof(int), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return fail_cuda(c, e, "status read");
   if (word != 0) {
-    e = cudaMemset(c->ws + c->off_status, 0, sizeof(int));
+    // the arrival tickets of the one-pass scorer too: a launch that gave up may have left some behind
+    e = cudaMemset(c->ws + c->off_status, 0, c->off_counters - c->off_status + score_counter_bytes(c->d));
     if (e != cudaSuccess) return fail_cuda(c, e, "status clear");
     snprintf(c->err, sizeof(c->err), "device status word 0x%x%s%s%s", word, (word & ST_BAD_MAP) ? " [map entry out of range]" : "",
              (word & ST_BAD_COUNT) ? " [selection count mismatch]" : "", (word & ST_TIMEOUT) ? " [bounded wait ran out]" : "");

@@ -118,6 +118,19 @@ size_t lse_scratch_bytes(const Dims& d);
 cudaError_t launch_action_lse(const Dims& d, const void* q, const void* k, float* lse, void* scratch,
                               cudaStream_t st, int* launches, int n_keys);
 
+// ---- score_tc.cu ----------------------------------------------------------
+// One pass over the keys for both the normalisers and the scores (bf16, head dim 64 or 128): a tcgen05 kernel streams K
+// once, leaves each key range's (max, sum) per action query in `partial` (lse_scratch_bytes()) and the raw products of
+// every future key with its frame's queries in `logits` (score_logits_bytes()); the last CTA of a head merges the
+// ranges into lambda (`lam2` in the log2 domain and `lse` in natural-log units, both [B,N_h,H]); a second small kernel
+// forms S [B,F,N_s].  `counters` (score_counter_bytes()) must be zero before the first launch and is left zero.
+bool score_one_pass_supported(const Dims& d);
+size_t score_logits_bytes(const Dims& d);
+size_t score_counter_bytes(const Dims& d);
+cudaError_t launch_score_one_pass(const Dims& d, const Alpha& alpha, const void* q, const void* k, float* lse, float* lam2,
+                                  void* partial, unsigned int* counters, float* logits, int* status, float* scores,
+                                  cudaStream_t st, int* launches, int n_keys);
+
 // static device scratch of the allocation-free scoring entry point
 constexpr size_t kStaticScratchBytes = 8u << 20;
 size_t static_scratch_need(const Dims& d);

@@ -158,6 +158,49 @@ def test_normalisers_computed_on_the_device_cover_every_action_row(n_frames, n_a
         assert np.isfinite(g).all() and rel.max() <= SCORE_REL, (name, rel.max())
 
 
+ONE_PASS_CASES = [
+    # the one-pass scorer's branches: copies of the query chunk in the tile (4, 2, 1), more than one chunk, side-output
+    # rows that start off a 16-byte boundary, frames shorter and longer than a key tile, several key ranges per head
+    ("single_view", dict(n_obs=70, grid_h=10, grid_w=9, n_heads=3), None, None),                      # H = 32: 4 copies
+    ("single_view", dict(n_obs=41, grid_h=7, grid_w=9, n_heads=2, batch=2), None, None),              # odd offsets: scalar stores
+    ("single_view", dict(n_obs=600, grid_h=16, grid_w=17, n_heads=2, n_frames=8, n_action=64), None, None),     # H = 64: 2 copies
+    ("larger_imagination", dict(n_obs=300, grid_h=12, grid_w=12, n_heads=2, n_frames=6, n_action=96), None, None),   # H = 96: 1 copy
+    ("larger_imagination", dict(n_obs=64, grid_h=6, grid_w=6, n_heads=2, n_frames=5, n_action=160), None, None),     # two chunks
+    ("larger_imagination", dict(n_obs=40, grid_h=5, grid_w=5, n_heads=3, n_frames=8, n_action=8), [1.0], None),     # g = 1
+    ("single_view", dict(n_obs=128, grid_h=8, grid_w=8, n_heads=4, n_frames=4, n_action=8), [0.25, 0.75], None),    # g = 2
+    ("single_view", dict(n_obs=2000, grid_h=24, grid_w=24, n_heads=4, n_kv_heads=2), None, (0, 1, 1)),               # GQA, action rows do not see action keys
+]
+
+
+@pytest.mark.parametrize("name,kw,alpha,sees", ONE_PASS_CASES,
+                         ids=["h32", "odd_offsets", "h64", "h96", "h160", "g1", "g2", "gqa_no_action_keys"])
+def test_one_pass_scorer_matches_oracle(name, kw, alpha, sees):
+    """swam_score without given normalisers on the tensor-core path: one stream over K yields the normalisers and the
+    future keys' products, a second kernel the scores (Eq. 12); both are compared with the oracle on every element."""
+    swam = _swam()
+    wl = W.WORKLOADS[name].with_(**kw)
+    x = W.generate_steps(wl, 1)[0]
+    kc, ks = wl.budgets
+    ctx = swam.Swam(wl.batch, wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, wl.n_heads, wl.head_dim, kc, ks,
+                    dtype=wl.dtype, n_kv_heads=wl.kv_heads, query_weights=alpha)
+    n_visible = None
+    if sees is not None:
+        ctx.set_visibility(*sees)
+        n_visible = [wl.n_obs, wl.n_obs + wl.n_frames * wl.n_spatial, wl.seq_len][sees[2]]
+    q, k = dev(x["q"], wl), dev(x["k"], wl)
+    k64 = ora.expand_kv(x["k"], wl.n_heads)
+    lse64 = ora.action_lse(x["q"], k64, wl.n_action, n_visible=n_visible)
+    want = ora.score(x["q"], k64, wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, lse=lse64,
+                     alpha=None if alpha is None else np.array(alpha))
+    for rep in range(2):      # the second call finds the arrival tickets as the first one left them
+        got = ctx.score(q, k).cpu().numpy().astype(np.float64)
+        ctx.check()
+        _, lse_dev, _ = ctx.cached_scores()
+        assert np.abs(lse_dev.cpu().numpy() - lse64).max() <= 1e-4, rep
+        rel = np.abs(got - want) / np.maximum(want, 1e-30)
+        assert np.isfinite(got).all() and rel.max() <= SCORE_REL, (rep, rel.max())
+
+
 def test_score_custom_weights():
     swam = _swam()
     wl = small(n_frames=4, n_action=12)                   # g = 3: only valid with explicit weights
