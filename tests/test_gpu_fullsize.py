@@ -149,3 +149,43 @@ def test_attention_is_deterministic_at_full_size():
     for _ in range(5):
         assert torch.equal(first, ctx.sparse_attn(q, k, v))
     ctx.check()
+
+
+@pytest.mark.parametrize("name", ["single_view", "larger_imagination", "multi_view"])
+def test_full_size_light_refresh_matches_oracle(name):
+    """SWAM_REFRESH_LIGHT at the benchmark sizes: the one-pass scorer's normalisers and scores (every element) and
+    the selection and maps built from them against the oracle, then the packed attention's retained rows on a seeded
+    sample and the omitted rows bit for bit."""
+    from paper_2609_38984_b200 import swam
+    wl = W.WORKLOADS[name]
+    kc, ks = wl.budgets
+    x = W.generate_steps(wl, 1)[0]
+    ctx = swam.Swam.from_workload(wl)
+    out = ctx.empty_full()
+    out.copy_(torch.randn(out.shape, device="cuda", generator=torch.Generator(device="cuda").manual_seed(3)).to(out.dtype))
+    before = out.clone()
+    q, k, v = (swam.to_device(x[n], wl.dtype) for n in "qkv")
+    ctx.step(q, k, v, swam.REFRESH_LIGHT, out)
+    ctx.check()
+    sc_dev, lse_dev, _ = ctx.cached_scores()
+    sel_dev, pm_dev, im_dev = (t.cpu().numpy().copy() for t in ctx.selection())
+    lse64 = ora.action_lse(x["q"], x["k"], wl.n_action)
+    assert np.abs(lse_dev.cpu().numpy() - lse64).max() <= 1e-4          # fp32 running sums over bf16 products
+    s64 = ora.score(x["q"], x["k"], wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, lse=lse64)
+    got_s = sc_dev.cpu().numpy()
+    rel = np.abs(got_s - s64) / np.maximum(s64, 1e-30)
+    assert np.isfinite(got_s).all() and rel.max() <= 1e-5, rel.max()
+    iso = ora.select(got_s, kc, ks)
+    ipm, iim = ora.maps(iso["sel_idx"], wl.n_obs, wl.n_spatial, wl.n_action)
+    assert np.array_equal(sel_dev, iso["sel_idx"]) and np.array_equal(pm_dev, ipm) and np.array_equal(im_dev, iim)
+    e2e = ora.select(s64.astype(np.float32), kc, ks)
+    assert np.array_equal(sel_dev, e2e["sel_idx"]), ("cut margins", e2e["margins"], "score rel err", rel.max())
+    omitted = torch.from_numpy(im_dev < 0).cuda()
+    assert torch.equal(out[omitted], before[omitted])
+    qp, kp, vp = (ora.pack(x[n], pm_dev) for n in "qkv")
+    rng = np.random.default_rng(11)
+    rows = sample_rows(rng, wl.batch, wl.packed_len, 40, extra=range(wl.packed_len - wl.n_action, wl.packed_len, 8))
+    want, _ = ora.attention_rows(qp, kp, vp, rows)
+    orig = pm_dev[rows[:, 0], rows[:, 1]]
+    got = out[rows[:, 0], orig].float().cpu().numpy().astype(np.float64)
+    check_bf16(got, want)
