@@ -10,7 +10,7 @@
  * host: swam_bind_workspace (one small synchronous cudaMemset of the status
  * word), swam_check (synchronises the stream and the internal copy streams)
  * and swam_destroy (destroys the internal streams and events, if any);
- * swam_bind_host_io creates two internal streams and five events on first use.
+ * swam_bind_host_io creates two internal streams and six events on first use.
  *
  * Tracing: every call that enqueues work opens an NVTX range named after itself
  * in the NVTX domain "swam" for the time it spends on the host, and swam_step
@@ -239,8 +239,15 @@ int swam_launch_floor(swam_ctx* ctx, void* stream);
  * at least the future tokens (they score them).  The setting applies to swam_step, to swam_sparse_attn at the full
  * and the packed length (segment boundaries N_o and N_o + F*N_s, or N_o and N_o + F*K; other lengths return
  * SWAM_ERR_UNSUPPORTED unless visibility is full) and to the normalisers swam_score computes, which then run over the
- * keys the action rows see. */
-enum { SWAM_OPT_ATTN_VARIANT = 1, SWAM_OPT_SPARSE_PATH = 2, SWAM_OPT_VISIBILITY = 3 };
+ * keys the action rows see.
+ *
+ * SWAM_OPT_HOST_ROWS selects what a SWAM_REUSE step of swam_step_host brings across PCIe: SWAM_HOST_ROWS_RETAINED
+ * (default) only the rows the cached maps retain (Sec. 4.2: the sparse step processes the compact sequence), fetched
+ * by a kernel on the library's copy-in stream straight from the caller's buffers, which must then be pinned memory
+ * the device can address (cudaHostAlloc / cudaHostRegister); buffers that are not are copied whole, as with
+ * SWAM_HOST_ROWS_ALL.  The result is the same either way. */
+enum { SWAM_OPT_ATTN_VARIANT = 1, SWAM_OPT_SPARSE_PATH = 2, SWAM_OPT_VISIBILITY = 3, SWAM_OPT_HOST_ROWS = 4 };
+enum { SWAM_HOST_ROWS_RETAINED = 0, SWAM_HOST_ROWS_ALL = 1 };
 enum { SWAM_ATTN_AUTO = 0, SWAM_ATTN_WARP_MMA = 1 };
 enum { SWAM_SPARSE_FUSED = 0, SWAM_SPARSE_STAGED = 1, SWAM_SPARSE_FUSED_KV = 2 };
 enum { SWAM_SEES_OBSERVED = 0, SWAM_SEES_FUTURE = 1, SWAM_SEES_ALL = 2 };

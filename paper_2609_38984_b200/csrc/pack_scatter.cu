@@ -223,6 +223,76 @@ cudaError_t launch_pack(const Dims& d, const void* const src[3], void* const dst
   return cudaSuccess;
 }
 
+// Sparse input transfer of a reuse step (Sec. 4.2: only the retained tokens are processed): the rows pack_map names
+// travel from full tensors in pinned, device-mapped HOST memory to the same rows of full tensors in device memory;
+// every other row of the destination keeps what it held and is never read by the sparse step.  The loads cross PCIe
+// (one warp per row, eight 16-byte loads per lane in flight), so the kernel is the copy: it runs on the copy-in stream.
+struct HostRowsParams {
+  const uint4* src[3];
+  uint4* dst[3];
+  const int32_t* idx;   // [B, n_idx] rows to bring
+  int* status;
+  int n_tensors, n_idx, rows, chunks;   // rows per sample of the full tensors, 16-byte chunks per row
+  long long total;                      // B * n_idx
+};
+
+__global__ void __launch_bounds__(256) host_rows_kernel(const HostRowsParams p) {
+  const int lane = threadIdx.x & 31;
+  const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long it = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; it < p.total; it += n_warps) {
+    const long long b = it / p.n_idx;
+    const int row = p.idx[it];
+    if (row < 0 || row >= p.rows) {
+      if (lane == 0) atomicOr(p.status, ST_BAD_MAP);
+      continue;
+    }
+    const long long off = (b * p.rows + row) * p.chunks;
+    for (int t = 0; t < p.n_tensors; ++t) {
+      const uint4* s = p.src[t] + off;
+      uint4* d = p.dst[t] + off;
+      for (int c0 = lane; c0 < p.chunks; c0 += 32 * 8) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          if (c0 + 32 * u < p.chunks) v[u] = __ldcs(s + c0 + 32 * u);
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          if (c0 + 32 * u < p.chunks) d[c0 + 32 * u] = v[u];
+      }
+    }
+  }
+}
+
+cudaError_t launch_host_rows(const Dims& d, const void* const src[3], void* const dst[3], const int32_t* pack_map,
+                             int* status, cudaStream_t st, int* launches) {
+  if (d.Lp == 0) return cudaSuccess;
+  const int eb = d.dtype == 0 ? 4 : 2;
+  const int rows_of[3] = {d.N_h * d.D * eb, d.N_kv * d.D * eb, d.N_kv * d.D * eb};
+  bool done[3] = {false, false, false};
+  for (int first = 0; first < 3; ++first) {
+    if (done[first]) continue;
+    HostRowsParams p{};
+    int n = 0;
+    for (int i = first; i < 3; ++i)
+      if (!done[i] && rows_of[i] == rows_of[first]) {
+        p.src[n] = (const uint4*)src[i];
+        p.dst[n] = (uint4*)dst[i];
+        ++n;
+        done[i] = true;
+      }
+    p.idx = pack_map; p.status = status;
+    p.n_tensors = n; p.n_idx = d.Lp; p.rows = d.L; p.chunks = rows_of[first] / 16;
+    p.total = (long long)d.B * d.Lp;
+    ++*launches;
+    const long long need = (p.total + 7) / 8;
+    const long long cap = (long long)sm_count() * 8;
+    host_rows_kernel<<<(int)(need < cap ? need : cap), 256, 0, st>>>(p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
 cudaError_t launch_scatter(const Dims& d, const void* out_p, const int32_t* pack_map, const int32_t* inv_map,
                            const void* cached, void* out, int* status, cudaStream_t st, int* launches) {
   const int row_bytes = d.N_h * d.D * (d.dtype == 0 ? 4 : 2);

@@ -24,13 +24,16 @@ struct swam_ctx {
   bool has_selection;
   int attn_variant;  // SWAM_ATTN_AUTO | SWAM_ATTN_WARP_MMA
   int sparse_path;   // SWAM_SPARSE_FUSED | SWAM_SPARSE_STAGED
+  int host_rows;     // SWAM_HOST_ROWS_RETAINED | SWAM_HOST_ROWS_ALL: what a reuse step with host buffers brings in
   int sees[3];       // what observed / future / action rows see: SWAM_SEES_*
   // host-io staging (device): two input slots of (q, k, v) and the persistent output, plus the copy pipeline
   unsigned char* io;
   size_t io_need;
   cudaStream_t s_in, s_out;           // host-to-device and device-to-host copy streams
-  cudaEvent_t ev_h2d[2], ev_done[2];  // per input slot: inputs arrived / step finished with the slot
+  cudaStream_t s_rows;                // the retained-row fetches of reuse steps (they wait for the maps; whole copies need not)
+  cudaEvent_t ev_h2d[3], ev_done[3];  // per input slot: inputs arrived / step finished with the slot
   cudaEvent_t ev_d2h;                 // the previous result has left the staged output
+  cudaEvent_t ev_pre;                 // everything the caller's stream held when a reuse step with host buffers was called
   int64_t host_steps;
   int launches_i;
   int64_t launches;
@@ -212,7 +215,7 @@ int swam_create(const swam_shape* s, swam_ctx** out_ctx) {
   c->off_logits = put(score_logits_bytes(d));
   c->off_lam2 = put((size_t)d.B * d.N_h * d.H * 4);
   c->ws_need = off;
-  c->io_need = 7 * align_up(full_bytes(d), 256);
+  c->io_need = 10 * align_up(full_bytes(d), 256);   // three input slots of (q, k, v) and the staged output
   *out_ctx = c;
   return SWAM_OK;
 }
@@ -220,9 +223,11 @@ int swam_create(const swam_shape* s, swam_ctx** out_ctx) {
 int swam_destroy(swam_ctx* ctx) {
   if (ctx && ctx->s_in) {
     cudaStreamDestroy(ctx->s_in);
+    cudaStreamDestroy(ctx->s_rows);
     cudaStreamDestroy(ctx->s_out);
-    for (int i = 0; i < 2; ++i) { cudaEventDestroy(ctx->ev_h2d[i]); cudaEventDestroy(ctx->ev_done[i]); }
+    for (int i = 0; i < 3; ++i) { cudaEventDestroy(ctx->ev_h2d[i]); cudaEventDestroy(ctx->ev_done[i]); }
     cudaEventDestroy(ctx->ev_d2h);
+    cudaEventDestroy(ctx->ev_pre);
   }
   delete ctx;
   return SWAM_OK;
@@ -265,11 +270,13 @@ int swam_bind_host_io(swam_ctx* c, void* dev_ptr, size_t bytes) {
   if (!c->s_in) {
     cudaError_t e = cudaStreamCreateWithFlags(&c->s_in, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->s_out, cudaStreamNonBlocking);
-    for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->s_rows, cudaStreamNonBlocking);
+    for (int i = 0; i < 3 && e == cudaSuccess; ++i) {
       e = cudaEventCreateWithFlags(&c->ev_h2d[i], cudaEventDisableTiming);
       if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_done[i], cudaEventDisableTiming);
     }
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_d2h, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_pre, cudaEventDisableTiming);
     if (e != cudaSuccess) return fail_cuda(c, e, "swam_bind_host_io: stream/event creation");
   }
   c->io = (unsigned char*)dev_ptr;
@@ -498,20 +505,53 @@ int swam_step_host(swam_ctx* c, const void* q_host, const void* k_host, const vo
   if (!c->io) return fail(c, SWAM_ERR_WORKSPACE, "swam_step_host: no staging area bound");
   cudaStream_t st = (cudaStream_t)stream;
   const size_t fb = full_bytes(c->d), kvb = kv_full_bytes(c->d), stride = align_up(fb, 256);
-  // Three-stage pipeline over two input slots: this step's inputs travel on the copy-in stream while the previous
-  // step still computes, the step runs on the caller's stream, and the result leaves on the copy-out stream while
-  // the next inputs arrive (PCIe is full duplex).
-  const int slot = (int)(c->host_steps & 1);
+  // Three-stage pipeline over three input slots: this step's inputs travel on a copy-in stream while the previous
+  // steps still compute, the step runs on the caller's stream, and the result leaves on the copy-out stream while
+  // the next inputs arrive (PCIe is full duplex).  The third slot lets the whole-tensor copy of the refresh step after
+  // a reuse step start while the refresh step before it still computes (the reuse step's own rows cannot: they are
+  // only known once that step has rebuilt the maps), so the host-to-device link never idles.
+  const int slot = (int)(c->host_steps % 3);
   unsigned char* in = c->io + (size_t)slot * 3 * stride;
   void* dq = in;
   void* dk = in + stride;
   void* dv = in + 2 * stride;
-  void* dout = c->io + 6 * stride;
-  cudaError_t e = cudaStreamWaitEvent(c->s_in, c->ev_done[slot], 0);   // the step two calls ago has read this slot
-  if (e == cudaSuccess) e = cudaMemcpyAsync(dq, q_host, fb, cudaMemcpyHostToDevice, c->s_in);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(dk, k_host, kvb, cudaMemcpyHostToDevice, c->s_in);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v_host, kvb, cudaMemcpyHostToDevice, c->s_in);
-  if (e == cudaSuccess) e = cudaEventRecord(c->ev_h2d[slot], c->s_in);
+  void* dout = c->io + 9 * stride;
+  // A reuse step reads only the rows its maps retain: where the caller's buffers are pinned memory the device can
+  // address, a kernel on the row-fetch stream brings just those rows across PCIe (Sec. 4.2's compact execution applied
+  // to the transfer as well); the other rows of the slot keep stale values that the sparse step never touches.
+  const void* mapped[3] = {nullptr, nullptr, nullptr};
+  bool retained_only = mode == SWAM_REUSE && c->has_selection && c->host_rows == SWAM_HOST_ROWS_RETAINED && c->ws;
+  if (retained_only) {
+    const void* host[3] = {q_host, k_host, v_host};
+    for (int i = 0; i < 3 && retained_only; ++i) {
+      cudaPointerAttributes at;
+      if (cudaPointerGetAttributes(&at, host[i]) != cudaSuccess || at.type != cudaMemoryTypeHost || !at.devicePointer) {
+        cudaGetLastError();          // pageable or foreign memory: plain copies of the whole tensors below
+        retained_only = false;
+      } else {
+        mapped[i] = at.devicePointer;
+      }
+    }
+  }
+  cudaStream_t s_copy = retained_only ? c->s_rows : c->s_in;
+  cudaError_t e = cudaStreamWaitEvent(s_copy, c->ev_done[slot], 0);   // the step three calls ago has read this slot
+  if (retained_only) {
+    // the maps are final once everything already on the caller's stream has run (the previous step, or a selection
+    // installed since)
+    if (e == cudaSuccess) e = cudaEventRecord(c->ev_pre, st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s_copy, c->ev_pre, 0);
+    if (e == cudaSuccess) {
+      void* dst[3] = {dq, dk, dv};
+      e = launch_host_rows(c->d, mapped, dst, (const int32_t*)(c->ws + c->off_pack), (int*)(c->ws + c->off_status), s_copy,
+                           &c->launches_i);
+      count(c);
+    }
+  } else {
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dq, q_host, fb, cudaMemcpyHostToDevice, s_copy);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dk, k_host, kvb, cudaMemcpyHostToDevice, s_copy);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dv, v_host, kvb, cudaMemcpyHostToDevice, s_copy);
+  }
+  if (e == cudaSuccess) e = cudaEventRecord(c->ev_h2d[slot], s_copy);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_h2d[slot], 0);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(st, c->ev_d2h, 0);     // the previous result has been copied out
   if (e != cudaSuccess) return fail_cuda(c, e, "host to device copy");
@@ -602,6 +642,7 @@ int swam_check(swam_ctx* c, void* stream) {
   if (int r = need_ws(c)) return r;
   cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
   if (e == cudaSuccess && c->s_in) e = cudaStreamSynchronize(c->s_in);
+  if (e == cudaSuccess && c->s_rows) e = cudaStreamSynchronize(c->s_rows);
   if (e == cudaSuccess && c->s_out) e = cudaStreamSynchronize(c->s_out);
   if (e != cudaSuccess) return fail_cuda(c, e, "cudaStreamSynchronize");
   int word = 0;
@@ -651,6 +692,10 @@ int swam_set_option(swam_ctx* c, int32_t option, int32_t value) {
     if (f < SWAM_SEES_FUTURE || a < SWAM_SEES_FUTURE)
       return fail(c, SWAM_ERR_INVALID_ARG, "swam_set_option: future and action rows must see the future tokens");
     c->sees[0] = o; c->sees[1] = f; c->sees[2] = a;
+    return SWAM_OK;
+  }
+  if (option == SWAM_OPT_HOST_ROWS && (value == SWAM_HOST_ROWS_RETAINED || value == SWAM_HOST_ROWS_ALL)) {
+    c->host_rows = value;
     return SWAM_OK;
   }
   if (option == SWAM_OPT_SPARSE_PATH &&

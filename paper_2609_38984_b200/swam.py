@@ -20,7 +20,8 @@ LIB_PATH = os.path.join(_HERE, "libswam.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_STATE, ERR_CUDA, ERR_DEVICE_CHECK, ERR_TIMEOUT = range(8)
 F32, BF16 = 0, 1
 REUSE, REFRESH_FULL, REFRESH_LIGHT = 0, 1, 2
-OPT_ATTN_VARIANT, OPT_SPARSE_PATH, OPT_VISIBILITY = 1, 2, 3
+OPT_ATTN_VARIANT, OPT_SPARSE_PATH, OPT_VISIBILITY, OPT_HOST_ROWS = 1, 2, 3, 4
+HOST_ROWS_RETAINED, HOST_ROWS_ALL = 0, 1
 SEES_OBSERVED, SEES_FUTURE, SEES_ALL = 0, 1, 2
 ATTN_AUTO, ATTN_WARP_MMA = 0, 1
 SPARSE_FUSED, SPARSE_STAGED, SPARSE_FUSED_KV = 0, 1, 2

@@ -847,15 +847,21 @@ def test_host_buffer_step_matches_device_step():
         assert torch.equal(out_dev.cpu(), out_host)
 
 
-def test_host_buffer_steps_pipeline_without_synchronising_in_between():
+@pytest.mark.parametrize("rows", ["retained", "all", "pageable"])
+def test_host_buffer_steps_pipeline_without_synchronising_in_between(rows):
+    """Five calls enqueued back to back; the reuse steps bring only the retained rows across PCIe (the default, from
+    pinned buffers), whole tensors on request, and whole tensors when the buffers are pageable: same bits each way."""
     swam = _swam()
     wl = small(steps=5)
     steps = W.generate_steps(wl)
     ctx_a, ctx_b = swam.Swam.from_workload(wl), swam.Swam.from_workload(wl)
     out_dev = ctx_a.empty_full()
     tdt = out_dev.dtype
-    host_in = [[torch.from_numpy(x[n]).to(tdt).pin_memory() for n in "qkv"] for x in steps]
+    pin = (lambda t: t) if rows == "pageable" else (lambda t: t.pin_memory())
+    host_in = [[pin(torch.from_numpy(x[n]).to(tdt)) for n in "qkv"] for x in steps]
     host_out = [torch.empty(out_dev.shape, dtype=tdt).pin_memory() for _ in steps]
+    if rows == "all":
+        ctx_b.set_option(swam.OPT_HOST_ROWS, swam.HOST_ROWS_ALL)
     want = []
     for t, (hq, hk, hv) in enumerate(host_in):
         mode = swam.REFRESH_FULL if t % 2 == 0 else swam.REUSE
