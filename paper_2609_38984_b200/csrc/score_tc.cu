@@ -6,13 +6,16 @@
 // both: the products of a tile of keys against all action queries of a head are one tensor-core instruction chain,
 // their running (max, sum) per query is the normaliser's share of this key range, and the g products per future key
 // that Eq. 12 uses are stored raw (fp32) beside it.  A second, small kernel then forms
-//   S(f, j) = 1/N_h sum_h sum_i w_i exp2(scale log2e x[h, j, i] - lambda2[h, i])
+//   S(f, j) = 1/N_h sum_h sum_i w_i exp2(scale log2e x[h, i, j] - lambda2[h, i])
 // from 4 g bytes per (head, key) instead of a second read of the 2 D bytes of the key row.
 //
 // lse_tc_kernel: CTA = (range of key tiles, head, sample x chunk of <= 128 action queries), two CTAs per SM.
-//   warp 4      TMA producer: the query tile once, then key tiles of 16 KB into a ring of four stages
-//   warp 5      one elected thread issues S = Q K_j^T (M = 128, N = keys per tile) into one of two TMEM buffers
-//   warps 0-3   statistics: thread = TMEM lane = row of S; running maximum and sum in the log2 domain; side output
+//   warp 8      TMA producer: the query tile once, then key tiles of 16 KB into a ring of four stages (marked as the
+//               first lines to leave L2, so that the side output is still there when the second kernel reads it)
+//   warp 9      one elected thread issues S = Q K_j^T (M = 128, N = keys per tile) into one of two TMEM buffers
+//   warps 0-7   statistics, two groups of four that take alternate tiles (a tile's pass is longer than the tile's
+//               share of the stream): thread = TMEM lane = row of S; running maximum and sum in the log2 domain; the
+//               products of the keys of the row's own frame go to the row's line of the [head][query][future key] block
 // The action queries of a head are few (H = 32 in the paper's set-ups), so the 128 rows of the query tile hold the
 // H queries 128 / Hpad times over (Hpad = 32, 64 or 128) and the copies split a tile's key columns among them: every
 // warp then has a full set of 32 useful rows and all four exp2 units work.  The last CTA to finish a (sample, head,
