@@ -225,12 +225,6 @@ __global__ void __launch_bounds__(kQualThreads) quality_kernel(const float* scor
 // [B, ranges, N_h, H]; a second kernel merges the ranges.  The scratch holds one range per 128 keys at most.
 constexpr int kLseKeys = 128;
 
-__device__ __forceinline__ void merge_ms(float& m, float& s, float m2, float s2) {
-  const float mn = fmaxf(m, m2);
-  if (mn == -INFINITY) { m = mn; s = 0.f; return; }
-  s = s * exp2f(m - mn) + s2 * exp2f(m2 - mn);
-  m = mn;
-}
 
 // ---------------------------------------------------------------------------------------------------------
 // lambda over all L keys, flash style (the first half of an attention step: scores and running row statistics,

@@ -42,13 +42,6 @@ struct LtParams {
   float scale_log2;
 };
 
-__device__ __forceinline__ void merge_ms2(float& m, float& s, float m2, float s2) {
-  const float mn = fmaxf(m, m2);
-  if (mn == -INFINITY) { m = mn; s = 0.f; return; }
-  s = s * exp2f(m - mn) + s2 * exp2f(m2 - mn);
-  m = mn;
-}
-
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
   uint32_t r[16];
   asm volatile(
@@ -282,7 +275,7 @@ lse_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   if (tid < HP && qc * HP + tid < p.H) {
     float m = -INFINITY, l = 0.f;
 #pragma unroll
-    for (int sh = 0; sh < 2 * REP; ++sh) merge_ms2(m, l, s_red[sh * HP + tid].x, s_red[sh * HP + tid].y);
+    for (int sh = 0; sh < 2 * REP; ++sh) merge_ms(m, l, s_red[sh * HP + tid].x, s_red[sh * HP + tid].y);
     p.partial[((int64_t)b * p.n_splits + split) * row_stride + (int64_t)h * p.H + qc * HP + tid] = make_float2(m, l);
     __threadfence();
   }
@@ -300,14 +293,14 @@ lse_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     for (; c + 4 <= p.n_splits; c += 4) {
       const float2 a0 = __ldcg(src + (int64_t)c * row_stride), a1 = __ldcg(src + (int64_t)(c + 1) * row_stride);
       const float2 a2 = __ldcg(src + (int64_t)(c + 2) * row_stride), a3 = __ldcg(src + (int64_t)(c + 3) * row_stride);
-      merge_ms2(m, l, a0.x, a0.y);
-      merge_ms2(m, l, a1.x, a1.y);
-      merge_ms2(m, l, a2.x, a2.y);
-      merge_ms2(m, l, a3.x, a3.y);
+      merge_ms(m, l, a0.x, a0.y);
+      merge_ms(m, l, a1.x, a1.y);
+      merge_ms(m, l, a2.x, a2.y);
+      merge_ms(m, l, a3.x, a3.y);
     }
     for (; c < p.n_splits; ++c) {
       const float2 a = __ldcg(src + (int64_t)c * row_stride);
-      merge_ms2(m, l, a.x, a.y);
+      merge_ms(m, l, a.x, a.y);
     }
     const float l2 = m + log2f(l);
     const int64_t o = ((int64_t)b * p.N_h + h) * p.H + qc * HP + tid;

@@ -97,6 +97,14 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
   }
 }
 
+// (max, sum) pairs of a log-sum-exp in the log2 domain: folds (m2, s2) into (m, s); an empty pair is (-inf, 0)
+__device__ __forceinline__ void merge_ms(float& m, float& s, float m2, float s2) {
+  const float mn = fmaxf(m, m2);
+  if (mn == -INFINITY) { m = mn; s = 0.f; return; }
+  s = s * exp2f(m - mn) + s2 * exp2f(m2 - mn);
+  m = mn;
+}
+
 // SMs of the current device (queried on every call: a process may hold contexts on several devices)
 inline int sm_count() {
   int dev = 0, sms = 0;
