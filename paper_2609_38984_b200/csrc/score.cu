@@ -46,6 +46,7 @@ struct ScoreParams {
   float scale_log2, inv_nh;
   Alpha alpha;
   int N_kv;          // heads of k; query head h reads key head h / (N_h / N_kv)
+  int keys_per_cta;  // keys of a frame per CTA (<= 16 * MT; fewer leaves the last 16-key tile partly empty)
 };
 
 
@@ -62,7 +63,8 @@ __global__ void __launch_bounds__(32 * MT * kHeadGroups, 16 / (MT * kHeadGroups)
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int f = blockIdx.y, b = blockIdx.z;
-  const int key0 = blockIdx.x * kScoreKeys;
+  const int key0 = blockIdx.x * p.keys_per_cta;
+  const int key_end = min(p.N_s, key0 + p.keys_per_cta);
   const int64_t act0 = (int64_t)p.n_obs + (int64_t)p.F * p.N_s;
   const int64_t tok = (int64_t)p.N_h * D;
 
@@ -90,7 +92,7 @@ __global__ void __launch_bounds__(32 * MT * kHeadGroups, 16 / (MT * kHeadGroups)
   const int mt = warp % MT, hg = warp / MT;
   const int gq = lane >> 2, t = lane & 3;
   const int r0 = key0 + mt * 16 + gq, r1 = r0 + 8;
-  const bool v0 = r0 < p.N_s, v1 = r1 < p.N_s;
+  const bool v0 = r0 < key_end, v1 = r1 < key_end;
   const int64_t tok_k = (int64_t)p.N_kv * D;
   const int kv_group = p.N_h / p.N_kv;
   const __nv_bfloat16* kbase = p.k + ((int64_t)b * p.L + p.n_obs + (int64_t)f * p.N_s) * tok_k + t * 8;
@@ -161,7 +163,7 @@ __global__ void __launch_bounds__(32 * MT * kHeadGroups, 16 / (MT * kHeadGroups)
     red[hg * kScoreKeys + mt * 16 + gq + 8] = sum1;
   }
   __syncthreads();
-  if (tid < kScoreKeys && key0 + tid < p.N_s) {
+  if (tid < kScoreKeys && key0 + tid < key_end) {
     float s = 0.f;
 #pragma unroll
     for (int q = 0; q < kHeadGroups; q += 4)
@@ -438,7 +440,7 @@ __global__ void __launch_bounds__(128) lse_f32_kernel(const float* q, const floa
 }
 
 template <int D, int NT, int HG, int MT>
-cudaError_t launch_score_bf16_hg(const Dims& d, const ScoreParams& p, cudaStream_t st) {
+cudaError_t launch_score_bf16_hg(const Dims& d, ScoreParams p, cudaStream_t st, int keys_per_cta) {
   constexpr int kScoreKeys = 16 * MT;
   const size_t smem = (size_t)d.N_h * (D / 32) * NT * 32 * sizeof(uint4) + (size_t)d.N_h * NT * 8 * sizeof(float) +
                       HG * kScoreKeys * sizeof(float);
@@ -446,19 +448,27 @@ cudaError_t launch_score_bf16_hg(const Dims& d, const ScoreParams& p, cudaStream
   cudaError_t e = cudaFuncSetAttribute(score_bf16_kernel<D, NT, HG, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  dim3 grid((d.N_s + kScoreKeys - 1) / kScoreKeys, d.F, d.B);
+  p.keys_per_cta = keys_per_cta;
+  dim3 grid((d.N_s + keys_per_cta - 1) / keys_per_cta, d.F, d.B);
   score_bf16_kernel<D, NT, HG, MT><<<grid, 32 * MT * HG, smem, st>>>(p);
   return cudaGetLastError();
 }
 
 template <int D, int NT>
 cudaError_t launch_score_bf16(const Dims& d, const ScoreParams& p, cudaStream_t st) {
-  // 32 keys per CTA, except when that gives between one and two CTAs per SM: then 64-key CTAs (one per SM, half the
-  // query-fragment staging) finish sooner
+  // 32 keys per CTA, except when that gives between one and two CTAs per SM: then one wave of larger CTAs (half the
+  // query-fragment staging) finishes sooner, and the frame is cut into as many equal pieces of at most 64 keys as
+  // fill the SMs (a piece of 57 keys leaves its last 16-key tile partly empty, which costs nothing: the kernel is
+  // bound by the loads)
   const int sms = sm_count();
   const long long n32 = (long long)((d.N_s + 31) / 32) * d.F * d.B;
-  if (n32 > sms && n32 <= 2 * sms) return launch_score_bf16_hg<D, NT, 4, 4>(d, p, st);
-  return launch_score_bf16_hg<D, NT, 4, 2>(d, p, st);
+  if (n32 > sms && n32 <= 2 * sms) {
+    const int pieces = sms / (d.F * d.B);                       // per frame
+    int keys = pieces > 0 ? (d.N_s + pieces - 1) / pieces : 64;
+    if (keys > 64 || keys < 33) keys = 64;
+    return launch_score_bf16_hg<D, NT, 4, 4>(d, p, st, keys);
+  }
+  return launch_score_bf16_hg<D, NT, 4, 2>(d, p, st, 32);
 }
 
 template <int D>
@@ -485,7 +495,7 @@ cudaError_t launch_score(const Dims& d, const Alpha& alpha, const void* q, const
     return cudaGetLastError();
   }
   ScoreParams p{(const __nv_bfloat16*)q, (const __nv_bfloat16*)k, lse, scores, d.n_obs, d.F, d.N_s, d.H,
-                d.N_h, d.L, d.g, d.scale * kLog2e, 1.0f / (float)d.N_h, alpha, d.N_kv};
+                d.N_h, d.L, d.g, d.scale * kLog2e, 1.0f / (float)d.N_h, alpha, d.N_kv, 32};
   switch (d.D) {
     case 32: return launch_score_bf16_d<32>(d, p, st);
     case 64: return launch_score_bf16_d<64>(d, p, st);
