@@ -162,8 +162,10 @@ int swam_step(swam_ctx* ctx, const void* q, const void* k, const void* v, int32_
  * and does not synchronise: q, k, v travel to a device staging slot on an internal copy stream, swam_step runs on
  * `stream`, and out leaves for out_host on a second internal copy stream, so that consecutive calls overlap one
  * step's copies with the neighbouring steps' compute and the two PCIe directions with each other.  The staging area
- * (7 full tensors: two input slots and the persistent out; caller-allocated, dev) is bound once; binding creates the
- * internal streams and events.  The host input buffers of a call must stay unchanged, and out_host is complete,
+ * (10 full tensors: three input slots and the persistent out; caller-allocated, dev) is bound once; binding creates the
+ * internal streams and events.  A SWAM_REUSE step brings only the rows its maps retain across PCIe when the host
+ * buffers are pinned memory the device can address (see SWAM_OPT_HOST_ROWS); a kernel then reads the caller's
+ * buffers directly.  The host input buffers of a call must stay unchanged, and out_host is complete,
  * once swam_check (which also waits for the internal streams) or a device-wide synchronisation has returned.  On
  * SWAM_REUSE steps the staged out of the previous step is the cache, so the staging area must not be touched between
  * steps.  Not capturable in a CUDA graph. */
