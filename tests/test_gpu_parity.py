@@ -192,9 +192,15 @@ def test_one_pass_scorer_matches_oracle(name, kw, alpha, sees):
     lse64 = ora.action_lse(x["q"], k64, wl.n_action, n_visible=n_visible)
     want = ora.score(x["q"], k64, wl.n_obs, wl.n_frames, wl.n_spatial, wl.n_action, lse=lse64,
                      alpha=None if alpha is None else np.array(alpha))
+    first = None
     for rep in range(2):      # the second call finds the arrival tickets as the first one left them
-        got = ctx.score(q, k).cpu().numpy().astype(np.float64)
+        got_t = ctx.score(q, k)
+        got = got_t.cpu().numpy().astype(np.float64)
         ctx.check()
+        if first is None:
+            first = got_t.clone()
+        else:
+            assert torch.equal(first, got_t)      # same bits whatever order the key ranges finish in
         _, lse_dev, _ = ctx.cached_scores()
         assert np.abs(lse_dev.cpu().numpy() - lse64).max() <= 1e-4, rep
         rel = np.abs(got - want) / np.maximum(want, 1e-30)
