@@ -76,7 +76,8 @@ typedef struct {
  * same shape. */
 
 /* Context: validates the shape (H divisible by F, Eq. 8; K_c + K_s <= N_s; head_dim in {32, 64, 128};
- * NULL weights need H/F divisible by 4) and fixes the workspace layout.  The shape (and the weights) are
+ * NULL weights need H/F divisible by 4; at most 65535 samples, half of that with more than 128 action tokens; L at most
+ * 2^24 and B*L at most 2^30: SWAM_ERR_UNSUPPORTED beyond) and fixes the workspace layout.  The shape (and the weights) are
  * copied.  The current CUDA device at creation is the device every later call must run on. */
 int swam_create(const swam_shape* shape, swam_ctx** out_ctx);
 int swam_destroy(swam_ctx* ctx);

@@ -167,6 +167,8 @@ int swam_create(const swam_shape* s, swam_ctx** out_ctx) {
   if (!s->query_weights && (g % 4) != 0) return SWAM_ERR_INVALID_ARG;
   const long long L = (long long)s->n_obs + (long long)s->n_frames * s->n_spatial + s->n_action;
   if (L > (1 << 24) || (long long)s->batch * L > (1ll << 30)) return SWAM_ERR_UNSUPPORTED;
+  // samples are a grid dimension of most kernels (times the chunks of 128 action queries in the one-pass scorer)
+  if ((long long)s->batch * ((s->n_action + 127) / 128) > 65535) return SWAM_ERR_UNSUPPORTED;
 
   swam_ctx* c = new (std::nothrow) swam_ctx();
   if (!c) return SWAM_ERR_INVALID_ARG;

@@ -81,6 +81,7 @@ def test_shapes_beyond_the_selection_kernels_shared_memory_are_rejected(lib):
     # F * N_s scores (two maps) + keys + flags must fit one SM's shared memory
     assert _create(lib, n_frames=8, n_spatial=8192, n_action=32, k_core=10, k_anchor=10) == swam.ERR_UNSUPPORTED
     assert _create(lib, n_obs=1 << 25) == swam.ERR_UNSUPPORTED            # sequence length limit
+    assert _create(lib, batch=70000, n_obs=0, n_frames=1, n_spatial=64, n_action=4, k_core=8, k_anchor=8) == swam.ERR_UNSUPPORTED   # samples are a grid dimension
 
 
 def test_degree4_exp2_polynomial_bound():
