@@ -398,7 +398,11 @@ cudaError_t launch_lse_tc(const Dims& d, const CUtensorMap& mq, const CUtensorMa
 
 }  // namespace
 
-bool score_one_pass_supported(const Dims& d) { return d.dtype != 0 && (d.D == 64 || d.D == 128); }
+bool score_one_pass_supported(const Dims& d) {
+  // bf16 on the tensor-core path; the second kernel keeps N_h * g normalisers in (default-sized) shared memory
+  return d.dtype != 0 && (d.D == 64 || d.D == 128) &&
+         ((size_t)d.N_h * d.g + kFinSlots * kFinKeys) * sizeof(float) <= 48 * 1024;
+}
 
 size_t score_logits_bytes(const Dims& d) {
   return score_one_pass_supported(d) ? (size_t)d.B * d.N_h * d.F * d.N_s * d.g * sizeof(float) : 0;
