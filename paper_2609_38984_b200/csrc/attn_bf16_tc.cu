@@ -33,7 +33,10 @@ struct TcParams {
   float* partial;      // split items: [slot][2 tiles][128 rows][D + 4]: unnormalised O, then reference max and sum
   const int32_t* pack_map;  // gather mode: [B, n] row of the full tensors that each attended row stands for
   int n_full;               // gather modes: rows per sample of the full tensors
-  int kv_rows;              // kGatherKV: rows of the 2-D view of K and V, B * n_full (a row coordinate beyond the tensor)
+  union {
+    int kv_rows;            // kGatherKV: rows of the 2-D view of K and V, B * n_full (a row coordinate beyond the tensor)
+    int direct_tiles;       // kGather: the first key tiles come from the full K and V (maps in the slots of map_q and map_o)
+  };
   const __nv_bfloat16* q_full;  // gather mode: the full [B, n_full, N_h, D] query tensor
   __nv_bfloat16* out_full;      // gather mode: the full [B, n_full, N_h, D] output tensor
   int lse_row0, lse_rows;
@@ -340,8 +343,14 @@ attn_bf16_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                           y[2], y[3]);
           } else {
             mbar_expect_tx(bar, C::kTileBytes);
+            // gather mode: the leading tiles (observed tokens, which the packed sequence shares with the full one) come
+            // straight from the full tensors, whose maps travel in the slots the direct mode uses for Q and the output
+            const CUtensorMap* mp = is_v ? &map_v : &map_k;
+            if constexpr (MODE == kGather) {
+              if (tile < p.direct_tiles) mp = is_v ? &map_o : &map_q;
+            }
             for (int db = 0; db < C::DB; ++db)
-              tma_load_4d(dst + db * C::kSubTile, is_v ? &map_v : &map_k, bar, db * 64, tile * kTile, h_kv, wk.b);
+              tma_load_4d(dst + db * C::kSubTile, mp, bar, db * 64, tile * kTile, h_kv, wk.b);
           }
         };
         // The first item's queries go first.  A later item's queries have to wait until the previous item's output has
@@ -934,14 +943,15 @@ cudaError_t launch_tc_v(const AttnArgs& a, const int32_t* pack_map, int n_full, 
   } else if (!make_map(&mk, a.k, a.B, a.n, a.N_kv, D) || !make_map(&mv, a.v, a.B, a.n, a.N_kv, D)) {
     return cudaErrorInvalidValue;
   }
+  // The gather modes neither load Q nor store the output through tensor maps (gathering warps and plain stores do):
+  // in kGather mode the two slots carry the maps of the full K and V for the leading key tiles that are read from there.
+  const bool direct_kv = MODE == kGather && a.direct_rows >= kTile && a.k_full && a.v_full;
   if (MODE != kDirect) {
-    mo = mk;   // not used by the kernel: the scattering epilogue writes the full output tensor with plain stores
-  } else if (!make_map(&mo, a.out, a.B, a.n, a.N_h, D)) {
-    return cudaErrorInvalidValue;
-  }
-  if (MODE != kDirect) {
-    mq = mk;   // not used by the kernel
-  } else if (!make_map(&mq, a.q, a.B, a.n, a.N_h, D)) {
+    mq = mk;
+    mo = mv;
+    if (direct_kv && (!make_map(&mq, a.k_full, a.B, n_full, a.N_kv, D) || !make_map(&mo, a.v_full, a.B, n_full, a.N_kv, D)))
+      return cudaErrorInvalidValue;
+  } else if (!make_map(&mo, a.out, a.B, a.n, a.N_h, D) || !make_map(&mq, a.q, a.B, a.n, a.N_h, D)) {
     return cudaErrorInvalidValue;
   }
   cudaError_t e = cudaFuncSetAttribute(attn_bf16_tc_kernel<D, MODE, VIS>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<D>::kSmemBytes);
@@ -965,6 +975,7 @@ cudaError_t launch_tc_v(const AttnArgs& a, const int32_t* pack_map, int n_full, 
   TcParams p{
       a.lse, status, partial, pack_map, n_full, a.B * n_full, (const __nv_bfloat16*)a.q, (__nv_bfloat16*)a.out, a.lse_row0, a.lse_rows, a.n, a.N_h, a.N_h / a.N_kv, pairs, n_whole + (splits ? rem * splits : 0), n_whole, splits, per,
       a.scale * kLog2e, a.obs_end, a.fut_end, a.lim[0], a.lim[1], a.lim[2]};
+  if (MODE == kGather) p.direct_tiles = direct_kv ? a.direct_rows / kTile : 0;
   const int grid = p.total_work < sms ? p.total_work : sms;   // one CTA per SM; each walks through its share of the work
   ++*launches;
   attn_bf16_tc_kernel<D, MODE, VIS><<<grid, kThreadsTc, TcCfg<D>::kSmemBytes, st>>>(mq, mk, mv, mo, p);

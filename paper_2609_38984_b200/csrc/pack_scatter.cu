@@ -26,7 +26,9 @@ struct RowCopyParams {
   const int32_t* dst_idx;  // [B, n_rows] row of dst for each listed row, or nullptr (identity)
   int* status;
   int n_tensors;
-  int n_rows;       // listed rows per sample
+  int n_rows;       // listed rows per sample that this launch copies: first_row .. first_row + n_rows - 1
+  int first_row;    // first listed row copied
+  int idx_rows;     // listed rows per sample in the maps (their stride from sample to sample)
   int src_rows;     // rows per sample in src
   int dst_rows;     // rows per sample in dst
   int row_bytes;
@@ -82,11 +84,11 @@ __global__ void __launch_bounds__(kWarps * 32, 1) row_copy_bulk_kernel(const Row
       z = (int)(row_id / rows_per_tensor);
       const long long br = row_id - (long long)z * rows_per_tensor;
       const long long b = br / p.n_rows;
-      const long long lr = br - b * p.n_rows;
+      const long long lr = p.first_row + (br - b * p.n_rows);
       long long srow = lr, drow = lr;
       bool valid = true;
-      if (p.src_idx) { srow = p.src_idx[br]; valid = srow >= 0 && srow < p.src_rows; }
-      if (p.dst_idx) { drow = p.dst_idx[br]; valid = valid && drow >= 0 && drow < p.dst_rows; }
+      if (p.src_idx) { srow = p.src_idx[b * p.idx_rows + lr]; valid = srow >= 0 && srow < p.src_rows; }
+      if (p.dst_idx) { drow = p.dst_idx[b * p.idx_rows + lr]; valid = valid && drow >= 0 && drow < p.dst_rows; }
       if (valid) {
         s_off = (b * p.src_rows + srow) * (long long)p.row_bytes + (long long)seg * p.seg_bytes;
         d_off = (b * p.dst_rows + drow) * (long long)p.row_bytes + (long long)seg * p.seg_bytes;
@@ -196,8 +198,8 @@ cudaError_t launch_row_copy(RowCopyParams& p, int batch, cudaStream_t st) {
 }  // namespace
 
 cudaError_t launch_pack(const Dims& d, const void* const src[3], void* const dst[3], const int32_t* pack_map,
-                        int* status, cudaStream_t st, int* launches) {
-  if (d.Lp == 0) return cudaSuccess;
+                        int* status, cudaStream_t st, int* launches, int first_row) {
+  if (d.Lp - first_row <= 0) return cudaSuccess;
   const int eb = d.dtype == 0 ? 4 : 2;
   // tensors with the same row size share a launch: Q has N_h heads per row, K and V have N_kv
   const int rows_of[3] = {d.N_h * d.D * eb, d.N_kv * d.D * eb, d.N_kv * d.D * eb};
@@ -214,7 +216,8 @@ cudaError_t launch_pack(const Dims& d, const void* const src[3], void* const dst
         done[i] = true;
       }
     p.src_idx = pack_map; p.dst_idx = nullptr; p.status = status;
-    p.n_tensors = n; p.n_rows = d.Lp; p.src_rows = d.L; p.dst_rows = d.Lp;
+    p.n_tensors = n; p.n_rows = d.Lp - first_row; p.first_row = first_row; p.idx_rows = d.Lp;
+    p.src_rows = d.L; p.dst_rows = d.Lp;
     p.row_bytes = rows_of[first];
     ++*launches;
     cudaError_t e = launch_row_copy(p, d.B, st);
@@ -301,7 +304,7 @@ cudaError_t launch_scatter(const Dims& d, const void* out_p, const int32_t* pack
     RowCopyParams p{};
     p.src[0] = (const unsigned char*)out_p; p.dst[0] = (unsigned char*)out;
     p.src_idx = nullptr; p.dst_idx = pack_map; p.status = status;
-    p.n_tensors = 1; p.n_rows = d.Lp; p.src_rows = d.Lp; p.dst_rows = d.L;
+    p.n_tensors = 1; p.n_rows = d.Lp; p.first_row = 0; p.idx_rows = d.Lp; p.src_rows = d.Lp; p.dst_rows = d.L;
     p.row_bytes = row_bytes;
     ++*launches;
     return launch_row_copy(p, d.B, st);

@@ -22,6 +22,7 @@ struct swam_ctx {
   size_t off_status, off_scores, off_quality, off_lse, off_sel, off_pack, off_inv, off_scratch, off_qp, off_kp,
       off_vp, off_op, off_attn, off_logits, off_lam2, off_counters, attn_scratch, ws_need;
   bool has_selection;
+  bool maps_own;     // the cached maps were built by this context's selection kernel (not installed or imported)
   int attn_variant;  // SWAM_ATTN_AUTO | SWAM_ATTN_WARP_MMA
   int sparse_path;   // SWAM_SPARSE_FUSED | SWAM_SPARSE_STAGED
   int host_rows;     // SWAM_HOST_ROWS_RETAINED | SWAM_HOST_ROWS_ALL: what a reuse step with host buffers brings in
@@ -254,6 +255,7 @@ int swam_bind_workspace(swam_ctx* c, void* dev_ptr, size_t bytes) {
   c->ws = (unsigned char*)dev_ptr;
   c->ws_bytes = bytes;
   c->has_selection = false;
+  c->maps_own = false;
   return SWAM_OK;
 }
 
@@ -462,6 +464,7 @@ int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t 
     count(c);
     if (e != cudaSuccess) return fail_cuda(c, e, "select launch");
     c->has_selection = true;
+    c->maps_own = true;     // built by the selection kernel: the observed rows lead the packed sequence in order
   }
   if (mode != SWAM_REFRESH_FULL && c->sparse_path != SWAM_SPARSE_STAGED && d.dtype == SWAM_BF16 && d.D >= 64 &&
       c->attn_variant == SWAM_ATTN_AUTO) {
@@ -473,13 +476,24 @@ int swam_step(swam_ctx* c, const void* q, const void* k, const void* v, int32_t 
     const bool gather_kv = c->sparse_path == SWAM_SPARSE_FUSED_KV;
     const void* kp = k;
     const void* vp = v;
+    // The observed tokens lead the packed sequence as they lead the full one: whole key tiles of them are read from
+    // the full K and V and are left out of the pack.
+    const int direct_rows = (gather_kv || !c->maps_own) ? 0 : (d.n_obs / 128) * 128;
     if (!gather_kv) {
       kp = c->ws + c->off_kp;
       vp = c->ws + c->off_vp;
-      if (int r = swam_pack(c, nullptr, k, v, pm, nullptr, c->ws + c->off_kp, c->ws + c->off_vp, stream)) return r;
+      Range stage_pack("swam_pack");
+      const void* src[3] = {nullptr, k, v};
+      void* dst[3] = {nullptr, c->ws + c->off_kp, c->ws + c->off_vp};
+      cudaError_t e = launch_pack(d, src, dst, pm, (int*)(c->ws + c->off_status), st, &c->launches_i, direct_rows);
+      count(c);
+      if (e != cudaSuccess) return fail_cuda(c, e, "pack launch");
     }
     Range stage("packed_attention");
     AttnArgs a{q, kp, vp, out, nullptr, 0, 0, d.B, d.Lp, d.N_h, d.D, d.scale, d.N_kv};
+    a.k_full = k;
+    a.v_full = v;
+    a.direct_rows = direct_rows;
     set_visibility(c, a);
     cudaError_t e = launch_attn_bf16_tc_gather(a, pm, d.L, gather_kv, (int*)(c->ws + c->off_status), c->ws + c->off_attn,
                                                c->attn_scratch, st, &c->launches_i);
@@ -598,6 +612,7 @@ int swam_set_selection(swam_ctx* c, const int32_t* sel_idx, const int32_t* pack_
     e = cudaMemcpyAsync(c->ws + c->off_inv, inv_map, (size_t)d.B * d.L * sizeof(int32_t), cudaMemcpyDeviceToDevice, st);
   if (e != cudaSuccess) return fail_cuda(c, e, "swam_set_selection");
   c->has_selection = true;
+  c->maps_own = false;     // installed maps are the caller's: the observed rows need not lead them
   return SWAM_OK;
 }
 
@@ -627,6 +642,7 @@ int swam_state_import(swam_ctx* c, const void* dev_buf, void* stream) {
                                   (cudaStream_t)stream);
   if (e != cudaSuccess) return fail_cuda(c, e, "swam_state_import");
   c->has_selection = true;
+  c->maps_own = false;     // restored maps: their origin is not known
   return SWAM_OK;
 }
 

@@ -162,8 +162,9 @@ cudaError_t launch_aggregate(const Dims& d, const float* layer_scores, const flo
 
 // ---- pack_scatter.cu ------------------------------------------------------
 // dst[b, p] = src[b, map[b,p]] for up to three tensor pairs (row_bytes per row).
+// first_row: the first listed row to copy (rows before it are left out of the launch)
 cudaError_t launch_pack(const Dims& d, const void* const src[3], void* const dst[3], const int32_t* pack_map,
-                        int* status, cudaStream_t st, int* launches);
+                        int* status, cudaStream_t st, int* launches, int first_row = 0);
 // in place: out[b, map[b,p]] = out_p[b,p];  blend: out[b,t] = inv[b,t] >= 0 ? out_p[b,inv[b,t]] : cached[b,t]
 // rows pack_map names, from full tensors in device-mapped host memory to the same rows of full tensors in device memory
 cudaError_t launch_host_rows(const Dims& d, const void* const src[3], void* const dst[3], const int32_t* pack_map,
@@ -189,6 +190,12 @@ struct AttnArgs {
   int B, n, N_h, D;  // n = sequence length of this call
   float scale;
   int N_kv;          // heads of k and v (q and out have N_h); query head h reads head h / (N_h / N_kv)
+  // Gather mode of the tensor-core kernel: the first direct_rows rows (a multiple of 128) of the packed K and V are the
+  // same rows of the full tensors k_full and v_full (the observed tokens lead both sequences), so the kernel reads those
+  // key tiles from the full tensors and the packed ones need not hold them.  0 = every tile comes from k and v.
+  const void* k_full = nullptr;
+  const void* v_full = nullptr;
+  int direct_rows = 0;
   // Segment-prefix visibility: rows [0, obs_end) see the first lim[0] keys, rows [obs_end, fut_end) the first lim[1],
   // the rest the first lim[2].  Full visibility: every lim = n (then obs_end and fut_end do not matter).
   int obs_end, fut_end, lim[3];

@@ -484,9 +484,10 @@ def test_light_refresh_step():
     small(batch=2),
     small("larger_imagination", n_obs=40, grid_h=7, grid_w=9, n_heads=2),
     small("larger_imagination", n_obs=300, grid_h=12, grid_w=11, n_heads=2, keep=0.5),   # whole tiles of observed rows
+    small(n_obs=260, batch=2, n_heads=4, n_kv_heads=2),                                    # the same at head dim 64, grouped heads
     small(keep=1.0),
     small(keep=0.0),
-], ids=["d64", "d128", "d128_long_obs", "keep_all", "keep_none"])
+], ids=["d64", "d128", "d128_long_obs", "d64_long_obs_gqa", "keep_all", "keep_none"])
 @pytest.mark.parametrize("mode", ["reuse", "light"])
 def test_fused_sparse_step_equals_staged_bit_for_bit(wl, mode):
     """Packed attention with the scatter and the query gather fused in, the same with the key and value rows gathered
