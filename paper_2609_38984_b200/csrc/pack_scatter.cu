@@ -236,15 +236,16 @@ struct HostRowsParams {
   const int32_t* idx;   // [B, n_idx] rows to bring
   int* status;
   int n_tensors, n_idx, rows, chunks;   // rows per sample of the full tensors, 16-byte chunks per row
-  long long total;                      // B * n_idx
+  int first, count;                     // listed rows first .. first + count - 1 of every sample are brought
+  long long total;                      // B * count
 };
 
 __global__ void __launch_bounds__(256) host_rows_kernel(const HostRowsParams p) {
   const int lane = threadIdx.x & 31;
   const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
   for (long long it = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; it < p.total; it += n_warps) {
-    const long long b = it / p.n_idx;
-    const int row = p.idx[it];
+    const long long b = it / p.count;
+    const int row = p.idx[b * p.n_idx + p.first + (it - b * p.count)];
     if (row < 0 || row >= p.rows) {
       if (lane == 0) atomicOr(p.status, ST_BAD_MAP);
       continue;
@@ -267,8 +268,8 @@ __global__ void __launch_bounds__(256) host_rows_kernel(const HostRowsParams p) 
 }
 
 cudaError_t launch_host_rows(const Dims& d, const void* const src[3], void* const dst[3], const int32_t* pack_map,
-                             int* status, cudaStream_t st, int* launches) {
-  if (d.Lp == 0) return cudaSuccess;
+                             int* status, cudaStream_t st, int* launches, int first_row) {
+  if (d.Lp - first_row <= 0) return cudaSuccess;
   const int eb = d.dtype == 0 ? 4 : 2;
   const int rows_of[3] = {d.N_h * d.D * eb, d.N_kv * d.D * eb, d.N_kv * d.D * eb};
   bool done[3] = {false, false, false};
@@ -285,7 +286,8 @@ cudaError_t launch_host_rows(const Dims& d, const void* const src[3], void* cons
       }
     p.idx = pack_map; p.status = status;
     p.n_tensors = n; p.n_idx = d.Lp; p.rows = d.L; p.chunks = rows_of[first] / 16;
-    p.total = (long long)d.B * d.Lp;
+    p.first = first_row; p.count = d.Lp - first_row;
+    p.total = (long long)d.B * p.count;
     ++*launches;
     const long long need = (p.total + 7) / 8;
     const long long cap = (long long)sm_count() * 8;

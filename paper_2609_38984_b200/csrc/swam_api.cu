@@ -35,6 +35,7 @@ struct swam_ctx {
   cudaEvent_t ev_h2d[3], ev_done[3];  // per input slot: inputs arrived / step finished with the slot
   cudaEvent_t ev_d2h;                 // the previous result has left the staged output
   cudaEvent_t ev_pre;                 // everything the caller's stream held when a reuse step with host buffers was called
+  cudaEvent_t ev_obs;                 // the observed rows of a reuse step's inputs have arrived (plain copies on s_in)
   int64_t host_steps;
   int launches_i;
   int64_t launches;
@@ -231,6 +232,7 @@ int swam_destroy(swam_ctx* ctx) {
     for (int i = 0; i < 3; ++i) { cudaEventDestroy(ctx->ev_h2d[i]); cudaEventDestroy(ctx->ev_done[i]); }
     cudaEventDestroy(ctx->ev_d2h);
     cudaEventDestroy(ctx->ev_pre);
+    cudaEventDestroy(ctx->ev_obs);
   }
   delete ctx;
   return SWAM_OK;
@@ -281,6 +283,7 @@ int swam_bind_host_io(swam_ctx* c, void* dev_ptr, size_t bytes) {
     }
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_d2h, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_pre, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_obs, cudaEventDisableTiming);
     if (e != cudaSuccess) return fail_cuda(c, e, "swam_bind_host_io: stream/event creation");
   }
   c->io = (unsigned char*)dev_ptr;
@@ -552,6 +555,21 @@ int swam_step_host(swam_ctx* c, const void* q_host, const void* k_host, const vo
   cudaStream_t s_copy = retained_only ? c->s_rows : c->s_in;
   cudaError_t e = cudaStreamWaitEvent(s_copy, c->ev_done[slot], 0);   // the step three calls ago has read this slot
   if (retained_only) {
+    // The observed rows are retained whatever the selection and lead every sample in one block: they travel as plain
+    // strided copies on the whole-copy stream at once (they need not wait for the maps).  With maps that this context
+    // did not build itself the block is not assumed and the kernel fetches every listed row.
+    const int n_block = c->maps_own ? c->d.n_obs : 0;
+    if (n_block > 0) {
+      const size_t row = fb / ((size_t)c->d.B * c->d.L), row_kv = kvb / ((size_t)c->d.B * c->d.L);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(c->s_in, c->ev_done[slot], 0);
+      if (e == cudaSuccess)
+        e = cudaMemcpy2DAsync(dq, c->d.L * row, q_host, c->d.L * row, n_block * row, c->d.B, cudaMemcpyHostToDevice, c->s_in);
+      if (e == cudaSuccess)
+        e = cudaMemcpy2DAsync(dk, c->d.L * row_kv, k_host, c->d.L * row_kv, n_block * row_kv, c->d.B, cudaMemcpyHostToDevice, c->s_in);
+      if (e == cudaSuccess)
+        e = cudaMemcpy2DAsync(dv, c->d.L * row_kv, v_host, c->d.L * row_kv, n_block * row_kv, c->d.B, cudaMemcpyHostToDevice, c->s_in);
+      if (e == cudaSuccess) e = cudaEventRecord(c->ev_obs, c->s_in);
+    }
     // the maps are final once everything already on the caller's stream has run (the previous step, or a selection
     // installed since)
     if (e == cudaSuccess) e = cudaEventRecord(c->ev_pre, st);
@@ -559,9 +577,10 @@ int swam_step_host(swam_ctx* c, const void* q_host, const void* k_host, const vo
     if (e == cudaSuccess) {
       void* dst[3] = {dq, dk, dv};
       e = launch_host_rows(c->d, mapped, dst, (const int32_t*)(c->ws + c->off_pack), (int*)(c->ws + c->off_status), s_copy,
-                           &c->launches_i);
+                           &c->launches_i, n_block);
       count(c);
     }
+    if (e == cudaSuccess && n_block > 0) e = cudaStreamWaitEvent(s_copy, c->ev_obs, 0);
   } else {
     if (e == cudaSuccess) e = cudaMemcpyAsync(dq, q_host, fb, cudaMemcpyHostToDevice, s_copy);
     if (e == cudaSuccess) e = cudaMemcpyAsync(dk, k_host, kvb, cudaMemcpyHostToDevice, s_copy);

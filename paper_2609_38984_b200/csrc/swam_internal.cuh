@@ -167,8 +167,9 @@ cudaError_t launch_pack(const Dims& d, const void* const src[3], void* const dst
                         int* status, cudaStream_t st, int* launches, int first_row = 0);
 // in place: out[b, map[b,p]] = out_p[b,p];  blend: out[b,t] = inv[b,t] >= 0 ? out_p[b,inv[b,t]] : cached[b,t]
 // rows pack_map names, from full tensors in device-mapped host memory to the same rows of full tensors in device memory
+// (first_row: the first listed row to bring)
 cudaError_t launch_host_rows(const Dims& d, const void* const src[3], void* const dst[3], const int32_t* pack_map,
-                             int* status, cudaStream_t st, int* launches);
+                             int* status, cudaStream_t st, int* launches, int first_row = 0);
 cudaError_t launch_scatter(const Dims& d, const void* out_p, const int32_t* pack_map, const int32_t* inv_map,
                            const void* cached, void* out, int* status, cudaStream_t st, int* launches);
 
