@@ -380,6 +380,16 @@ def measure_workload(wl0, args, rank, local_rank, world, device, peaks, peak_kin
                                                                 S())),
             "light_refresh_step": stage(step_call(swam.REFRESH_LIGHT), long_s / 3),
         })
+        # several profiled layers (Eq. 3, Eq. 9, Eq. 11): six layers' score maps and qualities -> core map over the
+        # three best layers and anchor map over all, then the selection from the two maps
+        n_layers, k_layer = 6, 3
+        layer_s = torch.stack([scores[i % N_ROT] for i in range(n_layers)]).contiguous()
+        layer_q = torch.rand((n_layers, B, 3), device=device, dtype=torch.float32)
+        v_core, v_all, core_layers = ctx.aggregate(layer_s, layer_q, k_layer)
+        stage_us["aggregate_6_layers"] = stage(lambda i: lambda: lib.swam_aggregate(
+            ctx.ctx, P(layer_s), P(layer_q), n_layers, k_layer, P(v_core), P(v_all), P(core_layers), S()))
+        stage_us["select_two_maps"] = stage(lambda i: lambda: lib.swam_select_maps(
+            ctx.ctx, P(v_core), P(v_all), P(sel), P(pm), P(im), S()))
     ctx.check()
     algo = {  # algorithmic bytes / flops per launch
         "score": ("hbm", B * (fut * row_kv + wl.n_action * row + fut * 4)),
@@ -415,6 +425,12 @@ def measure_workload(wl0, args, rank, local_rank, world, device, peaks, peak_kin
                             "launch_floor_us": round(stage_us["launch_floor"], 2),
                             "ratio_to_launch_floor": round(stage_us["select"] / stage_us["launch_floor"], 2),
                             "bytes": int(B * (fut * 4 + (wl.n_frames * wl.k_keep + Lp + L) * 4))}
+    if "aggregate_6_layers" in stage_us:
+        agg_bytes = B * fut * 4 * (6 + 2)
+        stages["aggregate_6_layers"] = {"us": round(stage_us["aggregate_6_layers"], 2), "bound": "latency", "bytes": int(agg_bytes),
+                                        "ratio_to_launch_floor": round(stage_us["aggregate_6_layers"] / stage_us["launch_floor"], 2)}
+        stages["select_two_maps"] = {"us": round(stage_us["select_two_maps"], 2), "bound": "latency",
+                                     "ratio_to_launch_floor": round(stage_us["select_two_maps"] / stage_us["launch_floor"], 2)}
     for name in ("full_step", "sparse_step", "sparse_step_kv_gathered_in_kernel", "light_refresh_step"):
         if name in stage_us:
             stages[name] = {"us": round(stage_us[name], 2)}
