@@ -390,6 +390,13 @@ def measure_workload(wl0, args, rank, local_rank, world, device, peaks, peak_kin
             ctx.ctx, P(layer_s), P(layer_q), n_layers, k_layer, P(v_core), P(v_all), P(core_layers), S()))
         stage_us["select_two_maps"] = stage(lambda i: lambda: lib.swam_select_maps(
             ctx.ctx, P(v_core), P(v_all), P(sel), P(pm), P(im), S()))
+        if wl.dtype == W.BF16 and wl.head_dim >= 64:
+            # restricted visibility (App. A.2's constraints in the segment-prefix form): observed rows see the observed
+            # tokens only, future rows the observed and future ones, action rows everything
+            ctx.set_visibility(swam.SEES_OBSERVED, swam.SEES_FUTURE, swam.SEES_ALL)
+            stage_us["full_step_segment_visibility"] = stage(step_call(swam.REFRESH_FULL), long_s / 3)
+            stage_us["sparse_step_segment_visibility"] = stage(step_call(swam.REUSE), long_s / 3)
+            ctx.set_visibility(swam.SEES_ALL, swam.SEES_ALL, swam.SEES_ALL)
     ctx.check()
     algo = {  # algorithmic bytes / flops per launch
         "score": ("hbm", B * (fut * row_kv + wl.n_action * row + fut * 4)),
@@ -431,7 +438,8 @@ def measure_workload(wl0, args, rank, local_rank, world, device, peaks, peak_kin
                                         "ratio_to_launch_floor": round(stage_us["aggregate_6_layers"] / stage_us["launch_floor"], 2)}
         stages["select_two_maps"] = {"us": round(stage_us["select_two_maps"], 2), "bound": "latency",
                                      "ratio_to_launch_floor": round(stage_us["select_two_maps"] / stage_us["launch_floor"], 2)}
-    for name in ("full_step", "sparse_step", "sparse_step_kv_gathered_in_kernel", "light_refresh_step"):
+    for name in ("full_step", "sparse_step", "sparse_step_kv_gathered_in_kernel", "light_refresh_step",
+                 "full_step_segment_visibility", "sparse_step_segment_visibility"):
         if name in stage_us:
             stages[name] = {"us": round(stage_us[name], 2)}
 
